@@ -1,0 +1,94 @@
+"""Seeded synthetic inputs shared by the tests, the benchmark and the CPU checker.
+
+Only random draws and data movement live here -- none of the arithmetic of the
+aggregation scheme.  Everything is generated on the host with NumPy's
+`Generator(PCG64(seed))` and handed, as data, to whoever consumes it.
+
+The value models follow the synthetic linear-regression recipe of the paper's
+Section V (features and true model Gaussian, labels = features . model + Gaussian
+noise); the aggregation-only workloads use Gaussian partition gradients, and the
+integer mode uses uniform integers.
+"""
+from __future__ import annotations
+
+import numpy as np
+
+
+def _rng(seed: int) -> np.random.Generator:
+    return np.random.Generator(np.random.PCG64(seed))
+
+
+def partition_gradients(P: int, d: int, seed: int, std: float = 1.0) -> np.ndarray:
+    """One fp32 gradient vector per atomic data partition, N(0, std^2), shape [P, d]."""
+    g = _rng(seed).standard_normal((P, d), dtype=np.float32)
+    if std != 1.0:
+        g *= np.float32(std)
+    return g
+
+
+def integer_gradients(P: int, d: int, seed: int, bound: int = 1 << 10) -> np.ndarray:
+    """One int32 gradient vector per partition, uniform in [-bound, bound]."""
+    return _rng(seed).integers(-bound, bound + 1, size=(P, d), dtype=np.int32)
+
+
+def linreg_partitions(P: int, rows: int, d: int, seed: int, x_std: float = 1.0,
+                      noise_std: float = 0.01):
+    """P partitions of a linear-regression data set.
+
+    Returns (X [P, rows, d] fp32 ~ N(0, x_std^2), y [P, rows] fp32, w_star [d] fp32)
+    with y = X w_star + noise_std * N(0, 1), the products formed in fp64 and
+    rounded once to fp32.
+    """
+    rng = _rng(seed)
+    w_star = rng.standard_normal(d, dtype=np.float32)
+    X = rng.standard_normal((P, rows, d), dtype=np.float32)
+    if x_std != 1.0:
+        X *= np.float32(x_std)
+    noise = rng.standard_normal((P, rows), dtype=np.float32)
+    y = np.empty((P, rows), dtype=np.float32)
+    for p in range(P):
+        y[p] = (X[p].astype(np.float64) @ w_star.astype(np.float64)
+                + noise_std * noise[p].astype(np.float64)).astype(np.float32)
+    return X, y, w_star
+
+
+def model_vector(d: int, seed: int) -> np.ndarray:
+    """A start model w_0 ~ N(0, I), fp32."""
+    return _rng(seed).standard_normal(d, dtype=np.float32)
+
+
+def group_count(n: int, L: int) -> int:
+    """Sibling groups of an (n, L) tree: one per parent, the master included."""
+    return sum(n ** l for l in range(L))
+
+
+def straggler_masks(n: int, L: int, s: int, batch: int, seed: int,
+                    exactly_s: bool = False) -> np.ndarray:
+    """Random straggler patterns, shape [batch, groups], dtype uint32.
+
+    Bit j of masks[b, g] marks child j of sibling group g as a straggler.  Per
+    group the number of stragglers is s (exactly_s) or uniform on {0..s}; the
+    straggling children are a uniform subset of that size.
+    """
+    rng = _rng(seed)
+    groups = group_count(n, L)
+    masks = np.zeros((batch, groups), dtype=np.uint32)
+    for b in range(batch):
+        for g in range(groups):
+            k = s if exactly_s else int(rng.integers(0, s + 1))
+            chosen = rng.choice(n, size=k, replace=False) if k else []
+            bits = 0
+            for j in chosen:
+                bits |= 1 << int(j)
+            masks[b, g] = bits
+    return masks
+
+
+def replicate_into_slots(G_parts: np.ndarray, slot_partition: np.ndarray) -> np.ndarray:
+    """Copy partition gradients into per-node slots: out[v, j] = G_parts[slot_partition[v, j]].
+
+    Every node that holds a partition computes the same gradient for it, so the
+    slot buffer of an aggregation-only workload is this gather (pure data
+    movement; `slot_partition` comes from whoever planned the allocation).
+    """
+    return G_parts[np.asarray(slot_partition, dtype=np.int64)]
