@@ -1,0 +1,397 @@
+#!/usr/bin/env python
+"""Benchmark of the coded tree aggregation on B200.
+
+A step is one cr_aggregate call (encode of every consumed node, masked decode at every level,
+root recovery) on one batch of straggler masks over synthetic partition gradients that are already
+resident in HBM.  The default workload is the large-gradient configuration (n=5, L=2, s=2,
+d=2^24, 270 slots = 17.3 GB, exactly two stragglers per sibling group); `--workload` selects the
+others.  Prints one JSON line (see README of the repo for the keys).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg4] [--impl reference]
+
+With N > 1 (launched by torch.distributed.run) every rank runs an independent replica on its own
+GPU -- the path has no exchange step -- and rank 0 reports the sum of units over the slowest rank's
+time.  `--impl reference` times the CPU oracle instead (rank 0 only).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_1902_01981_b200 import inputs  # noqa: E402
+
+METRIC = "CR aggregation GB/s (fraction of HBM peak) and coded iterations/sec"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the timed kernel, from the ncu capture
+# summarised under profiles/ (None until a capture of the current kernel exists).
+NCU_TRAFFIC_BYTES = {}
+
+
+def peak_hbm():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+# ----------------------------------------------------------------------------- multi-rank plumbing
+
+def combine_ranks(elapsed_s: float, units: float, world: int, dist=None, device=None):
+    """Whole-job figure: total units of all ranks over the slowest rank's time."""
+    if world == 1 or dist is None:
+        return elapsed_s, units
+    import torch
+    t = torch.tensor([elapsed_s], dtype=torch.float64, device=device)
+    u = torch.tensor([units], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(gpu_index), f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                         stdout=self.file, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.file.read().splitlines():
+            cols = [c.strip() for c in line.split(",")]
+            if len(cols) < 9:
+                continue
+            try:
+                sm.append(float(cols[1]))
+                mx.append(float(cols[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, cols[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.file.close()
+        os.unlink(self.file.name)
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons),
+                       samples=len(sm))
+        return out
+
+
+# ----------------------------------------------------------------------------- CPU oracle legs
+
+def oracle_sample(cfg, d_sample: int, steps: int, warmup: int, seed_shift: int = 0):
+    """Times the CPU oracle, as it stands, on the first `d_sample` columns of the workload.
+    Returns (seconds per step, algorithmic bytes per step, results of the last step, masks used)."""
+    from oracle import cr_oracle as O
+    from oracle import cr_setup
+    code, local, _ = cr_setup.setup(cfg)
+    batch = cfg.get("batch", 1)
+    G = inputs.partition_gradients(cfg["P"], d_sample, cfg["seed"] + seed_shift, cfg.get("std", 1.0))
+    masks = inputs.straggler_masks(cfg["n"], cfg["L"], cfg["s"], (steps + warmup) * batch, cfg["mask_seed"],
+                                   cfg.get("exactly_s", False)).reshape(steps + warmup, batch, -1)
+    m = len(local[0])
+    times, nbytes, last = [], [], None
+    for it in range(steps + warmup):
+        t0 = time.perf_counter()
+        last = [O.execute(code, local, G, masks[it, b]) for b in range(batch)]
+        dt = time.perf_counter() - t0
+        if it >= warmup:
+            times.append(dt)
+            union = set()
+            for b in range(batch):
+                union |= set(O.used_nodes(code, masks[it, b]))
+            nbytes.append(4 * d_sample * (m * len(union) + batch))
+    return float(np.mean(times)), float(np.mean(nbytes)), last, masks[-1]
+
+
+def host_threads() -> int:
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def run_reference(args, cfg):
+    """The oracle as the reference arm: same metric and unit, bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    d_sample = min(cfg["d"], args.ref_columns)
+    sec, nbytes, _, _ = oracle_sample(cfg, d_sample, args.steps, args.warmup)
+    value = nbytes / sec / 1e9
+    sample = f"first {d_sample} of {cfg['d']} columns, every step a fresh straggler pattern"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(args.workload, cfg, None),
+        "iterations_per_s": 1.0 / sec,
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
+                         "host_threads_available": host_threads()},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ----------------------------------------------------------------------------- our arm
+
+def workload_config(name, cfg, extra):
+    out = {"workload": f"{name}: n={cfg['n']} L={cfg['L']} s={cfg['s']} code={cfg['code']} P={cfg['P']} "
+                       f"d={cfg['d']} batch={cfg.get('batch', 1)}",
+           "l2": "inputs larger than L2 (no flush needed)" if cfg["d"] * 4 * cfg["P"] > 126e6 else "L2 flushed between steps",
+           "parallelism": "independent replicas (no exchange step)"}
+    if extra:
+        out.update(extra)
+    return out
+
+
+def run_ours(args, cfg):
+    import torch
+    from paper_1902_01981_b200 import binding as B
+    from paper_1902_01981_b200 import build as cr_build
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        cr_build.build()
+    if dist is not None:
+        dist.barrier()
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+
+    is_int = args.dtype == "int32"
+    code_id = {"printed_3_1": B.CR_CODE_PAPER_3_1, "cyclic": B.CR_CODE_CYCLIC_RANDOM,
+               "repetition": B.CR_CODE_FRACTIONAL_REPETITION}[cfg["code"]]
+    plan = B.cr_plan_create(cfg["n"], cfg["L"], cfg["s"], cfg["P"], cfg["d"], code=code_id,
+                            dtype=B.CR_I32 if is_int else B.CR_F32, seed=0, device=local_rank)
+    if args.tune:
+        B.cr_plan_tune(plan, *[int(x) for x in args.tune.split(",")])
+    N, m, groups = B.cr_plan_num_nodes(plan), B.cr_plan_load(plan), B.cr_plan_num_groups(plan)
+    d, batch = cfg["d"], cfg.get("batch", 1)
+    tdtype = torch.int32 if is_int else torch.float32
+
+    # synthetic inputs: one vector per partition on the host, replicated into the slots on the device
+    if is_int:
+        G_parts = inputs.integer_gradients(cfg["P"], d, cfg["seed"] + rank, cfg.get("int_bound", 1 << 10))
+    else:
+        G_parts = inputs.partition_gradients(cfg["P"], d, cfg["seed"] + rank, cfg.get("std", 1.0))
+    part = torch.from_numpy(B.slot_partitions(plan).astype(np.int64).reshape(-1)).to(dev)
+    parts_dev = torch.from_numpy(G_parts).to(dev)
+    G_slots = torch.empty((N * m, d), dtype=tdtype, device=dev)
+    step_rows = max(1, (1 << 30) // (4 * d))
+    for r0 in range(0, N * m, step_rows):
+        torch.index_select(parts_dev, 0, part[r0:r0 + step_rows], out=G_slots[r0:r0 + step_rows])
+    del parts_dev
+    out = torch.zeros((batch, d), dtype=tdtype, device=dev)
+    total = args.steps + args.warmup
+    masks = inputs.straggler_masks(cfg["n"], cfg["L"], cfg["s"], total * batch, cfg["mask_seed"],
+                                   cfg.get("exactly_s", False)).reshape(total, batch, groups)
+    step_bytes = [B.cr_aggregate_bytes(plan, masks[i])[0] for i in range(total)]
+    need_flush = d * 4 * cfg["P"] <= 126e6
+    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if need_flush else None
+    stream = torch.cuda.current_stream()
+
+    def timed_run(flags, ws=None, steps=args.steps, warmup=args.warmup):
+        starts = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        stops = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        for i in range(warmup):
+            B.cr_aggregate(plan, G_slots, masks[i], out, flags, ws, stream)
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for i in range(steps):
+            if flush_buf is not None:
+                flush_buf.fill_(i & 0xff)
+            starts[i].record(stream)
+            B.cr_aggregate(plan, G_slots, masks[warmup + i], out, flags, ws, stream)
+            stops[i].record(stream)
+        torch.cuda.synchronize()
+        wall = time.perf_counter() - t0
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+        per = np.array([a.elapsed_time(b) for a, b in zip(starts, stops)]) * 1e-3
+        span = starts[0].elapsed_time(stops[-1]) * 1e-3
+        return per, (span if flush_buf is None else float(per.sum()))
+
+    # ---- the timed region: K steps of the fused kernel
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid).replace("GPU-", "")
+    except Exception:
+        gpu_id = local_rank
+    sampler = ClockSampler(gpu_id)
+    launches0 = B.cr_plan_launch_count(plan)
+    per, wall = timed_run(B.CR_AGG_FUSED)
+    launches = B.cr_plan_launch_count(plan) - launches0
+    clocks = sampler.stop()
+    assert B.cr_plan_device_status(plan) == B.CR_OK, "a device-side wait timed out"
+    # device time of the K steps: first start event to last stop event on the launching stream (with
+    # an L2 flush between steps: the sum of the per-step intervals, which leaves the flushes out)
+    elapsed = float(wall)
+    units = float(sum(step_bytes[args.warmup:]))
+    elapsed_all, units_all = combine_ranks(elapsed, units, world, dist, dev)
+    value = units_all / elapsed_all / 1e9
+    result_last = out.clone()
+
+    # ---- comparators on the same slots (rank 0 only, outside the timed region)
+    extras = {}
+    if rank == 0 and not args.no_extras:
+        ksteps = min(args.steps, 10)
+        bytes_k = float(np.mean(step_bytes[args.warmup:args.warmup + ksteps]))
+        for name, flags in (("fused_plain_loads", B.CR_AGG_FUSED_LDG), ("uncoded_sum_same_bytes", B.CR_AGG_UNCODED_SUM)):
+            p2, _ = timed_run(flags, steps=ksteps)
+            extras[name] = {"GB/s": bytes_k / float(p2.mean()) / 1e9, "ms_per_step": float(p2.mean()) * 1e3}
+        nws = B.cr_aggregate_workspace_bytes(plan, batch, B.CR_AGG_UNFUSED)
+        free, _ = torch.cuda.mem_get_info()
+        if nws < free - (2 << 30):
+            ws = torch.empty(nws, dtype=torch.uint8, device=dev)
+            p2, _ = timed_run(B.CR_AGG_UNFUSED, ws, steps=min(ksteps, 5))
+            extras["unfused_per_level"] = {"GB/s": bytes_k / float(p2.mean()) / 1e9, "ms_per_step": float(p2.mean()) * 1e3}
+            del ws
+        B.cr_aggregate(plan, G_slots, masks[total - 1], out, B.CR_AGG_FUSED, None, stream)
+        torch.cuda.synchronize()
+
+    # ---- end to end through the host-buffer entry point: H2D of the slots and D2H of the result
+    # inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        e2e_steps = max(1, min(args.e2e_steps, args.steps))
+        host_slots = torch.empty((N * m, d), dtype=tdtype, pin_memory=True)
+        host_slots.copy_(G_slots)
+        host_out = torch.empty((batch, d), dtype=tdtype, pin_memory=True)
+        torch.cuda.synchronize()
+        B.cr_aggregate_host(plan, host_slots, masks[0], host_out, G_slots, out, B.CR_AGG_FUSED, None, stream)
+        if dist is not None:
+            dist.barrier()
+        t0 = time.perf_counter()
+        for i in range(e2e_steps):
+            B.cr_aggregate_host(plan, host_slots, masks[args.warmup + i], host_out, G_slots, out, B.CR_AGG_FUSED,
+                                None, stream)
+        torch.cuda.synchronize()
+        e2e_elapsed = time.perf_counter() - t0
+        e2e_units = float(sum(step_bytes[args.warmup:args.warmup + e2e_steps]))
+        e2e_elapsed, e2e_units = combine_ranks(e2e_elapsed, e2e_units, world, dist, dev)
+        e2e = {"value": e2e_units / e2e_elapsed / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": int(N * m * d * 4 + masks[0].nbytes), "d2h_bytes_per_step": int(batch * d * 4),
+               "steps": e2e_steps, "ms_per_step": e2e_elapsed / e2e_steps * 1e3}
+        del host_slots
+
+    if rank == 0:
+        peak, peak_kind = peak_hbm()
+        avg_launch = float(per.mean())
+        avg_bytes = float(np.mean(step_bytes[args.warmup:]))
+        achieved = avg_bytes / avg_launch / 1e9
+        kern = "cr_fused_batch_tma_kernel" if batch > 1 else "cr_fused_tma_kernel"
+        traffic = NCU_TRAFFIC_BYTES.get((args.workload, args.dtype))
+        roofline = {"bound": "hbm", "kernel": kern, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                    "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / 8000.0,
+                    "traffic": traffic, "algorithmic_bytes_per_launch": avg_bytes,
+                    "avg_launch_ms": avg_launch * 1e3, "best_launch_ms": float(per.min()) * 1e3}
+        cpu = None
+        if not args.no_cpu_baseline:
+            d_sample = min(d, args.cpu_columns)
+            sec, nbytes, last, last_masks = oracle_sample(cfg, d_sample, args.cpu_steps, 1, seed_shift=rank) \
+                if not is_int else (None, None, None, None)
+            if sec is not None:
+                cpu = {"value": nbytes / sec / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+                       "sample": f"first {d_sample} of {d} columns, {args.cpu_steps} steps, NumPy fp64",
+                       "ms_per_step_on_sample": sec * 1e3, "host_threads_available": host_threads()}
+                # by-product: the GPU result for the same masks on those columns against the oracle
+                B.cr_aggregate(plan, G_slots, last_masks, out, B.CR_AGG_FUSED, None, stream)
+                torch.cuda.synchronize()
+                got = out[:, :d_sample].cpu().numpy().astype(np.float64)
+                worst = max(float(np.linalg.norm(got[b] - last[b]) / np.linalg.norm(last[b])) for b in range(batch))
+                cpu["gpu_rel_l2_on_sample"] = worst
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": elapsed_all / args.steps * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int32" if is_int else "f32", "data": "synthetic",
+            "config": workload_config(args.workload, cfg, {"slots_gb": N * m * d * 4 / 1e9, "tune": args.tune or "auto"}),
+            "iterations_per_s": world * args.steps / elapsed_all,
+            "patterns_per_s": world * args.steps * batch / elapsed_all,
+            "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
+            "clocks": clocks, "comparators": extras,
+        }
+        print(json.dumps(line), flush=True)
+    B.cr_plan_destroy(plan)
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg4", choices=[k for k, v in inputs.CONFIGS.items() if v["kind"] == "aggregate"])
+    ap.add_argument("--dtype", default="f32", choices=["f32", "int32"])
+    ap.add_argument("--tune", default="", help="consumer_warps,stages,ctas_per_sm,rows_per_box (0 = auto)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-extras", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-columns", type=int, default=1 << 21)
+    ap.add_argument("--cpu-steps", type=int, default=4)
+    ap.add_argument("--ref-columns", type=int, default=1 << 19)
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    cfg = dict(inputs.CONFIGS[args.workload])
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.gpus != world and world > 1:
+        args.gpus = world
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

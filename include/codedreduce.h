@@ -1,0 +1,205 @@
+/*
+ * codedreduce.h -- C ABI of the B200 coded tree aggregation library (libcodedreduce.so).
+ *
+ * The library simulates, on ONE GPU, the per-iteration gradient aggregation of
+ * CodedReduce (CR): N = n + n^2 + .. + n^L workers arranged in an (n, L)-regular
+ * tree below a master (Section III-A), every worker holding r_CR * P data
+ * partitions with combining coefficients (CR.Allocate, Algorithm 2; CompAlloc,
+ * Algorithm 1), every parent recovering a combination of its children's
+ * messages from any n-s of them with a gradient-coding decode row and adding
+ * its own coded gradient (CR.Execute, Algorithm 2), the master ending with the
+ * exact gradient sum of Eq. (g).  Straggler sets are inputs (bit masks).
+ *
+ * Conventions common to all calls
+ *   - Indices are 0-based.  Layer l = 1..L holds n^l nodes; node (l, i) has flat
+ *     index offset(l) + i with offset(l) = n + .. + n^(l-1); its children are
+ *     (l+1, n*i .. n*i + n-1).  The master is layer 0.
+ *   - A sibling group is the n children of one parent.  Group 0 is the master's;
+ *     the group below flat node v is v + 1.  There are 1 + n + .. + n^(L-1) groups.
+ *   - A straggler mask is a uint32 whose bit j marks child j of the group as a
+ *     straggler.  More than s bits set in a group that is consulted makes the
+ *     pattern undecodable (the failure case of the second remark after
+ *     Theorem 1); masks of groups below an unused child are ignored.
+ *   - "device pointer" = memory of the plan's CUDA device, owned by the caller
+ *     (e.g. allocated through PyTorch); "host pointer" = ordinary host memory.
+ *     The library never frees or keeps caller buffers beyond the work it
+ *     enqueues.  Device buffers of element type float (CR_F32) or int32_t
+ *     (CR_I32) must be 4-byte aligned; 16-byte alignment and d % 4 == 0 enable
+ *     the TMA path, anything else silently takes the plain-load kernels.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Device
+ *     calls only enqueue work and small async copies; they do not synchronise.
+ *   - Every function returns a cr_status_t (CR_OK = 0) unless stated; nothing
+ *     aborts or traps.  All argument and mask validation happens on the host
+ *     before anything is launched.  There is no CPU fallback: device calls on a
+ *     host-only plan return CR_ERR_CUDA.
+ */
+#ifndef CODEDREDUCE_H
+#define CODEDREDUCE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct cr_plan cr_plan_t;
+
+typedef enum {
+    CR_OK = 0,
+    CR_ERR_INVALID_ARG = 1,         /* NULL pointer, n/L/s/d out of range, bad flags, mask bit >= n */
+    CR_ERR_BAD_PARTITION_COUNT = 2, /* P is not a multiple of sum_l n^l (s+1)^(L-l) */
+    CR_ERR_CODE_UNAVAILABLE = 3,    /* code does not exist for this (n, s) */
+    CR_ERR_ILL_CONDITIONED = 4,     /* no encoding matrix with kappa <= max_kappa / span property fails */
+    CR_ERR_UNDECODABLE_MASK = 5,    /* > s stragglers in a consulted group */
+    CR_ERR_DTYPE = 6,               /* integer mode asked of a non-integer code, or dtype mismatch */
+    CR_ERR_CUDA = 7,                /* a CUDA call failed, or device work asked of a host-only plan */
+    CR_ERR_OOM = 8,                 /* workspace too small / allocation failed */
+    CR_ERR_TIMEOUT = 9              /* a bounded device-side wait gave up (reported by cr_plan_device_status) */
+} cr_status_t;
+
+/* Which gradient-coding encoding matrix B the plan builds (Section II-C). */
+typedef enum {
+    CR_CODE_CYCLIC_RANDOM = 0,         /* cyclic support {i..i+s}, random null-space construction */
+    CR_CODE_FRACTIONAL_REPETITION = 1, /* 0/1 rows, n/(s+1) blocks of s+1 identical workers */
+    CR_CODE_PAPER_3_1 = 2,             /* the (A, B) printed in Eq. (gc3nodes); n = 3, s = 1 only */
+    CR_CODE_EXPLICIT = 3               /* caller supplies B per level */
+} cr_code_t;
+
+typedef enum { CR_F32 = 0, CR_I32 = 1 } cr_dtype_t;
+
+/* Problem statement, mirroring the inputs of Algorithm 2: the (n, L) tree, the
+ * straggler tolerance s per parent, the data set as P atomic partitions, the
+ * gradient length d (the paper's p). */
+typedef struct {
+    int32_t n;          /* children per parent, 2..16 */
+    int32_t L;          /* worker layers, 1..8 */
+    int32_t s;          /* stragglers tolerated per sibling group, 0..n-1 */
+    int32_t P;          /* atomic data partitions; multiple of sum_l n^l (s+1)^(L-l) */
+    int64_t d;          /* gradient length, >= 1 */
+    int32_t code;       /* cr_code_t */
+    int32_t dtype;      /* cr_dtype_t of G_slots / outputs */
+    uint64_t seed;      /* CR_CODE_CYCLIC_RANDOM: first sub-seed tried */
+    const double *B_explicit; /* host, [L][n][n] row-major (level l = matrix used by parents at layer l),
+                                 read during cr_plan_create only; NULL unless CR_CODE_EXPLICIT */
+    double max_kappa;   /* conditioning screen for random codes; <= 0 selects 100 */
+    int32_t device;     /* CUDA device ordinal, or -1 for a host-only plan (queries only) */
+    int32_t reserved;   /* must be 0 */
+} cr_plan_desc_t;
+
+/* Variants of cr_aggregate (low byte of `flags`) and option bits. */
+enum {
+    CR_AGG_FUSED = 0,        /* one kernel, TMA-staged tiles, all levels in registers/shared memory */
+    CR_AGG_FUSED_LDG = 1,    /* same dataflow with plain 128-bit loads (any d, any alignment) */
+    CR_AGG_UNFUSED = 2,      /* cr_encode + cr_decode per level through the workspace */
+    CR_AGG_UNCODED_SUM = 3,  /* comparator: plain sum of the same used slots, all weights 1 */
+    CR_AGG_VARIANT_MASK = 0xff,
+    CR_AGG_ALL_NODES = 0x100 /* CR_AGG_UNFUSED only: encode and decode every node, not just used ones */
+};
+
+/* ---- plan: CR.Allocate + the gradient-coding tables (host work, once) ------------------------
+ * cr_plan_create builds the tree indexing, the per-level encoding matrices B (Section II-C), the
+ * allocation of (partition, coefficient) pairs to every node by the recursion of Algorithm 2
+ * (CR.Allocate) over CompAlloc (Algorithm 1): a parent's pass-down list is cut into n equal
+ * consecutive chunks, child i receives chunk kappa scaled by b_{i,kappa} for every non-zero entry in
+ * increasing kappa, keeps the first m = r_CR * P pairs (Theorem 1) and passes the rest down.  It also
+ * solves, in fp64, the decode row a (a B = 1, supported on the lowest-indexed n-s non-stragglers)
+ * for every straggler mask with at most s bits, per level.  With device >= 0 it makes that device
+ * current for the call, allocates small device mirrors of the tables and a ring of pinned staging
+ * buffers; cr_plan_destroy frees them.  *out is written only on CR_OK. */
+cr_status_t cr_plan_create(const cr_plan_desc_t *desc, cr_plan_t **out);
+cr_status_t cr_plan_destroy(cr_plan_t *plan);
+
+/* Human-readable name of a status code (static storage). */
+const char *cr_status_string(int status);
+/* Text of the last CUDA error seen by the calling thread ("" if none); valid until the next error. */
+const char *cr_last_cuda_error(void);
+
+/* Read-only queries; outputs are caller-allocated host memory. */
+int32_t cr_plan_num_nodes(const cr_plan_t *plan);   /* N */
+int32_t cr_plan_num_groups(const cr_plan_t *plan);  /* N / n */
+int32_t cr_plan_load(const cr_plan_t *plan);        /* m = r_CR * P slots per node */
+int64_t cr_plan_int_scale(const cr_plan_t *plan);   /* CR_I32: S = sigma^L with sigma*B integer; else 1 */
+/* B used by the parents at `level` (0 = master .. L-1), n*n row-major; kappa and the sub-seed that
+ * produced it (either pointer may be NULL). */
+cr_status_t cr_plan_get_B(const cr_plan_t *plan, int32_t level, double *B, double *kappa, uint64_t *sub_seed);
+/* D(l,i) of flat node `node`: m partition ids and their combining coefficients (Section III-A,
+ * "scaled data sets").  In CR_I32 plans the coefficients returned are still the real ones; the
+ * device uses S * coeff. */
+cr_status_t cr_plan_get_slots(const cr_plan_t *plan, int32_t node, int32_t *part, double *coeff);
+/* Decode row (n doubles) a parent at `level` uses for `straggler_mask`; CR_ERR_UNDECODABLE_MASK if
+ * the mask has more than s bits. */
+cr_status_t cr_plan_get_decode(const cr_plan_t *plan, int32_t level, uint32_t straggler_mask, double *a);
+/* Host expansion of one straggler pattern (masks[num_groups]) into the post-order list of nodes
+ * whose data is consumed: nodes[k], layers[k] (1..L) and the decode weight with which node k's
+ * message enters its parent.  capacity >= N always suffices; *count receives the length. */
+cr_status_t cr_plan_expand(const cr_plan_t *plan, const uint32_t *masks, int32_t capacity,
+                           int32_t *nodes, int32_t *layers, double *weights, int32_t *count);
+/* Sticky status word written by bounded device-side waits: CR_OK, or CR_ERR_TIMEOUT if a kernel of
+ * this plan ever gave up waiting for a copy.  Synchronises the device. */
+cr_status_t cr_plan_device_status(cr_plan_t *plan);
+
+/* ---- CR.Execute, step "all nodes compute their local partial gradients" (Algorithm 2) ---------
+ * Linear-regression instance of Eq. (g): for every node v and slot j holding partition p,
+ *   G_slots[v][j][:] = X_p^T (X_p w - y_p).
+ * X [P][rows][d], y [P][rows], w [d], G_slots [N][m][d]: device pointers, fp32, row-major.
+ * workspace: device scratch of at least cr_partial_gradients_workspace_bytes(plan, rows) bytes
+ * (residuals, one per node, slot and row).  CR_F32 plans only. */
+size_t cr_partial_gradients_workspace_bytes(const cr_plan_t *plan, int32_t rows);
+cr_status_t cr_partial_gradients(cr_plan_t *plan, const float *X, const float *y, int32_t rows,
+                                 const float *w, float *G_slots, void *workspace,
+                                 size_t workspace_bytes, void *stream);
+
+/* ---- CR.Execute, local coded gradient g_{D(l,i)} (Section III-A) ------------------------------
+ * E[v][:] = sum_j c_{v,j} * G_slots[v][j][:] for every node v.  G_slots [N][m][d], E [N][d]:
+ * device pointers of the plan's dtype.  (Verification path; the fused kernel never writes E.) */
+cr_status_t cr_encode(cr_plan_t *plan, const void *G_slots, void *E, void *stream);
+
+/* ---- CR.Execute, one level of "decode from any n-s children, add own, upload" -----------------
+ * For every parent i at `parent_layer` (L-1 .. 0; 0 = master):
+ *   M_parent[i][:] = sum_j a[j] * M_child[n*i + j][:]  (+ E_parent[i][:] unless parent_layer == 0)
+ * with a the decode row for masks_host[i].  M_child [n^(parent_layer+1)][d], E_parent
+ * [n^parent_layer][d] (the slice of E for that layer; NULL at layer 0), M_parent
+ * [n^parent_layer][d]: device pointers.  masks_host: host, one per parent of the layer.
+ * Children with zero weight are not read. */
+cr_status_t cr_decode(cr_plan_t *plan, int32_t parent_layer, const void *M_child, const void *E_parent,
+                      const uint32_t *masks_host, void *M_parent, void *stream);
+
+/* ---- CR.Execute end to end for `batch` straggler patterns --------------------------------------
+ * g_out[b][:] = root result for pattern b.  G_slots [N][m][d] and g_out [batch][d] are device
+ * pointers; masks_host is host memory [batch][num_groups].  Only nodes with non-zero decode weight
+ * along the tree are read.  In CR_I32 plans all arithmetic is int32 on S-scaled integer
+ * coefficients and the root divides by S exactly (wrap-around on overflow is the caller's concern).
+ * workspace: device scratch, needed by CR_AGG_UNFUSED only
+ * (cr_aggregate_workspace_bytes); may be NULL otherwise. */
+size_t cr_aggregate_workspace_bytes(const cr_plan_t *plan, int32_t batch, uint32_t flags);
+cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *masks_host, int32_t batch,
+                         void *g_out, uint32_t flags, void *workspace, size_t workspace_bytes, void *stream);
+
+/* Same computation with HOST buffers: copies G_slots_host (pinned or pageable host memory,
+ * [N][m][d]) into dev_slots, runs cr_aggregate, copies the result into g_out_host and waits for the
+ * stream.  dev_slots [N][m][d] and dev_out [batch][d] are caller-owned device staging buffers. */
+cr_status_t cr_aggregate_host(cr_plan_t *plan, const void *G_slots_host, const uint32_t *masks_host,
+                              int32_t batch, void *g_out_host, uint32_t flags, void *dev_slots,
+                              void *dev_out, void *workspace, size_t workspace_bytes, void *stream);
+
+/* Algorithmic bytes of one cr_aggregate call: element size * d * (m * |union of used nodes| + batch),
+ * i.e. every used slot read once and every output written once.  *used_nodes (may be NULL)
+ * receives the size of the union. */
+cr_status_t cr_aggregate_bytes(const cr_plan_t *plan, const uint32_t *masks_host, int32_t batch,
+                               int64_t *bytes, int32_t *used_nodes);
+
+/* Launch shape of the TMA kernels of cr_aggregate; 0 keeps the built-in choice for that field.
+ * consumer_warps in {2,4,8} (single-pattern kernel: column tile = 128 * consumer_warps), stages = depth
+ * of the shared-memory ring (2..16), ctas_per_sm = persistent CTAs per SM (1..8), rows_per_box = slot
+ * rows per TMA box (must divide m).  Shapes that do not fit shared memory fall back to plain loads. */
+cr_status_t cr_plan_tune(cr_plan_t *plan, int32_t consumer_warps, int32_t stages, int32_t ctas_per_sm,
+                         int32_t rows_per_box);
+
+/* Kernel launches enqueued by this plan's device calls so far. */
+int64_t cr_plan_launch_count(const cr_plan_t *plan);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CODEDREDUCE_H */

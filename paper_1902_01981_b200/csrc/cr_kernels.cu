@@ -1,0 +1,915 @@
+// sm_100a kernels of the coded tree aggregation (CR.Execute, Algorithm 2).
+//
+// The aggregation is a chain of axpy-like passes over length-d vectors, one FMA per element read:
+// bound by HBM bandwidth, no dense contraction, so no tensor cores.  The fused kernels give each CTA
+// a tile of columns, stream the slot rows of the consumed nodes through a TMA -> shared-memory ring
+// and keep every intermediate coded vector (a node's coded gradient, every message) in registers
+// or shared memory; only the root tile is written.
+#include "cr_kernels.hpp"
+
+#include <algorithm>
+#include <cstdio>
+
+namespace cr {
+
+// ------------------------------------------------------------------------------------------------
+// PTX helpers: mbarrier, TMA, timers
+// ------------------------------------------------------------------------------------------------
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_timer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Every wait in these kernels is bounded: about two seconds of wall time or 2^30 polls, whichever
+// comes first, or as soon as another thread of the CTA has given up.  A correct launch never gets
+// near the bound; it exists so that a broken one returns with a status instead of hanging the GPU.
+constexpr uint64_t kWaitLimitNs = 2000000000ull;
+
+// `abort_flag` points at a shared-memory word that the other side of the pipeline sets when it has
+// given up (flags[0]: a consumer did, flags[1]: the producer did, flags[2]: never set).
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = global_timer_ns();
+    for (int outer = 0; outer < (1 << 22); ++outer) {
+#pragma unroll 1
+        for (int i = 0; i < 256; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (global_timer_ns() - t0 > kWaitLimitNs) return false;
+    }
+    return false;
+}
+
+// 2-D tiled TMA load global -> shared, completion counted in bytes on an mbarrier.  x (innermost
+// coordinate) times the element size must be a multiple of 16 bytes.
+__device__ __forceinline__ void tma_load_2d(void *smem_dst, const CUtensorMap *map, int x, int y, uint64_t *bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
+
+__device__ __forceinline__ void consumer_barrier(int threads) {
+    asm volatile("bar.sync 1, %0;" ::"r"(threads) : "memory");
+}
+
+// ------------------------------------------------------------------------------------------------
+// element-type helpers
+// ------------------------------------------------------------------------------------------------
+
+template <typename T> struct Vec4;
+template <> struct Vec4<float> { typedef float4 type; };
+template <> struct Vec4<int> { typedef int4 type; };
+
+template <typename T> __device__ __forceinline__ T weight_of(uint32_t bits);
+template <> __device__ __forceinline__ float weight_of<float>(uint32_t bits) { return __uint_as_float(bits); }
+template <> __device__ __forceinline__ int weight_of<int>(uint32_t bits) { return (int)bits; }
+
+template <typename T> __device__ __forceinline__ T finish(T v, int shift) { return v; }
+template <> __device__ __forceinline__ int finish<int>(int v, int shift) { return v >> shift; }
+
+__device__ __forceinline__ Step load_step(const Step *p) {
+    const int4 raw = __ldg(reinterpret_cast<const int4 *>(p));
+    Step s;
+    s.node = raw.x; s.layer = raw.y; s.wbits = (uint32_t)raw.z; s.index = raw.w;
+    return s;
+}
+
+// The tree recursion in registers.  acc[l] (l = 0..LMAX-1) holds, for the node of layer l currently
+// being assembled, the decoded combination of the children messages seen so far.  Visiting a node of
+// layer `layer` in post-order with coded gradient e and decode weight w at its parent:
+//     message = acc[layer] + e;   acc[layer-1] += w * message;   acc[layer] = 0
+// (leaves have no acc of their own: message = e).  After the last step acc[0] is the root's result.
+template <typename T, int LMAX, int V>
+__device__ __forceinline__ void fold(T (&acc)[LMAX][V], const T (&e)[V], int layer, T w) {
+#pragma unroll
+    for (int l = 1; l <= LMAX; ++l) {
+        if (layer == l) {
+#pragma unroll
+            for (int q = 0; q < V; ++q) {
+                T msg = e[q];
+                if (l < LMAX) { msg += acc[l < LMAX ? l : 0][q]; acc[l < LMAX ? l : 0][q] = T(0); }
+                acc[l - 1][q] += w * msg;
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// K4: fused aggregation, one straggler pattern, TMA-staged
+// ------------------------------------------------------------------------------------------------
+//
+// CTA = NCW consumer warps + 1 producer warp, persistent over column tiles of TILE = 128*NCW
+// elements.  Per tile the producer streams, for every consumed node in post-order, boxes of R slot
+// rows x TILE columns into a ring of `stages` buffers; consumer thread t owns 4 consecutive columns,
+// forms the node's coded gradient e = sum_j c_j * row_j from shared memory and folds it into the
+// register recursion above.  Shared-memory layout of a stage: [box][R][BOXW] with BOXW = min(TILE,256)
+// (a TMA box is at most 256 elements wide).
+
+struct FusedArgs {
+    const void *coeff;
+    const Step *steps;
+    int n_steps;
+    int m, R, cpn, stages;
+    long long d;
+    long long ntiles;
+    void *out;
+    int shift;
+    int *status;
+};
+
+template <typename T, int LMAX, int NCW>
+__global__ void __launch_bounds__((NCW + 1) * 32)
+cr_fused_tma_kernel(const __grid_constant__ CUtensorMap tmap, const FusedArgs a) {
+    constexpr int TILE = NCW * 128;
+    constexpr int BOXW = TILE < 256 ? TILE : 256;
+    constexpr int NBOX = TILE / BOXW;
+    typedef typename Vec4<T>::type V4;
+
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const int R = a.R, S = a.stages;
+    const size_t stage_elems = (size_t)R * TILE;
+    T *ring = reinterpret_cast<T *>(smem_raw);
+    uint64_t *full = reinterpret_cast<uint64_t *>(smem_raw + (size_t)S * stage_elems * sizeof(T));
+    uint64_t *empty = full + S;
+    volatile int *flags = reinterpret_cast<volatile int *>(empty + S);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], NCW); }
+        flags[0] = 0; flags[1] = 0; flags[2] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    const T *coeff = reinterpret_cast<const T *>(a.coeff);
+    const uint32_t stage_bytes = (uint32_t)(stage_elems * sizeof(T));
+
+    if (warp == NCW) {
+        // ---------------- producer: one thread issues every TMA of this CTA ----------------
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            long long issued = 0;
+            bool ok = true;
+            for (long long tile = blockIdx.x; tile < a.ntiles && ok; tile += gridDim.x) {
+                const int x0 = (int)(tile * TILE);
+                for (int k = 0; k < a.n_steps && ok; ++k) {
+                    const int row0 = __ldg(&a.steps[k].node) * a.m;
+                    for (int c = 0; c < a.cpn; ++c) {
+                        if (!mbar_wait(&empty[stage], phase ^ 1u, &flags[0])) { ok = false; break; }
+                        mbar_expect_tx(&full[stage], stage_bytes);
+                        T *dst = ring + (size_t)stage * stage_elems;
+#pragma unroll
+                        for (int b = 0; b < NBOX; ++b)
+                            tma_load_2d(dst + (size_t)b * R * BOXW, &tmap, x0 + b * BOXW, row0 + c * R, &full[stage]);
+                        ++issued;
+                        if (++stage == S) { stage = 0; phase ^= 1u; }
+                    }
+                }
+            }
+            if (!ok) {
+                // give up: flag it, then wait (bounded) for the copies still in flight so that none
+                // lands in shared memory after the CTA has gone
+                flags[1] = 1;
+                atomicExch(a.status, 1);
+                for (long long i = issued > S ? issued - S : 0; i < issued; ++i)
+                    mbar_wait(&full[i % S], (uint32_t)((i / S) & 1), &flags[2]);
+            }
+        }
+    } else {
+        // ---------------- consumers ----------------
+        T acc[LMAX][4];
+#pragma unroll
+        for (int l = 0; l < LMAX; ++l)
+#pragma unroll
+            for (int q = 0; q < 4; ++q) acc[l][q] = T(0);
+        const int col = tid * 4;
+        const int box = col / BOXW, within = col % BOXW;
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (long long tile = blockIdx.x; tile < a.ntiles && ok; tile += gridDim.x) {
+            for (int k = 0; k < a.n_steps && ok; ++k) {
+                const Step st = load_step(&a.steps[k]);
+                T e[4] = {T(0), T(0), T(0), T(0)};
+                for (int c = 0; c < a.cpn; ++c) {
+                    const T *cf = coeff + (size_t)st.node * a.m + c * R;
+                    if (!mbar_wait(&full[stage], phase, &flags[1])) { ok = false; break; }
+                    const T *src = ring + (size_t)stage * stage_elems + (size_t)box * R * BOXW + within;
+#pragma unroll 4
+                    for (int j = 0; j < R; ++j) {
+                        const V4 v = *reinterpret_cast<const V4 *>(src + (size_t)j * BOXW);
+                        const T cj = __ldg(cf + j);
+                        e[0] += cj * v.x; e[1] += cj * v.y; e[2] += cj * v.z; e[3] += cj * v.w;
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&empty[stage]);
+                    if (++stage == S) { stage = 0; phase ^= 1u; }
+                }
+                fold<T, LMAX, 4>(acc, e, st.layer, weight_of<T>(st.wbits));
+            }
+            if (!ok) break;
+            const long long gcol = tile * TILE + col;
+            if (gcol < a.d) {
+                V4 o;
+                o.x = finish<T>(acc[0][0], a.shift); o.y = finish<T>(acc[0][1], a.shift);
+                o.z = finish<T>(acc[0][2], a.shift); o.w = finish<T>(acc[0][3], a.shift);
+                *reinterpret_cast<V4 *>(reinterpret_cast<T *>(a.out) + gcol) = o;
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) acc[0][q] = T(0);
+        }
+        if (!ok) { flags[0] = 1; atomicExch(a.status, 1); }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// K4b: fused aggregation, a batch of straggler patterns over the same slots
+// ------------------------------------------------------------------------------------------------
+//
+// The coded gradient e_v of a node does not depend on the straggler pattern, so a CTA (tile of 128
+// columns, each consumer warp a full tile row of float4s) first forms e_v for every node of the union
+// of consumed nodes -- warp w takes nodes w, w+NCW, .. -- into shared memory E[n_union][128], then
+// replays every pattern's post-order schedule from E (warp w takes patterns w, w+NCW, ..) and writes
+// one output tile per pattern.  The slots are read from HBM once for the whole batch; the producer
+// warp keeps prefetching the next tile's rows through the ring while patterns are replayed.
+
+struct BatchArgs {
+    const void *coeff;
+    const Step *steps;
+    const int32_t *pat_off;
+    const int32_t *unodes;
+    int n_union, batch;
+    int m, R, cpn, stages;
+    long long d;
+    long long ntiles;
+    void *out;
+    int shift;
+    int *status;
+};
+
+template <typename T, int LMAX, int NCW>
+__global__ void __launch_bounds__((NCW + 1) * 32)
+cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchArgs a) {
+    constexpr int TILE = 128;
+    typedef typename Vec4<T>::type V4;
+
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const int R = a.R, S = a.stages;
+    const size_t stage_elems = (size_t)R * TILE;
+    T *ring = reinterpret_cast<T *>(smem_raw);
+    T *E = ring + (size_t)S * stage_elems;
+    uint64_t *full = reinterpret_cast<uint64_t *>(E + (size_t)a.n_union * TILE);
+    uint64_t *empty = full + S;
+    volatile int *flags = reinterpret_cast<volatile int *>(empty + S);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        flags[0] = 0; flags[1] = 0; flags[2] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    const T *coeff = reinterpret_cast<const T *>(a.coeff);
+    const uint32_t stage_bytes = (uint32_t)(stage_elems * sizeof(T));
+    const unsigned per_tile = (unsigned)a.n_union * (unsigned)a.cpn;  // ring iterations per tile
+
+    if (warp == NCW) {
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            long long issued = 0;
+            bool ok = true;
+            for (long long tile = blockIdx.x; tile < a.ntiles && ok; tile += gridDim.x) {
+                const int x0 = (int)(tile * TILE);
+                for (int u = 0; u < a.n_union && ok; ++u) {
+                    const int row0 = __ldg(&a.unodes[u]) * a.m;
+                    for (int c = 0; c < a.cpn; ++c) {
+                        if (!mbar_wait(&empty[stage], phase ^ 1u, &flags[0])) { ok = false; break; }
+                        mbar_expect_tx(&full[stage], stage_bytes);
+                        tma_load_2d(ring + (size_t)stage * stage_elems, &tmap, x0, row0 + c * R, &full[stage]);
+                        ++issued;
+                        if (++stage == S) { stage = 0; phase ^= 1u; }
+                    }
+                }
+            }
+            if (!ok) {
+                flags[1] = 1;
+                atomicExch(a.status, 1);
+                for (long long i = issued > S ? issued - S : 0; i < issued; ++i)
+                    mbar_wait(&full[i % S], (uint32_t)((i / S) & 1), &flags[2]);
+            }
+        }
+    } else {
+        bool ok = true;
+        unsigned tile_iter0 = 0;  // ring iteration index of this tile's first box
+        for (long long tile = blockIdx.x; tile < a.ntiles; tile += gridDim.x, tile_iter0 += per_tile) {
+            // phase 1: coded gradients of the union nodes -> E
+            for (int u = warp; u < a.n_union && ok; u += NCW) {
+                const int node = __ldg(&a.unodes[u]);
+                T e[4] = {T(0), T(0), T(0), T(0)};
+                for (int c = 0; c < a.cpn; ++c) {
+                    const unsigned it = tile_iter0 + (unsigned)u * (unsigned)a.cpn + (unsigned)c;
+                    const int stage = (int)(it % (unsigned)S);
+                    const uint32_t phase = (it / (unsigned)S) & 1u;
+                    const T *cf = coeff + (size_t)node * a.m + c * R;
+                    if (!mbar_wait(&full[stage], phase, &flags[1])) { ok = false; break; }
+                    const T *src = ring + (size_t)stage * stage_elems + lane * 4;
+#pragma unroll 4
+                    for (int j = 0; j < R; ++j) {
+                        const V4 v = *reinterpret_cast<const V4 *>(src + (size_t)j * TILE);
+                        const T cj = __ldg(cf + j);
+                        e[0] += cj * v.x; e[1] += cj * v.y; e[2] += cj * v.z; e[3] += cj * v.w;
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&empty[stage]);
+                }
+                V4 o; o.x = e[0]; o.y = e[1]; o.z = e[2]; o.w = e[3];
+                *reinterpret_cast<V4 *>(E + (size_t)u * TILE + lane * 4) = o;
+            }
+            // flags[0] is written only by consumers and only before this barrier, so every consumer
+            // warp reads the same value after it and they leave together
+            if (!ok) { flags[0] = 1; atomicExch(a.status, 1); }
+            consumer_barrier(NCW * 32);
+            if (flags[0]) break;
+            // phase 2: replay every pattern's schedule from E
+            const long long gcol = tile * TILE + lane * 4;
+            for (int b = warp; b < a.batch; b += NCW) {
+                T acc[LMAX][4];
+#pragma unroll
+                for (int l = 0; l < LMAX; ++l)
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) acc[l][q] = T(0);
+                const int k0 = __ldg(&a.pat_off[b]), k1 = __ldg(&a.pat_off[b + 1]);
+                for (int k = k0; k < k1; ++k) {
+                    const Step st = load_step(&a.steps[k]);
+                    const V4 v = *reinterpret_cast<const V4 *>(E + (size_t)st.index * TILE + lane * 4);
+                    const T e[4] = {v.x, v.y, v.z, v.w};
+                    fold<T, LMAX, 4>(acc, e, st.layer, weight_of<T>(st.wbits));
+                }
+                if (gcol < a.d) {
+                    V4 o;
+                    o.x = finish<T>(acc[0][0], a.shift); o.y = finish<T>(acc[0][1], a.shift);
+                    o.z = finish<T>(acc[0][2], a.shift); o.w = finish<T>(acc[0][3], a.shift);
+                    *reinterpret_cast<V4 *>(reinterpret_cast<T *>(a.out) + (size_t)b * a.d + gcol) = o;
+                }
+            }
+            consumer_barrier(NCW * 32);  // E is rewritten by the next tile
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Fused aggregation with plain loads (any d, any alignment); grid.y = pattern
+// ------------------------------------------------------------------------------------------------
+
+template <typename T, int V> struct Loader;
+template <typename T> struct Loader<T, 1> {
+    static __device__ __forceinline__ void load(const T *p, T (&v)[1]) { v[0] = __ldg(p); }
+    static __device__ __forceinline__ void store(T *p, const T (&v)[1]) { p[0] = v[0]; }
+};
+template <> struct Loader<float, 4> {
+    static __device__ __forceinline__ void load(const float *p, float (&v)[4]) {
+        float4 t;
+        asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
+                     : "=f"(t.x), "=f"(t.y), "=f"(t.z), "=f"(t.w) : "l"(p));
+        v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+    }
+    static __device__ __forceinline__ void store(float *p, const float (&v)[4]) {
+        *reinterpret_cast<float4 *>(p) = make_float4(v[0], v[1], v[2], v[3]);
+    }
+};
+template <> struct Loader<int, 4> {
+    static __device__ __forceinline__ void load(const int *p, int (&v)[4]) {
+        int4 t;
+        asm volatile("ld.global.nc.L1::no_allocate.v4.s32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(t.x), "=r"(t.y), "=r"(t.z), "=r"(t.w) : "l"(p));
+        v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w;
+    }
+    static __device__ __forceinline__ void store(int *p, const int (&v)[4]) {
+        *reinterpret_cast<int4 *>(p) = make_int4(v[0], v[1], v[2], v[3]);
+    }
+};
+
+template <typename T, int LMAX, int V>
+__global__ void __launch_bounds__(256)
+cr_fused_ldg_kernel(const T *__restrict__ G, const T *__restrict__ coeff, const Step *__restrict__ steps,
+                    const int32_t *__restrict__ pat_off, int m, long long d, T *__restrict__ out, int shift) {
+    const int b = blockIdx.y;
+    const long long col = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * V;
+    if (col >= d) return;
+    const int k0 = __ldg(&pat_off[b]), k1 = __ldg(&pat_off[b + 1]);
+    T acc[LMAX][V];
+#pragma unroll
+    for (int l = 0; l < LMAX; ++l)
+#pragma unroll
+        for (int q = 0; q < V; ++q) acc[l][q] = T(0);
+    for (int k = k0; k < k1; ++k) {
+        const Step st = load_step(&steps[k]);
+        const T *row = G + (size_t)st.node * m * d + col;
+        const T *cf = coeff + (size_t)st.node * m;
+        T e[V];
+#pragma unroll
+        for (int q = 0; q < V; ++q) e[q] = T(0);
+        int j = 0;
+        for (; j + 4 <= m; j += 4) {
+            T v0[V], v1[V], v2[V], v3[V];
+            Loader<T, V>::load(row + (size_t)(j + 0) * d, v0);
+            Loader<T, V>::load(row + (size_t)(j + 1) * d, v1);
+            Loader<T, V>::load(row + (size_t)(j + 2) * d, v2);
+            Loader<T, V>::load(row + (size_t)(j + 3) * d, v3);
+            const T c0 = __ldg(cf + j), c1 = __ldg(cf + j + 1), c2 = __ldg(cf + j + 2), c3 = __ldg(cf + j + 3);
+#pragma unroll
+            for (int q = 0; q < V; ++q) e[q] += c0 * v0[q] + c1 * v1[q] + c2 * v2[q] + c3 * v3[q];
+        }
+        for (; j < m; ++j) {
+            T v0[V];
+            Loader<T, V>::load(row + (size_t)j * d, v0);
+            const T c0 = __ldg(cf + j);
+#pragma unroll
+            for (int q = 0; q < V; ++q) e[q] += c0 * v0[q];
+        }
+        fold<T, LMAX, V>(acc, e, st.layer, weight_of<T>(st.wbits));
+    }
+    T o[V];
+#pragma unroll
+    for (int q = 0; q < V; ++q) o[q] = finish<T>(acc[0][q], shift);
+    Loader<T, V>::store(out + (size_t)b * d + col, o);
+}
+
+// ------------------------------------------------------------------------------------------------
+// K5: uncoded comparator -- plain sum of the same slot rows, all weights 1
+// ------------------------------------------------------------------------------------------------
+
+template <typename T, int V>
+__global__ void __launch_bounds__(256)
+cr_uncoded_sum_kernel(const T *__restrict__ G, const Step *__restrict__ steps, const int32_t *__restrict__ pat_off,
+                      int m, long long d, T *__restrict__ out) {
+    const int b = blockIdx.y;
+    const long long col = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * V;
+    if (col >= d) return;
+    const int k0 = __ldg(&pat_off[b]), k1 = __ldg(&pat_off[b + 1]);
+    T acc[V];
+#pragma unroll
+    for (int q = 0; q < V; ++q) acc[q] = T(0);
+    for (int k = k0; k < k1; ++k) {
+        const T *row = G + (size_t)__ldg(&steps[k].node) * m * d + col;
+        int j = 0;
+        for (; j + 4 <= m; j += 4) {
+            T v0[V], v1[V], v2[V], v3[V];
+            Loader<T, V>::load(row + (size_t)(j + 0) * d, v0);
+            Loader<T, V>::load(row + (size_t)(j + 1) * d, v1);
+            Loader<T, V>::load(row + (size_t)(j + 2) * d, v2);
+            Loader<T, V>::load(row + (size_t)(j + 3) * d, v3);
+#pragma unroll
+            for (int q = 0; q < V; ++q) acc[q] += (v0[q] + v1[q]) + (v2[q] + v3[q]);
+        }
+        for (; j < m; ++j) {
+            T v0[V];
+            Loader<T, V>::load(row + (size_t)j * d, v0);
+#pragma unroll
+            for (int q = 0; q < V; ++q) acc[q] += v0[q];
+        }
+    }
+    Loader<T, V>::store(out + (size_t)b * d + col, acc);
+}
+
+// ------------------------------------------------------------------------------------------------
+// K2 / K3: unfused verification path
+// ------------------------------------------------------------------------------------------------
+
+template <typename T, int V>
+__global__ void __launch_bounds__(256)
+cr_encode_kernel(const T *__restrict__ G, const T *__restrict__ coeff, const int32_t *__restrict__ nodes, int m,
+                 long long d, T *__restrict__ E) {
+    const int v = nodes ? __ldg(&nodes[blockIdx.y]) : (int)blockIdx.y;
+    const long long col = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * V;
+    if (col >= d) return;
+    const T *row = G + (size_t)v * m * d + col;
+    const T *cf = coeff + (size_t)v * m;
+    T e[V];
+#pragma unroll
+    for (int q = 0; q < V; ++q) e[q] = T(0);
+    for (int j = 0; j < m; ++j) {
+        T x[V];
+        Loader<T, V>::load(row + (size_t)j * d, x);
+        const T c = __ldg(cf + j);
+#pragma unroll
+        for (int q = 0; q < V; ++q) e[q] += c * x[q];
+    }
+    Loader<T, V>::store(E + (size_t)v * d + col, e);
+}
+
+template <typename T, int V>
+__global__ void __launch_bounds__(256)
+cr_decode_kernel(const T *__restrict__ M_child, const T *__restrict__ E_parent, const T *__restrict__ W,
+                 const int32_t *__restrict__ active, int n, long long d, T *__restrict__ M_parent, int shift) {
+    const int i = blockIdx.y;
+    if (active && __ldg(&active[i]) == 0) return;
+    const long long col = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * V;
+    if (col >= d) return;
+    T acc[V];
+#pragma unroll
+    for (int q = 0; q < V; ++q) acc[q] = T(0);
+    for (int j = 0; j < n; ++j) {
+        const T w = __ldg(&W[(size_t)i * n + j]);
+        if (w == T(0)) continue;  // stragglers and unused survivors are never read
+        T x[V];
+        Loader<T, V>::load(M_child + ((size_t)i * n + j) * d + col, x);
+#pragma unroll
+        for (int q = 0; q < V; ++q) acc[q] += w * x[q];
+    }
+    if (E_parent) {
+        T x[V];
+        Loader<T, V>::load(E_parent + (size_t)i * d + col, x);
+#pragma unroll
+        for (int q = 0; q < V; ++q) acc[q] += x[q];
+    }
+#pragma unroll
+    for (int q = 0; q < V; ++q) acc[q] = finish<T>(acc[q], shift);
+    Loader<T, V>::store(M_parent + (size_t)i * d + col, acc);
+}
+
+// ------------------------------------------------------------------------------------------------
+// K1: partial gradients of linear regression, X_p^T (X_p w - y_p), two passes
+// ------------------------------------------------------------------------------------------------
+
+// Pass 1: one warp per (slot item, row): r = <X_p[row,:], w> - y_p[row].
+template <int V>
+__global__ void __launch_bounds__(256)
+cr_residual_kernel(const float *__restrict__ X, const float *__restrict__ y, const float *__restrict__ w,
+                   const int32_t *__restrict__ part, long long total_rows, int rows, long long d,
+                   float *__restrict__ resid) {
+    const int lane = threadIdx.x & 31;
+    const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
+    for (long long idx = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; idx < total_rows; idx += warps) {
+        const long long item = idx / rows;
+        const int row = (int)(idx - item * rows);
+        const int p = __ldg(&part[item]);
+        const float *xr = X + ((size_t)p * rows + row) * d;
+        float acc = 0.f;
+        if (V == 4) {
+            for (long long c = lane * 4; c < d; c += 128) {
+                const float4 xv = __ldg(reinterpret_cast<const float4 *>(xr + c));
+                const float4 wv = __ldg(reinterpret_cast<const float4 *>(w + c));
+                acc += xv.x * wv.x + xv.y * wv.y + xv.z * wv.z + xv.w * wv.w;
+            }
+        } else {
+            for (long long c = lane; c < d; c += 32) acc += __ldg(xr + c) * __ldg(w + c);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+        if (lane == 0) resid[idx] = acc - __ldg(&y[(size_t)p * rows + row]);
+    }
+}
+
+// Pass 2: grid (column tiles, items); a thread owns V columns and walks all rows of the item.
+template <int V>
+__global__ void __launch_bounds__(128)
+cr_xt_r_kernel(const float *__restrict__ X, const int32_t *__restrict__ part, const float *__restrict__ resid,
+               int rows, long long d, float *__restrict__ G) {
+    const long long item = blockIdx.y;
+    const long long col = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * V;
+    if (col >= d) return;
+    const int p = __ldg(&part[item]);
+    const float *xp = X + (size_t)p * rows * d + col;
+    const float *r = resid + item * rows;
+    float acc[V];
+#pragma unroll
+    for (int q = 0; q < V; ++q) acc[q] = 0.f;
+    int row = 0;
+    for (; row + 4 <= rows; row += 4) {
+        float v0[V], v1[V], v2[V], v3[V];
+        Loader<float, V>::load(xp + (size_t)(row + 0) * d, v0);
+        Loader<float, V>::load(xp + (size_t)(row + 1) * d, v1);
+        Loader<float, V>::load(xp + (size_t)(row + 2) * d, v2);
+        Loader<float, V>::load(xp + (size_t)(row + 3) * d, v3);
+        const float r0 = __ldg(r + row), r1 = __ldg(r + row + 1), r2 = __ldg(r + row + 2), r3 = __ldg(r + row + 3);
+#pragma unroll
+        for (int q = 0; q < V; ++q) acc[q] += r0 * v0[q] + r1 * v1[q] + r2 * v2[q] + r3 * v3[q];
+    }
+    for (; row < rows; ++row) {
+        float v0[V];
+        Loader<float, V>::load(xp + (size_t)row * d, v0);
+        const float r0 = __ldg(r + row);
+#pragma unroll
+        for (int q = 0; q < V; ++q) acc[q] += r0 * v0[q];
+    }
+    Loader<float, V>::store(G + (size_t)item * d + col, acc);
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side: launch wrappers
+// ------------------------------------------------------------------------------------------------
+
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+bool tma_eligible(const AggArgs &a) {
+    return a.d % 4 == 0 && a.d >= 256 && a.d < (1ll << 31) && aligned16(a.G) && aligned16(a.out) &&
+           a.rows_total < (1ll << 31);
+}
+
+static bool vec4_ok(const void *G, const void *out, int64_t d) { return d % 4 == 0 && aligned16(G) && aligned16(out); }
+
+static int pick_lmax(int L) { return L <= 2 ? 2 : (L <= 4 ? 4 : 8); }
+
+static CUresult make_map(EncodeTiledFn encode, CUtensorMap *map, const AggArgs &a, int boxw, int boxrows) {
+    const cuuint64_t dims[2] = {(cuuint64_t)a.d, (cuuint64_t)a.rows_total};
+    const cuuint64_t strides[1] = {(cuuint64_t)a.d * 4u};
+    const cuuint32_t box[2] = {(cuuint32_t)boxw, (cuuint32_t)boxrows};
+    const cuuint32_t estr[2] = {1, 1};
+    return encode(map, a.is_int ? CU_TENSOR_MAP_DATA_TYPE_INT32 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2,
+                  const_cast<void *>(a.G), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                  CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+}
+
+// Largest divisor of m not above `cap`.
+static int rows_per_box(int m, int cap) {
+    int best = 1;
+    for (int r = 1; r <= m && r <= cap; ++r)
+        if (m % r == 0) best = r;
+    return best;
+}
+
+template <typename T, int LMAX, int NCW>
+static cudaError_t run_fused(const CUtensorMap &map, const FusedArgs &fa, int grid, size_t smem, cudaStream_t stream) {
+    auto kern = cr_fused_tma_kernel<T, LMAX, NCW>;
+    cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) return err;
+    kern<<<grid, (NCW + 1) * 32, smem, stream>>>(map, fa);
+    return cudaGetLastError();
+}
+
+template <typename T, int NCW>
+static cudaError_t run_fused_l(int lmax, const CUtensorMap &map, const FusedArgs &fa, int grid, size_t smem,
+                               cudaStream_t stream) {
+    switch (lmax) {
+        case 2: return run_fused<T, 2, NCW>(map, fa, grid, smem, stream);
+        case 4: return run_fused<T, 4, NCW>(map, fa, grid, smem, stream);
+        default: return run_fused<T, 8, NCW>(map, fa, grid, smem, stream);
+    }
+}
+
+template <typename T>
+static cudaError_t run_fused_ncw(int ncw, int lmax, const CUtensorMap &map, const FusedArgs &fa, int grid, size_t smem,
+                                 cudaStream_t stream) {
+    switch (ncw) {
+        case 2: return run_fused_l<T, 2>(lmax, map, fa, grid, smem, stream);
+        case 4: return run_fused_l<T, 4>(lmax, map, fa, grid, smem, stream);
+        default: return run_fused_l<T, 8>(lmax, map, fa, grid, smem, stream);
+    }
+}
+
+cudaError_t launch_fused_tma(const AggArgs &a, const DeviceInfo &dev, const Tuning &tune, EncodeTiledFn encode,
+                             cudaStream_t stream, int64_t *launches, bool *done) {
+    *done = false;
+    if (!encode || !tma_eligible(a) || a.batch != 1) return cudaSuccess;
+    int ncw = tune.ncw ? tune.ncw : 4;
+    if (ncw != 2 && ncw != 4 && ncw != 8) ncw = 4;
+    const int tile = ncw * 128;
+    const int boxw = tile < 256 ? tile : 256;
+    // rows per box: a divisor of m, at most 16, stage no larger than ~36 KB
+    int cap = std::min(16, std::max(1, (36 * 1024) / (tile * 4)));
+    int R = tune.rows && a.m % tune.rows == 0 && tune.rows <= 256 ? tune.rows : rows_per_box(a.m, cap);
+    const size_t stage_bytes = (size_t)R * tile * 4;
+    int ctas = tune.ctas_per_sm ? tune.ctas_per_sm : 2;
+    int stages = tune.stages ? tune.stages : 0;
+    const size_t usable = (size_t)dev.smem_per_sm - 2048;  // leave room for the per-CTA reserve
+    if (!stages) {
+        stages = (int)((usable / ctas - 1024) / stage_bytes);
+        stages = std::min(stages, 8);
+    }
+    if (stages < 2) { ctas = 1; stages = (int)(((size_t)dev.smem_optin - 1024) / stage_bytes); stages = std::min(stages, 8); }
+    if (stages < 2) return cudaSuccess;  // does not fit: caller falls back to plain loads
+    const size_t smem = (size_t)stages * stage_bytes + (size_t)stages * 16 + 32;
+    if (smem > (size_t)dev.smem_optin) return cudaSuccess;
+
+    CUtensorMap map;
+    if (make_map(encode, &map, a, boxw, R) != CUDA_SUCCESS) return cudaSuccess;
+
+    FusedArgs fa;
+    fa.coeff = a.coeff; fa.steps = a.steps; fa.n_steps = a.total_steps; fa.m = a.m; fa.R = R; fa.cpn = a.m / R;
+    fa.stages = stages; fa.d = a.d; fa.ntiles = (a.d + tile - 1) / tile; fa.out = a.out; fa.shift = a.shift;
+    fa.status = a.status;
+    const long long max_grid = (long long)dev.sm_count * ctas;
+    const int grid = (int)std::min<long long>(fa.ntiles, max_grid);
+    cudaError_t err = a.is_int ? run_fused_ncw<int>(ncw, pick_lmax(a.L), map, fa, grid, smem, stream)
+                               : run_fused_ncw<float>(ncw, pick_lmax(a.L), map, fa, grid, smem, stream);
+    if (err == cudaSuccess) { *done = true; ++*launches; }
+    return err;
+}
+
+template <typename T, int LMAX, int NCW>
+static cudaError_t run_batch(const CUtensorMap &map, const BatchArgs &ba, int grid, size_t smem, cudaStream_t stream) {
+    auto kern = cr_fused_batch_tma_kernel<T, LMAX, NCW>;
+    cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) return err;
+    kern<<<grid, (NCW + 1) * 32, smem, stream>>>(map, ba);
+    return cudaGetLastError();
+}
+
+template <typename T, int NCW>
+static cudaError_t run_batch_l(int lmax, const CUtensorMap &map, const BatchArgs &ba, int grid, size_t smem,
+                               cudaStream_t stream) {
+    switch (lmax) {
+        case 2: return run_batch<T, 2, NCW>(map, ba, grid, smem, stream);
+        case 4: return run_batch<T, 4, NCW>(map, ba, grid, smem, stream);
+        default: return run_batch<T, 8, NCW>(map, ba, grid, smem, stream);
+    }
+}
+
+cudaError_t launch_fused_batch_tma(const AggArgs &a, const DeviceInfo &dev, const Tuning &tune, EncodeTiledFn encode,
+                                   cudaStream_t stream, int64_t *launches, bool *done) {
+    *done = false;
+    if (!encode || !tma_eligible(a)) return cudaSuccess;
+    const int tile = 128;
+    int R = tune.rows && a.m % tune.rows == 0 && tune.rows <= 256 ? tune.rows : rows_per_box(a.m, 16);
+    const size_t stage_bytes = (size_t)R * tile * 4;
+    const size_t e_bytes = (size_t)a.n_union * tile * 4;
+    const size_t usable = (size_t)dev.smem_per_sm - 2048;
+    int ctas = tune.ctas_per_sm ? tune.ctas_per_sm : 2;
+    int stages = 0;
+    for (; ctas >= 1; --ctas) {
+        const size_t budget = std::min(usable / ctas - 1024, (size_t)dev.smem_optin);
+        if (budget <= e_bytes + 64) continue;
+        stages = (int)((budget - e_bytes - 64) / stage_bytes);
+        if (stages >= 3 || (ctas == 1 && stages >= 2)) break;
+    }
+    if (ctas < 1 || stages < 2) return cudaSuccess;  // union too large for shared memory
+    stages = std::min(stages, tune.stages ? tune.stages : 8);
+    if (stages < 2) stages = 2;
+    const int ncw = (tune.ncw == 2 || tune.ncw == 4 || tune.ncw == 8) ? tune.ncw : 4;
+    const size_t smem = (size_t)stages * stage_bytes + e_bytes + (size_t)stages * 16 + 32;
+    if (smem > (size_t)dev.smem_optin) return cudaSuccess;
+    const long long ntiles = (a.d + tile - 1) / tile;
+    const int grid = (int)std::min<long long>(ntiles, (long long)dev.sm_count * ctas);
+    // ring iteration counters are 32-bit
+    if ((ntiles / grid + 1) * (long long)a.n_union * (a.m / R) >= (1ll << 31)) return cudaSuccess;
+
+    CUtensorMap map;
+    if (make_map(encode, &map, a, tile, R) != CUDA_SUCCESS) return cudaSuccess;
+
+    BatchArgs ba;
+    ba.coeff = a.coeff; ba.steps = a.steps; ba.pat_off = a.pat_off; ba.unodes = a.unodes; ba.n_union = a.n_union;
+    ba.batch = a.batch; ba.m = a.m; ba.R = R; ba.cpn = a.m / R; ba.stages = stages; ba.d = a.d; ba.ntiles = ntiles;
+    ba.out = a.out; ba.shift = a.shift; ba.status = a.status;
+    const int lmax = pick_lmax(a.L);
+    cudaError_t err;
+    if (a.is_int) {
+        err = ncw == 2 ? run_batch_l<int, 2>(lmax, map, ba, grid, smem, stream)
+            : ncw == 8 ? run_batch_l<int, 8>(lmax, map, ba, grid, smem, stream)
+                       : run_batch_l<int, 4>(lmax, map, ba, grid, smem, stream);
+    } else {
+        err = ncw == 2 ? run_batch_l<float, 2>(lmax, map, ba, grid, smem, stream)
+            : ncw == 8 ? run_batch_l<float, 8>(lmax, map, ba, grid, smem, stream)
+                       : run_batch_l<float, 4>(lmax, map, ba, grid, smem, stream);
+    }
+    if (err == cudaSuccess) { *done = true; ++*launches; }
+    return err;
+}
+
+template <typename T, int V>
+static cudaError_t run_ldg(const AggArgs &a, cudaStream_t stream) {
+    const long long threads = (a.d + V - 1) / V;
+    dim3 grid((unsigned)((threads + 255) / 256), (unsigned)a.batch);
+    const T *G = reinterpret_cast<const T *>(a.G);
+    const T *cf = reinterpret_cast<const T *>(a.coeff);
+    T *out = reinterpret_cast<T *>(a.out);
+    switch (pick_lmax(a.L)) {
+        case 2: cr_fused_ldg_kernel<T, 2, V><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift); break;
+        case 4: cr_fused_ldg_kernel<T, 4, V><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift); break;
+        default: cr_fused_ldg_kernel<T, 8, V><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift); break;
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_fused_ldg(const AggArgs &a, cudaStream_t stream, int64_t *launches) {
+    const bool v4 = vec4_ok(a.G, a.out, a.d);
+    cudaError_t err;
+    if (a.is_int) err = v4 ? run_ldg<int, 4>(a, stream) : run_ldg<int, 1>(a, stream);
+    else err = v4 ? run_ldg<float, 4>(a, stream) : run_ldg<float, 1>(a, stream);
+    if (err == cudaSuccess) ++*launches;
+    return err;
+}
+
+template <typename T, int V>
+static cudaError_t run_uncoded(const AggArgs &a, cudaStream_t stream) {
+    const long long threads = (a.d + V - 1) / V;
+    dim3 grid((unsigned)((threads + 255) / 256), (unsigned)a.batch);
+    cr_uncoded_sum_kernel<T, V><<<grid, 256, 0, stream>>>(reinterpret_cast<const T *>(a.G), a.steps, a.pat_off, a.m,
+                                                          a.d, reinterpret_cast<T *>(a.out));
+    return cudaGetLastError();
+}
+
+cudaError_t launch_uncoded_sum(const AggArgs &a, cudaStream_t stream, int64_t *launches) {
+    const bool v4 = vec4_ok(a.G, a.out, a.d);
+    cudaError_t err;
+    if (a.is_int) err = v4 ? run_uncoded<int, 4>(a, stream) : run_uncoded<int, 1>(a, stream);
+    else err = v4 ? run_uncoded<float, 4>(a, stream) : run_uncoded<float, 1>(a, stream);
+    if (err == cudaSuccess) ++*launches;
+    return err;
+}
+
+template <typename T, int V>
+static cudaError_t run_encode(const void *G, const void *coeff, const int32_t *nodes, int count, int m, int64_t d,
+                              void *E, cudaStream_t stream) {
+    const long long threads = (d + V - 1) / V;
+    dim3 grid((unsigned)((threads + 255) / 256), (unsigned)count);
+    cr_encode_kernel<T, V><<<grid, 256, 0, stream>>>(reinterpret_cast<const T *>(G), reinterpret_cast<const T *>(coeff),
+                                                     nodes, m, d, reinterpret_cast<T *>(E));
+    return cudaGetLastError();
+}
+
+cudaError_t launch_encode(const void *G, const void *coeff, const int32_t *nodes, int count, int m, int64_t d,
+                          void *E, int is_int, cudaStream_t stream, int64_t *launches) {
+    if (count <= 0) return cudaSuccess;
+    const bool v4 = vec4_ok(G, E, d);
+    cudaError_t err;
+    if (is_int) err = v4 ? run_encode<int, 4>(G, coeff, nodes, count, m, d, E, stream)
+                         : run_encode<int, 1>(G, coeff, nodes, count, m, d, E, stream);
+    else err = v4 ? run_encode<float, 4>(G, coeff, nodes, count, m, d, E, stream)
+                  : run_encode<float, 1>(G, coeff, nodes, count, m, d, E, stream);
+    if (err == cudaSuccess) ++*launches;
+    return err;
+}
+
+template <typename T, int V>
+static cudaError_t run_decode(const void *M_child, const void *E_parent, const void *W, const int32_t *active,
+                              int parents, int n, int64_t d, void *M_parent, int shift, cudaStream_t stream) {
+    const long long threads = (d + V - 1) / V;
+    dim3 grid((unsigned)((threads + 255) / 256), (unsigned)parents);
+    cr_decode_kernel<T, V><<<grid, 256, 0, stream>>>(reinterpret_cast<const T *>(M_child),
+                                                     reinterpret_cast<const T *>(E_parent),
+                                                     reinterpret_cast<const T *>(W), active, n, d,
+                                                     reinterpret_cast<T *>(M_parent), shift);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_decode(const void *M_child, const void *E_parent, const void *W, const int32_t *active,
+                          int parents, int n, int64_t d, void *M_parent, int shift, int is_int,
+                          cudaStream_t stream, int64_t *launches) {
+    const bool v4 = d % 4 == 0 && aligned16(M_child) && aligned16(M_parent) && (!E_parent || aligned16(E_parent));
+    cudaError_t err;
+    if (is_int) err = v4 ? run_decode<int, 4>(M_child, E_parent, W, active, parents, n, d, M_parent, shift, stream)
+                         : run_decode<int, 1>(M_child, E_parent, W, active, parents, n, d, M_parent, shift, stream);
+    else err = v4 ? run_decode<float, 4>(M_child, E_parent, W, active, parents, n, d, M_parent, shift, stream)
+                  : run_decode<float, 1>(M_child, E_parent, W, active, parents, n, d, M_parent, shift, stream);
+    if (err == cudaSuccess) ++*launches;
+    return err;
+}
+
+cudaError_t launch_partial_gradients(const float *X, const float *y, const float *w, const int32_t *part,
+                                     int items, int rows, int64_t d, float *resid, float *G,
+                                     cudaStream_t stream, int64_t *launches) {
+    const bool v4 = d % 4 == 0 && aligned16(X) && aligned16(w) && aligned16(G);
+    const long long total_rows = (long long)items * rows;
+    const long long want_blocks = (total_rows + 7) / 8;  // 8 warps per block
+    const int blocks = (int)std::min<long long>(want_blocks, 148 * 32);
+    if (v4) cr_residual_kernel<4><<<blocks, 256, 0, stream>>>(X, y, w, part, total_rows, rows, d, resid);
+    else cr_residual_kernel<1><<<blocks, 256, 0, stream>>>(X, y, w, part, total_rows, rows, d, resid);
+    cudaError_t err = cudaGetLastError();
+    if (err != cudaSuccess) return err;
+    ++*launches;
+    if (v4) {
+        dim3 grid((unsigned)((d / 4 + 127) / 128), (unsigned)items);
+        cr_xt_r_kernel<4><<<grid, 128, 0, stream>>>(X, part, resid, rows, d, G);
+    } else {
+        dim3 grid((unsigned)((d + 127) / 128), (unsigned)items);
+        cr_xt_r_kernel<1><<<grid, 128, 0, stream>>>(X, part, resid, rows, d, G);
+    }
+    err = cudaGetLastError();
+    if (err == cudaSuccess) ++*launches;
+    return err;
+}
+
+}  // namespace cr

@@ -1,0 +1,84 @@
+// Launch wrappers of the sm_100a kernels (implemented in cr_kernels.cu).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+namespace cr {
+
+// One consumed node of an expanded straggler pattern, as the kernels read it (16 bytes).
+struct Step {
+    int32_t node;    // flat node index: its slots are rows node*m .. node*m+m-1 of G_slots
+    int32_t layer;   // 1..L
+    uint32_t wbits;  // decode weight of the node's message at its parent: float bits (CR_F32) or int32 (CR_I32)
+    int32_t index;   // batch kernel: position of the node in the union list; otherwise unused
+};
+
+// Tuning of the TMA kernels; 0 selects the built-in choice.
+struct Tuning {
+    int ncw = 0;          // consumer warps per CTA (single-pattern kernel: tile = 128 * ncw columns)
+    int stages = 0;       // depth of the shared-memory ring
+    int ctas_per_sm = 0;  // persistent CTAs per SM
+    int rows = 0;         // slot rows per TMA box (must divide m)
+};
+
+struct DeviceInfo {
+    int sm_count = 0;
+    int smem_optin = 0;  // bytes of dynamic shared memory a CTA may opt in to
+    int smem_per_sm = 0;
+};
+
+struct AggArgs {
+    const void *G;        // [N*m][d]
+    const void *coeff;    // [N*m] element type T
+    const Step *steps;    // device: all patterns' steps, concatenated
+    const int32_t *pat_off;  // device [batch+1]: pattern b owns steps pat_off[b] .. pat_off[b+1]-1
+    const int32_t *unodes;   // device [n_union]: union of used nodes (batch kernel)
+    int n_union;
+    int batch;
+    int total_steps;
+    int m;
+    int L;
+    int64_t d;
+    int64_t rows_total;   // N*m
+    void *out;            // [batch][d]
+    int shift;            // CR_I32: arithmetic right shift applied at the root
+    int *status;          // device status word (bounded waits)
+    int is_int;
+};
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// Each returns cudaSuccess or the first CUDA error; *launches is incremented per kernel launched.
+// `can_tma` tells whether d and the pointers meet the TMA alignment rules.
+bool tma_eligible(const AggArgs &a);
+
+cudaError_t launch_fused_tma(const AggArgs &a, const DeviceInfo &dev, const Tuning &tune, EncodeTiledFn encode,
+                             cudaStream_t stream, int64_t *launches, bool *done);
+cudaError_t launch_fused_batch_tma(const AggArgs &a, const DeviceInfo &dev, const Tuning &tune, EncodeTiledFn encode,
+                                   cudaStream_t stream, int64_t *launches, bool *done);
+cudaError_t launch_fused_ldg(const AggArgs &a, cudaStream_t stream, int64_t *launches);
+cudaError_t launch_uncoded_sum(const AggArgs &a, cudaStream_t stream, int64_t *launches);
+
+// E[v][:] = sum_j coeff[v*m+j] * G[v*m+j][:] for the nodes listed in `nodes` (device, count entries) or
+// for all N nodes when nodes == nullptr.
+cudaError_t launch_encode(const void *G, const void *coeff, const int32_t *nodes, int count, int m, int64_t d,
+                          void *E, int is_int, cudaStream_t stream, int64_t *launches);
+
+// One level of decode: for parent i < parents: M_parent[i] = sum_j W[i*n+j] * M_child[n*i+j] (+ E_parent[i]);
+// parents with active[i] == 0 are skipped.  W and active are device arrays.
+cudaError_t launch_decode(const void *M_child, const void *E_parent, const void *W, const int32_t *active,
+                          int parents, int n, int64_t d, void *M_parent, int shift, int is_int,
+                          cudaStream_t stream, int64_t *launches);
+
+// Partial gradients of linear regression, two passes over X: residuals r = X_p w - y_p into `resid`
+// ([items][rows]), then G[item][:] = X_p^T r.  part[item] is the partition of slot `item`.
+cudaError_t launch_partial_gradients(const float *X, const float *y, const float *w, const int32_t *part,
+                                     int items, int rows, int64_t d, float *resid, float *G,
+                                     cudaStream_t stream, int64_t *launches);
+
+}  // namespace cr

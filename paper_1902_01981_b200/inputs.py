@@ -92,3 +92,24 @@ def replicate_into_slots(G_parts: np.ndarray, slot_partition: np.ndarray) -> np.
     movement; `slot_partition` comes from whoever planned the allocation).
     """
     return G_parts[np.asarray(slot_partition, dtype=np.int64)]
+
+
+# Benchmark workloads.  Tree shape, partition count, gradient length and value model of each; no
+# arithmetic of the scheme.  `code` names the encoding-matrix family ("printed_3_1": the matrices the
+# paper prints for n=3, s=1; "cyclic": random cyclic-support code; "repetition": 0/1 fractional
+# repetition).  `P` of cfg3 is 48, the nearest count above the nominal 40 that the (4,2,1) tree can
+# split into whole chunks.
+CONFIGS = {
+    "cfg1": dict(n=3, L=1, s=1, P=6, d=256, rows=64, code="printed_3_1", kind="linreg", x_std=1.0,
+                 noise_std=0.01, iters=10, lr=5e-4, seed=0),
+    "cfg2": dict(n=4, L=2, s=1, P=24, d=1 << 20, code="cyclic", kind="aggregate", std=1.0, iters=100,
+                 batch=1, exactly_s=False, seed=0, mask_seed=1),
+    "cfg3": dict(n=4, L=2, s=1, P=48, d=4096, rows=2048, code="cyclic", kind="linreg", x_std=1.0 / 64.0,
+                 noise_std=0.01, iters=50, lr=0.1, seed=0, mask_seed=1),
+    "cfg4": dict(n=5, L=2, s=2, P=40, d=1 << 24, code="cyclic", kind="aggregate", std=1e-3 ** 0.5, iters=20,
+                 batch=1, exactly_s=True, seed=0, mask_seed=1),
+    "cfg5": dict(n=3, L=4, s=1, P=195, d=1 << 22, code="printed_3_1", kind="aggregate", std=1.0, iters=5,
+                 batch=64, exactly_s=False, seed=0, mask_seed=1, int_bound=1 << 10),
+    "cfg_rep": dict(n=4, L=2, s=1, P=24, d=1 << 20, code="repetition", kind="aggregate", std=1.0, iters=20,
+                    batch=1, exactly_s=False, seed=0, mask_seed=1, int_bound=1 << 10),
+}

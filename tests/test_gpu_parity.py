@@ -1,0 +1,246 @@
+"""CUDA path against the CPU oracle, element by element, through the C ABI."""
+from itertools import combinations, product
+
+import numpy as np
+import pytest
+
+from oracle import cr_oracle as O
+from oracle import cr_setup
+from paper_1902_01981_b200 import binding as B
+from paper_1902_01981_b200 import build as cr_build
+from paper_1902_01981_b200 import inputs
+from tests.gpu_common import CODE_ID, REL_L2_BAR, check_slot_table, make_plan, rel_l2, slots_on_device
+
+pytestmark = pytest.mark.gpu
+torch = pytest.importorskip("torch")
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    cr_build.build()
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+
+
+def tree(n, L, s, code, d, P=None, **kw):
+    return dict(n=n, L=L, s=s, P=P or O.partition_quantum(n, L, s), d=d, code=code, **kw)
+
+
+FUSED_VARIANTS = [B.CR_AGG_FUSED, B.CR_AGG_FUSED_LDG, B.CR_AGG_UNFUSED, B.CR_AGG_UNFUSED | B.CR_AGG_ALL_NODES]
+
+
+def run_aggregate(plan, G_dev, masks, d, flags, dtype=torch.float32):
+    masks = np.asarray(masks, dtype=np.uint32).reshape(-1, B.cr_plan_num_groups(plan))
+    out = torch.full((masks.shape[0], d), 7, dtype=dtype, device="cuda")
+    ws = None
+    nbytes = B.cr_aggregate_workspace_bytes(plan, masks.shape[0], flags)
+    if nbytes:
+        ws = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    B.cr_aggregate(plan, G_dev, masks, out, flags, ws)
+    torch.cuda.synchronize()
+    assert B.cr_plan_device_status(plan) == B.CR_OK
+    return out.cpu().numpy()
+
+
+def all_patterns(n, L, s):
+    per_group = [sum(1 << j for j in S) for k in range(s + 1) for S in combinations(range(n), k)]
+    return np.array(list(product(per_group, repeat=O.num_groups(n, L))), dtype=np.uint32)
+
+
+# --------------------------------------------------------------------------- unfused steps
+
+@pytest.mark.parametrize("cfg", [tree(3, 2, 1, "printed_3_1", 2500), tree(4, 2, 1, "cyclic", 1027),
+                                 tree(3, 3, 1, "printed_3_1", 4096), tree(5, 2, 2, "cyclic", 3000, P=80)])
+def test_encode_and_decode_levels(cfg):
+    n, L, s, d = cfg["n"], cfg["L"], cfg["s"], cfg["d"]
+    plan = make_plan(cfg)
+    try:
+        code, local = check_slot_table(plan, cfg)
+        G = inputs.partition_gradients(cfg["P"], d, seed=21)
+        G_dev = slots_on_device(plan, G, torch)
+        N = O.num_nodes(n, L)
+        E = torch.zeros((N, d), device="cuda")
+        B.cr_encode(plan, G_dev, E)
+        E_or = O.encode_all(local, G)
+        for v in range(N):
+            assert rel_l2(E[v].cpu().numpy(), E_or[v]) <= REL_L2_BAR
+        masks = inputs.straggler_masks(n, L, s, 1, seed=5)[0]
+        g_or, M_or = O.execute_levels(code, local, G, masks)
+        M = {L: E[O.layer_offset(n, L):]}
+        for l in range(L - 1, -1, -1):
+            parents = n ** l
+            groups = [0] if l == 0 else [O.layer_offset(n, l) + i + 1 for i in range(parents)]
+            M[l] = torch.zeros((parents, d), device="cuda")
+            E_par = None if l == 0 else E[O.layer_offset(n, l): O.layer_offset(n, l) + parents]
+            B.cr_decode(plan, l, M[l + 1].contiguous(), E_par, masks[groups], M[l])
+            if l > 0:
+                for i in range(parents):
+                    assert rel_l2(M[l][i].cpu().numpy(), M_or[l][i]) <= REL_L2_BAR
+        assert rel_l2(M[0][0].cpu().numpy(), g_or) <= REL_L2_BAR
+        assert rel_l2(M[0][0].cpu().numpy(), O.full_gradient(G)) <= REL_L2_BAR
+    finally:
+        B.cr_plan_destroy(plan)
+
+
+# --------------------------------------------------------------------------- aggregate, all variants
+
+@pytest.mark.parametrize("cfg", [tree(3, 1, 1, "printed_3_1", 256, P=6), tree(3, 2, 1, "printed_3_1", 1536),
+                                 tree(4, 2, 1, "cyclic", 2052), tree(5, 1, 2, "cyclic", 777),
+                                 tree(4, 2, 1, "repetition", 1300), tree(4, 1, 1, "repetition", 260)])
+@pytest.mark.parametrize("flags", FUSED_VARIANTS)
+def test_every_pattern_on_tiny_trees(cfg, flags):
+    n, L, s, d = cfg["n"], cfg["L"], cfg["s"], cfg["d"]
+    plan = make_plan(cfg)
+    try:
+        code, local = check_slot_table(plan, cfg)
+        G = inputs.partition_gradients(cfg["P"], d, seed=3)
+        G_dev = slots_on_device(plan, G, torch)
+        pats = all_patterns(n, L, s)
+        if len(pats) > 700:                      # (4,2,1): 3125 patterns; a spread of 700 keeps the oracle quick
+            pats = pats[np.random.default_rng(0).choice(len(pats), 700, replace=False)]
+        want_sum = O.full_gradient(G)
+        got = np.concatenate([run_aggregate(plan, G_dev, pats[i:i + 256], d, flags) for i in range(0, len(pats), 256)])
+        for b in range(0, len(pats), max(1, len(pats) // 40)):        # oracle algorithm on a subset
+            assert rel_l2(got[b], O.execute(code, local, G, pats[b])) <= REL_L2_BAR
+        for b in range(len(pats)):                                     # the plain definition on all
+            assert rel_l2(got[b], want_sum) <= REL_L2_BAR
+        # single-pattern launches take the single-pattern kernel
+        for b in (0, len(pats) // 2, len(pats) - 1):
+            one = run_aggregate(plan, G_dev, pats[b], d, flags)[0]
+            assert rel_l2(one, O.execute(code, local, G, pats[b])) <= REL_L2_BAR
+    finally:
+        B.cr_plan_destroy(plan)
+
+
+@pytest.mark.parametrize("cfg,batch", [(tree(4, 2, 1, "cyclic", 1 << 15), 9), (tree(5, 2, 2, "cyclic", 70000, P=80), 5),
+                                       (tree(3, 4, 1, "printed_3_1", 5000), 64), (tree(4, 3, 1, "cyclic", 4100), 7),
+                                       (tree(2, 5, 0, "cyclic", 1000), 2), (tree(12, 2, 3, "cyclic", 1200, max_kappa=1e6), 3)])
+@pytest.mark.parametrize("flags", FUSED_VARIANTS)
+def test_random_patterns_medium_trees(cfg, batch, flags):
+    n, L, s, d = cfg["n"], cfg["L"], cfg["s"], cfg["d"]
+    plan = make_plan(cfg)
+    try:
+        code, local = check_slot_table(plan, cfg)
+        G = inputs.partition_gradients(cfg["P"], d, seed=8)
+        G_dev = slots_on_device(plan, G, torch)
+        masks = inputs.straggler_masks(n, L, s, batch, seed=4, exactly_s=(n == 5))
+        bar = REL_L2_BAR if n < 12 else 1e-3     # (12,2,3): kappa in the thousands, outside the 1e-5 regime
+        got = run_aggregate(plan, G_dev, masks, d, flags)
+        for b in range(batch):
+            assert rel_l2(got[b], O.execute(code, local, G, masks[b])) <= bar
+        one = run_aggregate(plan, G_dev, masks[batch - 1], d, flags)[0]
+        assert rel_l2(one, O.execute(code, local, G, masks[batch - 1])) <= bar
+    finally:
+        B.cr_plan_destroy(plan)
+
+
+def test_fused_matches_unfused_closely():
+    cfg = tree(5, 2, 2, "cyclic", 1 << 16)
+    plan = make_plan(cfg)
+    try:
+        G = inputs.partition_gradients(cfg["P"], cfg["d"], seed=1)
+        G_dev = slots_on_device(plan, G, torch)
+        masks = inputs.straggler_masks(5, 2, 2, 4, seed=2, exactly_s=True)
+        ref = run_aggregate(plan, G_dev, masks, cfg["d"], B.CR_AGG_UNFUSED)
+        for flags in (B.CR_AGG_FUSED, B.CR_AGG_FUSED_LDG):
+            got = run_aggregate(plan, G_dev, masks, cfg["d"], flags)
+            assert max(rel_l2(got[b], ref[b]) for b in range(4)) <= 1e-6
+            one = run_aggregate(plan, G_dev, masks[0], cfg["d"], flags)[0]
+            assert rel_l2(one, ref[0]) <= 1e-6
+    finally:
+        B.cr_plan_destroy(plan)
+
+
+def test_uncoded_sum_reads_the_same_slots():
+    cfg = tree(4, 2, 1, "cyclic", 3000)
+    plan = make_plan(cfg)
+    try:
+        G = inputs.partition_gradients(cfg["P"], cfg["d"], seed=1)
+        G_dev = slots_on_device(plan, G, torch)
+        masks = inputs.straggler_masks(4, 2, 1, 3, seed=2)
+        got = run_aggregate(plan, G_dev, masks, cfg["d"], B.CR_AGG_UNCODED_SUM)
+        part = B.slot_partitions(plan)
+        for b in range(3):
+            nodes, _, _ = B.cr_plan_expand(plan, masks[b])
+            want = sum(G[p].astype(np.float64) for v in nodes for p in part[v])
+            assert rel_l2(got[b], want) <= REL_L2_BAR
+    finally:
+        B.cr_plan_destroy(plan)
+
+
+# --------------------------------------------------------------------------- integer-exact mode
+
+@pytest.mark.parametrize("cfg,batch", [(tree(3, 2, 1, "printed_3_1", 1200), 20), (tree(3, 4, 1, "printed_3_1", 4104), 64),
+                                       (tree(4, 2, 1, "repetition", 2000), 16), (tree(6, 2, 2, "repetition", 520), 8)])
+@pytest.mark.parametrize("flags", FUSED_VARIANTS)
+def test_integer_mode_is_bit_exact(cfg, batch, flags):
+    n, L, s, d = cfg["n"], cfg["L"], cfg["s"], cfg["d"]
+    plan = make_plan(cfg, dtype=B.CR_I32)
+    try:
+        code, local = check_slot_table(plan, cfg)
+        G = inputs.integer_gradients(cfg["P"], d, seed=12)
+        G_dev = slots_on_device(plan, G, torch)
+        masks = inputs.straggler_masks(n, L, s, batch, seed=13)
+        got = run_aggregate(plan, G_dev, masks, d, flags, dtype=torch.int32)
+        want = G.astype(np.int64).sum(0)
+        for b in range(batch):
+            assert np.array_equal(got[b].astype(np.int64), want)
+        assert np.array_equal(O.execute_integer(code, local, G, masks[0]), want)
+        one = run_aggregate(plan, G_dev, masks[1], d, flags, dtype=torch.int32)[0]
+        assert np.array_equal(one.astype(np.int64), want)
+    finally:
+        B.cr_plan_destroy(plan)
+
+
+# --------------------------------------------------------------------------- partial gradients
+
+@pytest.mark.parametrize("cfg,rows", [(tree(3, 1, 1, "printed_3_1", 256, P=6), 64), (tree(4, 2, 1, "cyclic", 1000), 100),
+                                      (tree(3, 2, 1, "printed_3_1", 1027), 37), (tree(4, 2, 1, "cyclic", 4096, P=48), 96)])
+def test_partial_gradients(cfg, rows):
+    n, L, s, d, P = cfg["n"], cfg["L"], cfg["s"], cfg["d"], cfg["P"]
+    plan = make_plan(cfg)
+    try:
+        X, y, w_star = inputs.linreg_partitions(P, rows, d, seed=2, x_std=1.0 / np.sqrt(d))
+        w = inputs.model_vector(d, seed=3)
+        N, m = B.cr_plan_num_nodes(plan), B.cr_plan_load(plan)
+        G_slots = torch.zeros((N, m, d), device="cuda")
+        ws = torch.empty(B.cr_partial_gradients_workspace_bytes(plan, rows), dtype=torch.uint8, device="cuda")
+        B.cr_partial_gradients(plan, torch.from_numpy(X).cuda(), torch.from_numpy(y).cuda(), rows,
+                               torch.from_numpy(w).cuda(), G_slots, ws)
+        torch.cuda.synchronize()
+        got = G_slots.cpu().numpy()
+        part = B.slot_partitions(plan)
+        want = [O.partial_gradient_linreg(X[p], y[p], w) for p in range(P)]
+        for v in range(N):
+            for j in range(m):
+                assert rel_l2(got[v, j], want[part[v, j]]) <= REL_L2_BAR
+    finally:
+        B.cr_plan_destroy(plan)
+
+
+# --------------------------------------------------------------------------- error paths
+
+def test_device_error_paths():
+    cfg = tree(4, 2, 1, "cyclic", 512)
+    plan = make_plan(cfg)
+    try:
+        G_dev = torch.zeros((20, 4, 512), device="cuda")
+        out = torch.zeros((1, 512), device="cuda")
+        with pytest.raises(B.CodedReduceError) as e:
+            B.cr_aggregate(plan, G_dev, [0b0101, 0, 0, 0, 0], out)
+        assert e.value.status == B.CR_ERR_UNDECODABLE_MASK
+        with pytest.raises(B.CodedReduceError) as e:
+            B.cr_aggregate(plan, G_dev, [0, 0, 0, 0, 0], out, B.CR_AGG_UNFUSED, None)
+        assert e.value.status == B.CR_ERR_OOM
+        with pytest.raises(B.CodedReduceError) as e:
+            B.cr_aggregate(plan, G_dev, [0, 0, 0, 0, 0], out, 0x55)
+        assert e.value.status == B.CR_ERR_INVALID_ARG
+        # ALL_NODES decodes every group, so an over-full mask below a straggler is an error there
+        ws = torch.empty(B.cr_aggregate_workspace_bytes(plan, 1, B.CR_AGG_UNFUSED), dtype=torch.uint8, device="cuda")
+        with pytest.raises(B.CodedReduceError) as e:
+            B.cr_aggregate(plan, G_dev, [0b0001, 0b0110, 0, 0, 0], out, B.CR_AGG_UNFUSED | B.CR_AGG_ALL_NODES, ws)
+        assert e.value.status == B.CR_ERR_UNDECODABLE_MASK
+        B.cr_aggregate(plan, G_dev, [0b0001, 0b0110, 0, 0, 0], out, B.CR_AGG_UNFUSED, ws)   # ignored when unused
+        torch.cuda.synchronize()
+        assert B.cr_plan_launch_count(plan) > 0
+    finally:
+        B.cr_plan_destroy(plan)
