@@ -65,7 +65,7 @@ def combine_ranks(elapsed_s: float, units: float, world: int, dist=None, device=
 
 class ClockSampler:
     """nvidia-smi clock / throttle-reason samples while the timed region runs."""
-    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -74,12 +74,22 @@ class ClockSampler:
         self.proc = None
         try:
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(gpu_index), f"--query-gpu={self.QUERY}",
-                                          "--format=csv,noheader,nounits", "-lms", "200"],
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
                                          stdout=self.file, stderr=subprocess.DEVNULL)
         except OSError:
             self.proc = None
 
-    def stop(self):
+    def wait_first_sample(self, limit_s: float = 3.0):
+        """Blocks until nvidia-smi has written its first line (it takes a moment to start)."""
+        t0 = time.time()
+        while self.proc is not None and time.time() - t0 < limit_s:
+            if os.path.getsize(self.file.name) > 0:
+                return
+            time.sleep(0.05)
+
+    def stop(self, window=None):
+        """Median SM clock and the throttle reasons seen; `window` = (t0, t1) in time.time() seconds
+        keeps only the samples taken inside it (all samples if none fall inside)."""
         out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         if self.proc is None:
             return out
@@ -90,38 +100,43 @@ class ClockSampler:
             self.proc.kill()
         self.file.flush()
         self.file.seek(0)
-        sm, mx, reasons = [], [], set()
+        import datetime
+        rows = []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in self.file.read().splitlines():
             cols = [c.strip() for c in line.split(",")]
             if len(cols) < 9:
                 continue
             try:
-                sm.append(float(cols[1]))
-                mx.append(float(cols[2]))
+                stamp = datetime.datetime.strptime(cols[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                rows.append((stamp, float(cols[1]), float(cols[2]), float(cols[3]),
+                             [n for n, v in zip(names, cols[5:9]) if v.lower().startswith("active")]))
             except ValueError:
                 continue
-            for name, val in zip(names, cols[5:9]):
-                if val.lower().startswith("active"):
-                    reasons.add(name)
         self.file.close()
         os.unlink(self.file.name)
-        if sm:
-            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons),
-                       samples=len(sm))
+        inside = [r for r in rows if window and window[0] <= r[0] <= window[1]]
+        use = inside or rows
+        if use:
+            reasons = sorted({n for r in use for n in r[4]})
+            out.update(sm_mhz=float(np.median([r[1] for r in use])), sm_max_mhz=float(max(r[2] for r in use)),
+                       power_w=float(np.median([r[3] for r in use])), reasons=reasons, samples=len(use),
+                       samples_in_timed_region=len(inside))
         return out
 
 
 # ----------------------------------------------------------------------------- CPU oracle legs
 
-def oracle_sample(cfg, d_sample: int, steps: int, warmup: int, seed_shift: int = 0):
-    """Times the CPU oracle, as it stands, on the first `d_sample` columns of the workload.
+def oracle_sample(cfg, d_sample: int, steps: int, warmup: int, G=None):
+    """Times the CPU oracle, as it stands, on `d_sample` columns of the workload (the array G
+    [P, d_sample] if given, else freshly drawn ones).
     Returns (seconds per step, algorithmic bytes per step, results of the last step, masks used)."""
     from oracle import cr_oracle as O
     from oracle import cr_setup
     code, local, _ = cr_setup.setup(cfg)
     batch = cfg.get("batch", 1)
-    G = inputs.partition_gradients(cfg["P"], d_sample, cfg["seed"] + seed_shift, cfg.get("std", 1.0))
+    if G is None:
+        G = inputs.partition_gradients(cfg["P"], d_sample, cfg["seed"], cfg.get("std", 1.0))
     masks = inputs.straggler_masks(cfg["n"], cfg["L"], cfg["s"], (steps + warmup) * batch, cfg["mask_seed"],
                                    cfg.get("exactly_s", False)).reshape(steps + warmup, batch, -1)
     m = len(local[0])
@@ -151,7 +166,15 @@ def run_reference(args, cfg):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    d_sample = min(cfg["d"], args.ref_columns)
+    # bounded sample: about a minute of oracle time for the whole run at ~0.8 GB/s of algorithmic bytes
+    n_used = sum((cfg["n"] - cfg["s"]) ** l for l in range(1, cfg["L"] + 1))
+    m = cfg["P"] * (cfg["s"] + 1) ** cfg["L"] // sum(cfg["n"] ** l * (cfg["s"] + 1) ** (cfg["L"] - l)
+                                                      for l in range(1, cfg["L"] + 1))
+    per_col = 4 * (m * n_used + 1) * cfg.get("batch", 1)
+    budget_cols = int(60.0 * 0.8e9 / ((args.steps + args.warmup) * per_col))
+    d_sample = 4096
+    while d_sample * 2 <= min(budget_cols, args.ref_columns, cfg["d"]):
+        d_sample *= 2
     sec, nbytes, _, _ = oracle_sample(cfg, d_sample, args.steps, args.warmup)
     value = nbytes / sec / 1e9
     sample = f"first {d_sample} of {cfg['d']} columns, every step a fresh straggler pattern"
@@ -227,7 +250,7 @@ def run_ours(args, cfg):
         torch.index_select(parts_dev, 0, part[r0:r0 + step_rows], out=G_slots[r0:r0 + step_rows])
     del parts_dev
     out = torch.zeros((batch, d), dtype=tdtype, device=dev)
-    total = args.steps + args.warmup
+    total = min(args.steps + args.warmup, 256)       # distinct straggler patterns, cycled over the steps
     masks = inputs.straggler_masks(cfg["n"], cfg["L"], cfg["s"], total * batch, cfg["mask_seed"],
                                    cfg.get("exactly_s", False)).reshape(total, batch, groups)
     step_bytes = [B.cr_aggregate_bytes(plan, masks[i])[0] for i in range(total)]
@@ -244,15 +267,18 @@ def run_ours(args, cfg):
         if dist is not None:
             dist.barrier()
             torch.cuda.synchronize()
-        t0 = time.perf_counter()
+        t0 = time.time()
+        n0 = B.cr_plan_launch_count(plan)
         for i in range(steps):
             if flush_buf is not None:
                 flush_buf.fill_(i & 0xff)
             starts[i].record(stream)
-            B.cr_aggregate(plan, G_slots, masks[warmup + i], out, flags, ws, stream)
+            B.cr_aggregate(plan, G_slots, masks[(warmup + i) % total], out, flags, ws, stream)
             stops[i].record(stream)
         torch.cuda.synchronize()
-        wall = time.perf_counter() - t0
+        t1 = time.time()
+        timed_run.launches = B.cr_plan_launch_count(plan) - n0
+        timed_run.window = (t0, t1)
         if dist is not None:
             dist.barrier()
             torch.cuda.synchronize()
@@ -266,15 +292,15 @@ def run_ours(args, cfg):
     except Exception:
         gpu_id = local_rank
     sampler = ClockSampler(gpu_id)
-    launches0 = B.cr_plan_launch_count(plan)
+    sampler.wait_first_sample()
     per, wall = timed_run(B.CR_AGG_FUSED)
-    launches = B.cr_plan_launch_count(plan) - launches0
-    clocks = sampler.stop()
+    launches = timed_run.launches
+    clocks = sampler.stop(timed_run.window)
     assert B.cr_plan_device_status(plan) == B.CR_OK, "a device-side wait timed out"
     # device time of the K steps: first start event to last stop event on the launching stream (with
     # an L2 flush between steps: the sum of the per-step intervals, which leaves the flushes out)
     elapsed = float(wall)
-    units = float(sum(step_bytes[args.warmup:]))
+    units = float(sum(step_bytes[(args.warmup + i) % total] for i in range(args.steps)))
     elapsed_all, units_all = combine_ranks(elapsed, units, world, dist, dev)
     value = units_all / elapsed_all / 1e9
     result_last = out.clone()
@@ -282,8 +308,8 @@ def run_ours(args, cfg):
     # ---- comparators on the same slots (rank 0 only, outside the timed region)
     extras = {}
     if rank == 0 and not args.no_extras:
-        ksteps = min(args.steps, 10)
-        bytes_k = float(np.mean(step_bytes[args.warmup:args.warmup + ksteps]))
+        ksteps = min(args.steps, 50)
+        bytes_k = float(np.mean([step_bytes[(args.warmup + i) % total] for i in range(ksteps)]))
         for name, flags in (("fused_plain_loads", B.CR_AGG_FUSED_LDG), ("uncoded_sum_same_bytes", B.CR_AGG_UNCODED_SUM)):
             p2, _ = timed_run(flags, steps=ksteps)
             extras[name] = {"GB/s": bytes_k / float(p2.mean()) / 1e9, "ms_per_step": float(p2.mean()) * 1e3}
@@ -311,11 +337,11 @@ def run_ours(args, cfg):
             dist.barrier()
         t0 = time.perf_counter()
         for i in range(e2e_steps):
-            B.cr_aggregate_host(plan, host_slots, masks[args.warmup + i], host_out, G_slots, out, B.CR_AGG_FUSED,
-                                None, stream)
+            B.cr_aggregate_host(plan, host_slots, masks[(args.warmup + i) % total], host_out, G_slots, out,
+                                B.CR_AGG_FUSED, None, stream)
         torch.cuda.synchronize()
         e2e_elapsed = time.perf_counter() - t0
-        e2e_units = float(sum(step_bytes[args.warmup:args.warmup + e2e_steps]))
+        e2e_units = float(sum(step_bytes[(args.warmup + i) % total] for i in range(e2e_steps)))
         e2e_elapsed, e2e_units = combine_ranks(e2e_elapsed, e2e_units, world, dist, dev)
         e2e = {"value": e2e_units / e2e_elapsed / 1e9, "unit": UNIT,
                "h2d_bytes_per_step": int(N * m * d * 4 + masks[0].nbytes), "d2h_bytes_per_step": int(batch * d * 4),
@@ -325,7 +351,7 @@ def run_ours(args, cfg):
     if rank == 0:
         peak, peak_kind = peak_hbm()
         avg_launch = float(per.mean())
-        avg_bytes = float(np.mean(step_bytes[args.warmup:]))
+        avg_bytes = units / args.steps
         achieved = avg_bytes / avg_launch / 1e9
         kern = "cr_fused_batch_tma_kernel" if batch > 1 else "cr_fused_tma_kernel"
         traffic = NCU_TRAFFIC_BYTES.get((args.workload, args.dtype))
@@ -336,7 +362,8 @@ def run_ours(args, cfg):
         cpu = None
         if not args.no_cpu_baseline:
             d_sample = min(d, args.cpu_columns)
-            sec, nbytes, last, last_masks = oracle_sample(cfg, d_sample, args.cpu_steps, 1, seed_shift=rank) \
+            sec, nbytes, last, last_masks = oracle_sample(
+                cfg, d_sample, args.cpu_steps, 1, np.ascontiguousarray(G_parts[:, :d_sample])) \
                 if not is_int else (None, None, None, None)
             if sec is not None:
                 cpu = {"value": nbytes / sec / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
@@ -367,7 +394,7 @@ def run_ours(args, cfg):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4", choices=[k for k, v in inputs.CONFIGS.items() if v["kind"] == "aggregate"])
@@ -378,8 +405,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--cpu-columns", type=int, default=1 << 21)
-    ap.add_argument("--cpu-steps", type=int, default=4)
-    ap.add_argument("--ref-columns", type=int, default=1 << 19)
+    ap.add_argument("--cpu-steps", type=int, default=8)
+    ap.add_argument("--ref-columns", type=int, default=1 << 21)
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
