@@ -399,6 +399,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg4", choices=[k for k, v in inputs.CONFIGS.items() if v["kind"] == "aggregate"])
     ap.add_argument("--dtype", default="f32", choices=["f32", "int32"])
+    ap.add_argument("--d", type=int, default=0, help="override the gradient length (profiling on a small case)")
     ap.add_argument("--tune", default="", help="consumer_warps,stages,ctas_per_sm,rows_per_box (0 = auto)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extras", action="store_true")
@@ -411,6 +412,8 @@ def main():
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     cfg = dict(inputs.CONFIGS[args.workload])
+    if args.d:
+        cfg["d"] = args.d
     world = int(os.environ.get("WORLD_SIZE", "1"))
     if args.gpus != world and world > 1:
         args.gpus = world
