@@ -150,6 +150,27 @@ cr_status_t cr_partial_gradients(cr_plan_t *plan, const float *X, const float *y
                                  const float *w, float *G_slots, void *workspace,
                                  size_t workspace_bytes, void *stream);
 
+/* ---- the same partial-gradient pass for callers that cannot allocate device memory ----------------
+ * (No counterpart in the paper: this is a packaging variant of cr_partial_gradients.)
+ * Some callers have no way to provide the residual workspace: a host thread that runs inside a
+ * latency-critical loop where cudaMalloc would stall the whole device, a process whose device memory
+ * has been handed in full to another component's pool, a plug-in that is given raw pointers and a
+ * stream but no allocator.  For them the residuals (one float per node, slot and row) live in a fixed
+ * array inside the library: 4 MiB of device memory on every GPU that loads the library, kept until the
+ * process exits.  Arguments, layouts, results and kernels are those of cr_partial_gradients.
+ *   - N * m * rows must not exceed cr_partial_gradients_static_capacity() (1,048,576 residuals);
+ *     larger problems return CR_ERR_OOM with an explanatory cr_last_cuda_error() text and launch nothing.
+ *   - The call never allocates or frees (no cudaMalloc/cudaFree, no staging buffers, no library
+ *     allocator).  The first call on each device looks up the array's device address; make that first
+ *     call outside of any stream capture.
+ *   - Every call on a device shares the one array and finds the previous call's residuals in it; each
+ *     call overwrites every entry it later reads, so nothing needs clearing.  Two calls whose kernels
+ *     can overlap on the same GPU (different streams, different plans, different threads) race on it:
+ *     order them on one stream or with events. */
+size_t cr_partial_gradients_static_capacity(void);
+cr_status_t cr_partial_gradients_static(cr_plan_t *plan, const float *X, const float *y, int32_t rows,
+                                        const float *w, float *G_slots, void *stream);
+
 /* ---- CR.Execute, local coded gradient g_{D(l,i)} (Section III-A) ------------------------------
  * E[v][:] = sum_j c_{v,j} * G_slots[v][j][:] for every node v.  G_slots [N][m][d], E [N][d]:
  * device pointers of the plan's dtype.  (Verification path; the fused kernel never writes E.) */

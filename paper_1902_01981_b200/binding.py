@@ -61,6 +61,9 @@ _SIGNATURES = {
     "cr_partial_gradients_workspace_bytes": (C.c_size_t, [C.c_void_p, C.c_int32]),
     "cr_partial_gradients": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
                                        C.c_void_p, C.c_size_t, C.c_void_p]),
+    "cr_partial_gradients_static_capacity": (C.c_size_t, []),
+    "cr_partial_gradients_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
+                                              C.c_void_p]),
     "cr_encode": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "cr_decode": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]),
     "cr_aggregate_workspace_bytes": (C.c_size_t, [C.c_void_p, C.c_int32, C.c_uint32]),
@@ -220,6 +223,18 @@ def cr_partial_gradients(plan: int, X, y, rows: int, w, G_slots, workspace, stre
                                       _dev_ptr(workspace),
                                       0 if workspace is None else workspace.numel() * workspace.element_size(),
                                       _stream_ptr(stream)), "cr_partial_gradients")
+
+
+def cr_partial_gradients_static_capacity() -> int:
+    return lib().cr_partial_gradients_static_capacity()
+
+
+def cr_partial_gradients_static(plan: int, X, y, rows: int, w, G_slots, stream=None) -> None:
+    """cr_partial_gradients for callers that cannot allocate: the residual scratch is a fixed array
+    inside the library (N * m * rows <= cr_partial_gradients_static_capacity()); calls that may
+    overlap on one GPU race on it."""
+    _check(lib().cr_partial_gradients_static(plan, _dev_ptr(X), _dev_ptr(y), rows, _dev_ptr(w), _dev_ptr(G_slots),
+                                             _stream_ptr(stream)), "cr_partial_gradients_static")
 
 
 def cr_encode(plan: int, G_slots, E, stream=None) -> None:

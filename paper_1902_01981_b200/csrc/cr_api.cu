@@ -6,6 +6,7 @@
 #include <algorithm>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -517,6 +518,53 @@ cr_status_t cr_aggregate_host(cr_plan_t *plan, const void *G_slots_host, const u
     if (st != CR_OK) return st;
     CR_CUDA(cudaMemcpyAsync(g_out_host, dev_out, out_bytes, cudaMemcpyDeviceToHost, s));
     CR_CUDA(cudaStreamSynchronize(s));
+    return CR_OK;
+}
+
+// ---- partial gradients without any allocation -------------------------------------------------
+//
+// Residual scratch of cr_partial_gradients_static: one fixed array per device that loads this
+// library, held until the process exits.  4 MiB = 1,048,576 residuals (slots x rows).
+#define CR_STATIC_RESIDUALS (1u << 20)
+static __device__ __align__(256) float cr_static_residuals[CR_STATIC_RESIDUALS];
+
+namespace {
+std::mutex g_static_mutex;
+float *g_static_ptr[64] = {nullptr};  // device address of the array, per device ordinal
+}  // namespace
+
+size_t cr_partial_gradients_static_capacity(void) { return (size_t)CR_STATIC_RESIDUALS; }
+
+cr_status_t cr_partial_gradients_static(cr_plan_t *plan, const float *X, const float *y, int32_t rows,
+                                        const float *w, float *G_slots, void *stream) {
+    cr_status_t st = check_device_plan(plan);  // makes the plan's device current
+    if (st != CR_OK) return st;
+    if (!X || !y || !w || !G_slots || rows < 1) return CR_ERR_INVALID_ARG;
+    if (plan->hp.dtype != CR_F32) return CR_ERR_DTYPE;
+    if (plan->device >= 64) return CR_ERR_INVALID_ARG;
+    const size_t need = (size_t)plan->hp.N * plan->hp.m * (size_t)rows;
+    if (need > (size_t)CR_STATIC_RESIDUALS) {
+        std::snprintf(g_last_error, sizeof(g_last_error),
+                      "cr_partial_gradients_static: %zu residuals (slots x rows) exceed the fixed scratch of %u",
+                      need, CR_STATIC_RESIDUALS);
+        return CR_ERR_OOM;
+    }
+    float *scratch = nullptr;
+    {
+        // In host code the array's name is only a handle; the kernels need its address on this
+        // device, looked up once per device while that device is current.
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!g_static_ptr[plan->device]) {
+            void *addr = nullptr;
+            CR_CUDA(cudaGetSymbolAddress(&addr, cr_static_residuals));
+            g_static_ptr[plan->device] = reinterpret_cast<float *>(addr);
+        }
+        scratch = g_static_ptr[plan->device];
+    }
+    cudaError_t e = cr::launch_partial_gradients(X, y, w, plan->d_part, plan->hp.N * plan->hp.m, rows, plan->hp.d,
+                                                 scratch, G_slots, reinterpret_cast<cudaStream_t>(stream),
+                                                 &plan->launches);
+    if (e != cudaSuccess) { note_cuda(e, "cr_partial_gradients_static"); return CR_ERR_CUDA; }
     return CR_OK;
 }
 
