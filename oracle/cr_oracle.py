@@ -430,12 +430,12 @@ def partial_gradient_linreg(X: np.ndarray, y: np.ndarray, w: np.ndarray) -> np.n
     """Gradient of l(w) = 1/2 ||X w - y||^2 summed over the rows of one
     partition: X^T (X w - y), in fp64 from whatever precision the inputs have.
     Pinned by a central finite difference of the loss."""
-    X = X.astype(np.float64)
-    return X.T @ (X @ w.astype(np.float64) - y.astype(np.float64))
+    X = np.asarray(X, dtype=np.float64)
+    return X.T @ (X @ np.asarray(w, dtype=np.float64) - np.asarray(y, dtype=np.float64))
 
 
 def loss_linreg(X: np.ndarray, y: np.ndarray, w: np.ndarray) -> float:
-    r = X.astype(np.float64) @ w.astype(np.float64) - y.astype(np.float64)
+    r = np.asarray(X, dtype=np.float64) @ np.asarray(w, dtype=np.float64) - np.asarray(y, dtype=np.float64)
     return 0.5 * float(r @ r)
 
 
