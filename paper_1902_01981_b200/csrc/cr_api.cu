@@ -241,7 +241,7 @@ cr_status_t cr_plan_tune(cr_plan_t *plan, int32_t consumer_warps, int32_t stages
     if (!plan || consumer_warps < 0 || stages < 0 || ctas_per_sm < 0 || rows_per_box < 0) return CR_ERR_INVALID_ARG;
     if (consumer_warps != 0 && consumer_warps != 2 && consumer_warps != 4 && consumer_warps != 8) return CR_ERR_INVALID_ARG;
     if (stages == 1 || stages > 16 || ctas_per_sm > 8) return CR_ERR_INVALID_ARG;
-    if (rows_per_box != 0 && (plan->hp.m % rows_per_box != 0 || rows_per_box > 64)) return CR_ERR_INVALID_ARG;
+    if (rows_per_box != 0 && (plan->hp.m % rows_per_box != 0 || rows_per_box > 16)) return CR_ERR_INVALID_ARG;
     plan->tune.ncw = consumer_warps; plan->tune.stages = stages; plan->tune.ctas_per_sm = ctas_per_sm;
     plan->tune.rows = rows_per_box;
     return CR_OK;

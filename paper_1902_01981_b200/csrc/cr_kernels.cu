@@ -51,6 +51,9 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
 // near the bound; it exists so that a broken one returns with a status instead of hanging the GPU.
 constexpr uint64_t kWaitLimitNs = 2000000000ull;
 
+// Most slot rows one TMA box may hold (the consumers keep that many coefficients in registers).
+constexpr int kMaxBoxRows = 16;
+
 // `abort_flag` points at a shared-memory word that the other side of the pipeline sets when it has
 // given up (flags[0]: a consumer did, flags[1]: the producer did, flags[2]: never set).
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
@@ -145,7 +148,7 @@ struct FusedArgs {
 };
 
 template <typename T, int LMAX, int NCW>
-__global__ void __launch_bounds__((NCW + 1) * 32)
+__global__ void __launch_bounds__((NCW + 1) * 32, 1)
 cr_fused_tma_kernel(const __grid_constant__ CUtensorMap tmap, const FusedArgs a) {
     constexpr int TILE = NCW * 128;
     constexpr int BOXW = TILE < 256 ? TILE : 256;
@@ -206,6 +209,8 @@ cr_fused_tma_kernel(const __grid_constant__ CUtensorMap tmap, const FusedArgs a)
         }
     } else {
         // ---------------- consumers ----------------
+        // The schedule entry and the R coefficients of a box are fetched one box ahead, before the
+        // wait on the current box, so that their latency hides behind the wait for the data.
         T acc[LMAX][4];
 #pragma unroll
         for (int l = 0; l < LMAX; ++l)
@@ -216,19 +221,38 @@ cr_fused_tma_kernel(const __grid_constant__ CUtensorMap tmap, const FusedArgs a)
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
+        Step st_next = load_step(&a.steps[0]);
+        T cj_next[kMaxBoxRows];
+        {
+            const T *cf = coeff + (size_t)st_next.node * a.m;
+#pragma unroll
+            for (int j = 0; j < kMaxBoxRows; ++j) cj_next[j] = j < R ? __ldg(cf + j) : T(0);
+        }
         for (long long tile = blockIdx.x; tile < a.ntiles && ok; tile += gridDim.x) {
             for (int k = 0; k < a.n_steps && ok; ++k) {
-                const Step st = load_step(&a.steps[k]);
                 T e[4] = {T(0), T(0), T(0), T(0)};
+                Step st = st_next;
                 for (int c = 0; c < a.cpn; ++c) {
-                    const T *cf = coeff + (size_t)st.node * a.m + c * R;
+                    T cj[kMaxBoxRows];
+#pragma unroll
+                    for (int j = 0; j < kMaxBoxRows; ++j) cj[j] = cj_next[j];
+                    st = st_next;
+                    {
+                        int kn = k, cn = c + 1;
+                        if (cn == a.cpn) { cn = 0; kn = k + 1 == a.n_steps ? 0 : k + 1; }
+                        st_next = load_step(&a.steps[kn]);
+                        const T *cf = coeff + (size_t)st_next.node * a.m + cn * R;
+#pragma unroll
+                        for (int j = 0; j < kMaxBoxRows; ++j) cj_next[j] = j < R ? __ldg(cf + j) : T(0);
+                    }
                     if (!mbar_wait(&full[stage], phase, &flags[1])) { ok = false; break; }
                     const T *src = ring + (size_t)stage * stage_elems + (size_t)box * R * BOXW + within;
-#pragma unroll 4
-                    for (int j = 0; j < R; ++j) {
-                        const V4 v = *reinterpret_cast<const V4 *>(src + (size_t)j * BOXW);
-                        const T cj = __ldg(cf + j);
-                        e[0] += cj * v.x; e[1] += cj * v.y; e[2] += cj * v.z; e[3] += cj * v.w;
+#pragma unroll
+                    for (int j = 0; j < kMaxBoxRows; ++j) {
+                        if (j < R) {
+                            const V4 v = *reinterpret_cast<const V4 *>(src + (size_t)j * BOXW);
+                            e[0] += cj[j] * v.x; e[1] += cj[j] * v.y; e[2] += cj[j] * v.z; e[3] += cj[j] * v.w;
+                        }
                     }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&empty[stage]);
@@ -260,7 +284,14 @@ cr_fused_tma_kernel(const __grid_constant__ CUtensorMap tmap, const FusedArgs a)
 // of consumed nodes -- warp w takes nodes w, w+NCW, .. -- into shared memory E[n_union][128], then
 // replays every pattern's post-order schedule from E (warp w takes patterns w, w+NCW, ..) and writes
 // one output tile per pattern.  The slots are read from HBM once for the whole batch; the producer
-// warp keeps prefetching the next tile's rows through the ring while patterns are replayed.
+// warp keeps prefetching the next tile's rows while patterns are replayed.
+//
+// Every consumer warp has a PRIVATE ring of `stages` buffers that only it drains, in order.  (With one
+// ring shared by warps that each take every NCW-th box, a warp can reach a buffer whose previous box --
+// another warp's -- has not landed yet, since TMA completions are unordered; a parity wait cannot tell
+// "one phase behind" from "done", the warp would read early and release the buffer twice.)
+// Box number q of warp w (counted over the whole kernel) lives in buffer w*stages + q % stages with
+// phase (q / stages) & 1; producer and consumer derive q from (tile, node, chunk) the same way.
 
 struct BatchArgs {
     const void *coeff;
@@ -277,23 +308,23 @@ struct BatchArgs {
 };
 
 template <typename T, int LMAX, int NCW>
-__global__ void __launch_bounds__((NCW + 1) * 32)
+__global__ void __launch_bounds__((NCW + 1) * 32, 1)
 cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchArgs a) {
     constexpr int TILE = 128;
     typedef typename Vec4<T>::type V4;
 
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    const int R = a.R, S = a.stages;
+    const int R = a.R, S = a.stages, NS = NCW * a.stages;
     const size_t stage_elems = (size_t)R * TILE;
     T *ring = reinterpret_cast<T *>(smem_raw);
-    T *E = ring + (size_t)S * stage_elems;
+    T *E = ring + (size_t)NS * stage_elems;
     uint64_t *full = reinterpret_cast<uint64_t *>(E + (size_t)a.n_union * TILE);
-    uint64_t *empty = full + S;
-    volatile int *flags = reinterpret_cast<volatile int *>(empty + S);
+    uint64_t *empty = full + NS;
+    volatile int *flags = reinterpret_cast<volatile int *>(empty + NS);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
-        for (int s = 0; s < S; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
         flags[0] = 0; flags[1] = 0; flags[2] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -302,54 +333,71 @@ cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchA
 
     const T *coeff = reinterpret_cast<const T *>(a.coeff);
     const uint32_t stage_bytes = (uint32_t)(stage_elems * sizeof(T));
-    const unsigned per_tile = (unsigned)a.n_union * (unsigned)a.cpn;  // ring iterations per tile
 
     if (warp == NCW) {
         if (lane == 0) {
-            int stage = 0;
-            uint32_t phase = 0;
-            long long issued = 0;
             bool ok = true;
+            unsigned tiles_done = 0;
+            int u_stop = 0, c_stop = 0;  // where issuing stopped if a wait gave up
             for (long long tile = blockIdx.x; tile < a.ntiles && ok; tile += gridDim.x) {
                 const int x0 = (int)(tile * TILE);
                 for (int u = 0; u < a.n_union && ok; ++u) {
+                    const int w = u % NCW;
+                    const unsigned nodes_w = (unsigned)(a.n_union - w + NCW - 1) / NCW;  // nodes of warp w per tile
+                    const unsigned q0 = (tiles_done * nodes_w + (unsigned)(u / NCW)) * (unsigned)a.cpn;
                     const int row0 = __ldg(&a.unodes[u]) * a.m;
                     for (int c = 0; c < a.cpn; ++c) {
-                        if (!mbar_wait(&empty[stage], phase ^ 1u, &flags[0])) { ok = false; break; }
+                        const unsigned q = q0 + (unsigned)c;
+                        const int stage = w * S + (int)(q % (unsigned)S);
+                        const uint32_t phase = (q / (unsigned)S) & 1u;
+                        if (!mbar_wait(&empty[stage], phase ^ 1u, &flags[0])) { ok = false; u_stop = u; c_stop = c; break; }
                         mbar_expect_tx(&full[stage], stage_bytes);
                         tma_load_2d(ring + (size_t)stage * stage_elems, &tmap, x0, row0 + c * R, &full[stage]);
-                        ++issued;
-                        if (++stage == S) { stage = 0; phase ^= 1u; }
                     }
                 }
+                if (ok) ++tiles_done;
             }
             if (!ok) {
+                // give up: flag it, then wait (bounded) for the last `stages` boxes issued to every
+                // ring, so that no copy lands in shared memory after the CTA has gone
                 flags[1] = 1;
                 atomicExch(a.status, 1);
-                for (long long i = issued > S ? issued - S : 0; i < issued; ++i)
-                    mbar_wait(&full[i % S], (uint32_t)((i / S) & 1), &flags[2]);
+                for (int w = 0; w < NCW; ++w) {
+                    const unsigned nodes_w = (unsigned)(a.n_union - w + NCW - 1) / NCW;
+                    const unsigned before = u_stop > w ? (unsigned)(u_stop - w + NCW - 1) / NCW : 0u;  // nodes of w below u_stop
+                    const unsigned issued = (tiles_done * nodes_w + before) * (unsigned)a.cpn + (u_stop % NCW == w ? (unsigned)c_stop : 0u);
+                    for (unsigned q = issued > (unsigned)S ? issued - (unsigned)S : 0u; q < issued; ++q)
+                        mbar_wait(&full[w * S + (int)(q % (unsigned)S)], (q / (unsigned)S) & 1u, &flags[2]);
+                }
             }
         }
     } else {
         bool ok = true;
-        unsigned tile_iter0 = 0;  // ring iteration index of this tile's first box
-        for (long long tile = blockIdx.x; tile < a.ntiles; tile += gridDim.x, tile_iter0 += per_tile) {
-            // phase 1: coded gradients of the union nodes -> E
+        const unsigned nodes_w = (unsigned)(a.n_union - warp + NCW - 1) / NCW;
+        unsigned tiles_done = 0;
+        for (long long tile = blockIdx.x; tile < a.ntiles; tile += gridDim.x, ++tiles_done) {
+            // phase 1: coded gradients of the union nodes -> E.  The coefficients of a box are
+            // fetched before the wait on its data.
             for (int u = warp; u < a.n_union && ok; u += NCW) {
                 const int node = __ldg(&a.unodes[u]);
+                const unsigned q0 = (tiles_done * nodes_w + (unsigned)(u / NCW)) * (unsigned)a.cpn;
                 T e[4] = {T(0), T(0), T(0), T(0)};
                 for (int c = 0; c < a.cpn; ++c) {
-                    const unsigned it = tile_iter0 + (unsigned)u * (unsigned)a.cpn + (unsigned)c;
-                    const int stage = (int)(it % (unsigned)S);
-                    const uint32_t phase = (it / (unsigned)S) & 1u;
+                    const unsigned q = q0 + (unsigned)c;
+                    const int stage = warp * S + (int)(q % (unsigned)S);
+                    const uint32_t phase = (q / (unsigned)S) & 1u;
                     const T *cf = coeff + (size_t)node * a.m + c * R;
+                    T cj[kMaxBoxRows];
+#pragma unroll
+                    for (int j = 0; j < kMaxBoxRows; ++j) cj[j] = j < R ? __ldg(cf + j) : T(0);
                     if (!mbar_wait(&full[stage], phase, &flags[1])) { ok = false; break; }
                     const T *src = ring + (size_t)stage * stage_elems + lane * 4;
-#pragma unroll 4
-                    for (int j = 0; j < R; ++j) {
-                        const V4 v = *reinterpret_cast<const V4 *>(src + (size_t)j * TILE);
-                        const T cj = __ldg(cf + j);
-                        e[0] += cj * v.x; e[1] += cj * v.y; e[2] += cj * v.z; e[3] += cj * v.w;
+#pragma unroll
+                    for (int j = 0; j < kMaxBoxRows; ++j) {
+                        if (j < R) {
+                            const V4 v = *reinterpret_cast<const V4 *>(src + (size_t)j * TILE);
+                            e[0] += cj[j] * v.x; e[1] += cj[j] * v.y; e[2] += cj[j] * v.z; e[3] += cj[j] * v.w;
+                        }
                     }
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&empty[stage]);
@@ -362,7 +410,9 @@ cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchA
             if (!ok) { flags[0] = 1; atomicExch(a.status, 1); }
             consumer_barrier(NCW * 32);
             if (flags[0]) break;
-            // phase 2: replay every pattern's schedule from E
+            // phase 2: replay every pattern's schedule from E.  Lane i fetches entry i of the
+            // pattern's schedule (one coalesced load per 32 entries); entries are then broadcast
+            // with shuffles.
             const long long gcol = tile * TILE + lane * 4;
             for (int b = warp; b < a.batch; b += NCW) {
                 T acc[LMAX][4];
@@ -371,11 +421,18 @@ cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchA
 #pragma unroll
                     for (int q = 0; q < 4; ++q) acc[l][q] = T(0);
                 const int k0 = __ldg(&a.pat_off[b]), k1 = __ldg(&a.pat_off[b + 1]);
-                for (int k = k0; k < k1; ++k) {
-                    const Step st = load_step(&a.steps[k]);
-                    const V4 v = *reinterpret_cast<const V4 *>(E + (size_t)st.index * TILE + lane * 4);
-                    const T e[4] = {v.x, v.y, v.z, v.w};
-                    fold<T, LMAX, 4>(acc, e, st.layer, weight_of<T>(st.wbits));
+                for (int kb = k0; kb < k1; kb += 32) {
+                    int4 mine = make_int4(0, 0, 0, 0);
+                    if (kb + lane < k1) mine = __ldg(reinterpret_cast<const int4 *>(&a.steps[kb + lane]));
+                    const int cnt = k1 - kb < 32 ? k1 - kb : 32;
+                    for (int i = 0; i < cnt; ++i) {
+                        const int layer = __shfl_sync(0xffffffffu, mine.y, i);
+                        const uint32_t wb = (uint32_t)__shfl_sync(0xffffffffu, mine.z, i);
+                        const int idx = __shfl_sync(0xffffffffu, mine.w, i);
+                        const V4 v = *reinterpret_cast<const V4 *>(E + (size_t)idx * TILE + lane * 4);
+                        const T e[4] = {v.x, v.y, v.z, v.w};
+                        fold<T, LMAX, 4>(acc, e, layer, weight_of<T>(wb));
+                    }
                 }
                 if (gcol < a.d) {
                     V4 o;
@@ -700,7 +757,7 @@ cudaError_t launch_fused_tma(const AggArgs &a, const DeviceInfo &dev, const Tuni
     const int boxw = tile < 256 ? tile : 256;
     // rows per box: a divisor of m, at most 16, stage no larger than ~36 KB
     int cap = std::min(16, std::max(1, (36 * 1024) / (tile * 4)));
-    int R = tune.rows && a.m % tune.rows == 0 && tune.rows <= 256 ? tune.rows : rows_per_box(a.m, cap);
+    int R = tune.rows && a.m % tune.rows == 0 && tune.rows <= kMaxBoxRows ? tune.rows : rows_per_box(a.m, cap);
     const size_t stage_bytes = (size_t)R * tile * 4;
     int ctas = tune.ctas_per_sm ? tune.ctas_per_sm : 2;
     int stages = tune.stages ? tune.stages : 0;
@@ -753,27 +810,34 @@ cudaError_t launch_fused_batch_tma(const AggArgs &a, const DeviceInfo &dev, cons
     *done = false;
     if (!encode || !tma_eligible(a)) return cudaSuccess;
     const int tile = 128;
-    int R = tune.rows && a.m % tune.rows == 0 && tune.rows <= 256 ? tune.rows : rows_per_box(a.m, 16);
-    const size_t stage_bytes = (size_t)R * tile * 4;
+    const int ncw = (tune.ncw == 2 || tune.ncw == 4 || tune.ncw == 8) ? tune.ncw : 4;
     const size_t e_bytes = (size_t)a.n_union * tile * 4;
     const size_t usable = (size_t)dev.smem_per_sm - 2048;
-    int ctas = tune.ctas_per_sm ? tune.ctas_per_sm : 2;
-    int stages = 0;
-    for (; ctas >= 1; --ctas) {
+    // Shared memory = E + ncw private rings of `stages` boxes of R rows.  Prefer two CTAs per SM (one
+    // replays patterns while the other streams), at least 2 boxes per ring, boxes as tall as fit.
+    int ctas = tune.ctas_per_sm ? tune.ctas_per_sm : 2, stages = 0, R = 0;
+    for (; ctas >= 1 && !stages; --ctas) {
         const size_t budget = std::min(usable / ctas - 1024, (size_t)dev.smem_optin);
-        if (budget <= e_bytes + 64) continue;
-        stages = (int)((budget - e_bytes - 64) / stage_bytes);
-        if (stages >= 3 || (ctas == 1 && stages >= 2)) break;
+        if (budget <= e_bytes + 256) continue;
+        const size_t ring_budget = budget - e_bytes - 256;
+        const int want_stages = tune.stages ? tune.stages : 3;
+        for (int depth = want_stages; depth >= 2 && !stages; --depth) {
+            // tallest box (a divisor of m, at most kMaxBoxRows) such that ncw * depth boxes fit
+            const int cap = (int)std::min<size_t>(kMaxBoxRows, ring_budget / ((size_t)ncw * depth * tile * 4));
+            if (cap < 1) continue;
+            const int r = tune.rows && a.m % tune.rows == 0 && tune.rows <= cap ? tune.rows : rows_per_box(a.m, cap);
+            if (r * 4 < std::min(a.m, 8) && depth > 2) continue;  // prefer taller boxes over a third buffer
+            R = r; stages = depth;
+        }
+        if (stages) break;
     }
-    if (ctas < 1 || stages < 2) return cudaSuccess;  // union too large for shared memory
-    stages = std::min(stages, tune.stages ? tune.stages : 8);
-    if (stages < 2) stages = 2;
-    const int ncw = (tune.ncw == 2 || tune.ncw == 4 || tune.ncw == 8) ? tune.ncw : 4;
-    const size_t smem = (size_t)stages * stage_bytes + e_bytes + (size_t)stages * 16 + 32;
+    if (!stages) return cudaSuccess;  // union too large for shared memory: caller falls back
+    const size_t stage_bytes = (size_t)R * tile * 4;
+    const size_t smem = (size_t)ncw * stages * stage_bytes + e_bytes + (size_t)ncw * stages * 16 + 32;
     if (smem > (size_t)dev.smem_optin) return cudaSuccess;
     const long long ntiles = (a.d + tile - 1) / tile;
     const int grid = (int)std::min<long long>(ntiles, (long long)dev.sm_count * ctas);
-    // ring iteration counters are 32-bit
+    // box counters are 32-bit
     if ((ntiles / grid + 1) * (long long)a.n_union * (a.m / R) >= (1ll << 31)) return cudaSuccess;
 
     CUtensorMap map;
