@@ -36,8 +36,9 @@ UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the timed kernel, from the ncu capture
-# summarised under profiles/ (None until a capture of the current kernel exists).
-NCU_TRAFFIC_BYTES = {}
+# summarised under profiles/ (absent = no capture of the current kernel on that workload).
+# cfg4: 917.4 MB measured at d = 2^21, scaled by 8 to d = 2^24 (traffic is proportional to d).
+NCU_TRAFFIC_BYTES = {("cfg4", "f32", 1 << 24): 8 * 917.37e6}
 
 
 def peak_hbm():
@@ -354,7 +355,7 @@ def run_ours(args, cfg):
         avg_bytes = units / args.steps
         achieved = avg_bytes / avg_launch / 1e9
         kern = "cr_fused_batch_tma_kernel" if batch > 1 else "cr_fused_tma_kernel"
-        traffic = NCU_TRAFFIC_BYTES.get((args.workload, args.dtype))
+        traffic = NCU_TRAFFIC_BYTES.get((args.workload, args.dtype, d))
         roofline = {"bound": "hbm", "kernel": kern, "achieved": achieved, "peak": peak, "unit": "GB/s",
                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / 8000.0,
                     "traffic": traffic, "algorithmic_bytes_per_launch": avg_bytes,

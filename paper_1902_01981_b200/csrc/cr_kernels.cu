@@ -755,21 +755,22 @@ cudaError_t launch_fused_tma(const AggArgs &a, const DeviceInfo &dev, const Tuni
     if (ncw != 2 && ncw != 4 && ncw != 8) ncw = 4;
     const int tile = ncw * 128;
     const int boxw = tile < 256 ? tile : 256;
-    // rows per box: a divisor of m, at most 16, stage no larger than ~36 KB
-    int cap = std::min(16, std::max(1, (36 * 1024) / (tile * 4)));
-    int R = tune.rows && a.m % tune.rows == 0 && tune.rows <= kMaxBoxRows ? tune.rows : rows_per_box(a.m, cap);
+    // Launch shape.  Measured on B200 (d = 2^24, m = 9): throughput peaks with about 100 KB of loads
+    // in flight per SM and falls off on both sides (too little: latency-bound; too much: the DRAM
+    // pages of too many slot rows are open at once), and several small CTAs per SM beat one large
+    // one.  So: boxes of at most ~18 KB (R = a divisor of m), three CTAs per SM, and as many stages
+    // as bring the total to ~36 KB per CTA, at least two.
+    const int cap = std::min(kMaxBoxRows, std::max(1, (18 * 1024) / (tile * 4)));
+    const int R = tune.rows && a.m % tune.rows == 0 && tune.rows <= kMaxBoxRows ? tune.rows : rows_per_box(a.m, cap);
     const size_t stage_bytes = (size_t)R * tile * 4;
-    int ctas = tune.ctas_per_sm ? tune.ctas_per_sm : 2;
-    int stages = tune.stages ? tune.stages : 0;
+    int ctas = tune.ctas_per_sm ? tune.ctas_per_sm : 3;
+    int stages = tune.stages ? tune.stages
+                             : std::max(2, std::min(8, (int)((36 * 1024 + stage_bytes / 2) / stage_bytes)));
     const size_t usable = (size_t)dev.smem_per_sm - 2048;  // leave room for the per-CTA reserve
-    if (!stages) {
-        stages = (int)((usable / ctas - 1024) / stage_bytes);
-        stages = std::min(stages, 8);
-    }
-    if (stages < 2) { ctas = 1; stages = (int)(((size_t)dev.smem_optin - 1024) / stage_bytes); stages = std::min(stages, 8); }
-    if (stages < 2) return cudaSuccess;  // does not fit: caller falls back to plain loads
+    while (ctas > 1 && ((size_t)stages * stage_bytes + 1024 + 256) * ctas > usable) --ctas;
+    while (stages > 2 && (size_t)stages * stage_bytes + 256 > (size_t)dev.smem_optin) --stages;
     const size_t smem = (size_t)stages * stage_bytes + (size_t)stages * 16 + 32;
-    if (smem > (size_t)dev.smem_optin) return cudaSuccess;
+    if (smem > (size_t)dev.smem_optin) return cudaSuccess;  // does not fit: caller falls back to plain loads
 
     CUtensorMap map;
     if (make_map(encode, &map, a, boxw, R) != CUDA_SUCCESS) return cudaSuccess;
