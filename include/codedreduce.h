@@ -211,9 +211,11 @@ cr_status_t cr_aggregate_bytes(const cr_plan_t *plan, const uint32_t *masks_host
                                int64_t *bytes, int32_t *used_nodes);
 
 /* Launch shape of the TMA kernels of cr_aggregate; 0 keeps the built-in choice for that field.
- * consumer_warps in {2,4,8} (single-pattern kernel: column tile = 128 * consumer_warps), stages = depth
+ * Single-pattern kernel: consumer_warps in {2,4,8} (column tile = 128 * consumer_warps), stages = depth
  * of the shared-memory ring (2..16), ctas_per_sm = persistent CTAs per SM (1..8), rows_per_box = slot
- * rows per TMA box (must divide m, at most 16).  Shapes that do not fit shared memory fall back to plain loads. */
+ * rows per TMA box (must divide m, at most 16).  Batch kernel (one CTA per SM): consumer_warps = replay
+ * warps (4 or 8), stages = boxes per loader warp, ctas_per_sm = loader warps (4 or 6), rows_per_box as
+ * above.  Shapes that do not fit shared memory fall back to smaller ones or to plain loads. */
 cr_status_t cr_plan_tune(cr_plan_t *plan, int32_t consumer_warps, int32_t stages, int32_t ctas_per_sm,
                          int32_t rows_per_box);
 

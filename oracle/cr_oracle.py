@@ -213,6 +213,8 @@ def decode_row(B: np.ndarray, s: int, straggler_mask: int) -> np.ndarray:
     n = B.shape[0]
     U = survivors(n, s, straggler_mask)
     a_U, *_ = np.linalg.lstsq(B[U, :].T, np.ones(n), rcond=None)
+    # a survivor that is not needed comes out of the solver as rounding noise: that is a zero
+    a_U[np.abs(a_U) <= 1e-13 * np.max(np.abs(a_U))] = 0.0
     a = np.zeros(n)
     a[U] = a_U
     return a

@@ -106,6 +106,7 @@ struct Expanded {
     std::vector<cr::Step> steps;       // all patterns, concatenated
     std::vector<int32_t> pat_off;      // [batch+1]
     std::vector<int32_t> unodes;       // union of used nodes, ascending
+    std::vector<uint32_t> wtab;        // distinct decode-weight bit patterns of the batch (empty: none / too many)
     std::vector<std::vector<cr::UsedNode>> per_pattern;
 };
 
@@ -121,10 +122,30 @@ cr_status_t expand_all(const cr::HostPlan &hp, const uint32_t *masks, int batch,
     }
     for (int v = 0; v < hp.N; ++v)
         if (seen[v]) { pos[v] = (int32_t)ex.unodes.size(); ex.unodes.push_back(v); }
+    // Step.index = position of the node in the union list (bits 0..11 when it fits) and, above it, the
+    // index of the step's weight in the table of distinct weights: the batch kernel can then keep a
+    // 4-byte entry per step and pattern in shared memory.
+    bool table_ok = batch > 1 && ex.unodes.size() <= 4096;
     for (int b = 0; b < batch; ++b) {
-        for (const cr::UsedNode &u : ex.per_pattern[b])
-            ex.steps.push_back(cr::Step{u.node, u.layer, weight_bits(hp, u.weight), pos[u.node]});
+        for (const cr::UsedNode &u : ex.per_pattern[b]) {
+            const uint32_t wb = weight_bits(hp, u.weight);
+            int32_t index = pos[u.node];
+            if (table_ok) {
+                size_t wi = 0;
+                while (wi < ex.wtab.size() && ex.wtab[wi] != wb) ++wi;
+                if (wi == ex.wtab.size()) {
+                    if (ex.wtab.size() >= 1024) table_ok = false;
+                    else ex.wtab.push_back(wb);
+                }
+                if (table_ok) index |= (int32_t)(wi << 12);
+            }
+            ex.steps.push_back(cr::Step{u.node, u.layer | (u.first ? 0x100 : 0), wb, index});
+        }
         ex.pat_off.push_back((int32_t)ex.steps.size());
+    }
+    if (!table_ok) {
+        ex.wtab.clear();
+        for (cr::Step &st : ex.steps) st.index = pos[st.node];   // plain positions
     }
     return CR_OK;
 }
@@ -470,13 +491,15 @@ cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *m
     const size_t steps_bytes = align16(ex.steps.size() * sizeof(cr::Step));
     const size_t off_bytes = align16(ex.pat_off.size() * 4);
     const size_t nodes_bytes = align16(ex.unodes.size() * 4);
-    const size_t total = steps_bytes + off_bytes + nodes_bytes;
+    const size_t wtab_bytes = align16(ex.wtab.size() * 4);
+    const size_t total = steps_bytes + off_bytes + nodes_bytes + wtab_bytes;
     StageSlot *slot = nullptr;
     st = stage_acquire(plan, total, &slot);
     if (st != CR_OK) return st;
     std::memcpy(slot->host, ex.steps.data(), ex.steps.size() * sizeof(cr::Step));
     std::memcpy(slot->host + steps_bytes, ex.pat_off.data(), ex.pat_off.size() * 4);
     std::memcpy(slot->host + steps_bytes + off_bytes, ex.unodes.data(), ex.unodes.size() * 4);
+    std::memcpy(slot->host + steps_bytes + off_bytes + nodes_bytes, ex.wtab.data(), ex.wtab.size() * 4);
     st = stage_commit(slot, total, s);
     if (st != CR_OK) return st;
 
@@ -485,9 +508,18 @@ cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *m
     a.steps = reinterpret_cast<const cr::Step *>(slot->dev);
     a.pat_off = reinterpret_cast<const int32_t *>(slot->dev + steps_bytes);
     a.unodes = reinterpret_cast<const int32_t *>(slot->dev + steps_bytes + off_bytes);
+    a.wtab = reinterpret_cast<const uint32_t *>(slot->dev + steps_bytes + off_bytes + nodes_bytes);
+    a.n_wtab = (int)ex.wtab.size();
     a.n_union = (int)ex.unodes.size(); a.batch = batch; a.total_steps = (int)ex.steps.size();
     a.m = hp.m; a.L = hp.L; a.d = hp.d; a.rows_total = (int64_t)hp.N * hp.m; a.out = g_out;
     a.shift = hp.dtype == CR_I32 ? hp.int_shift : 0; a.status = plan->d_status; a.is_int = hp.dtype == CR_I32;
+    a.same_shape = 1;
+    for (int b = 1; b < batch && a.same_shape; ++b) {
+        const auto &p0 = ex.per_pattern[0], &pb = ex.per_pattern[b];
+        if (pb.size() != p0.size()) { a.same_shape = 0; break; }
+        for (size_t k = 0; k < p0.size(); ++k)
+            if (pb[k].layer != p0[k].layer) { a.same_shape = 0; break; }
+    }
 
     cudaError_t e = cudaSuccess;
     if (variant == CR_AGG_UNCODED_SUM) {

@@ -69,6 +69,12 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
     return false;
 }
 
+// The same wait for a whole warp (all 32 lanes call it): the answer is made uniform, so that the lanes
+// take the give-up path together or not at all.
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag) ? 1 : 0) != 0;
+}
+
 // 2-D tiled TMA load global -> shared, completion counted in bytes on an mbarrier.  x (innermost
 // coordinate) times the element size must be a multiple of 16 bytes.
 __device__ __forceinline__ void tma_load_2d(void *smem_dst, const CUtensorMap *map, int x, int y, uint64_t *bar) {
@@ -97,10 +103,11 @@ template <> __device__ __forceinline__ int weight_of<int>(uint32_t bits) { retur
 template <typename T> __device__ __forceinline__ T finish(T v, int shift) { return v; }
 template <> __device__ __forceinline__ int finish<int>(int v, int shift) { return v >> shift; }
 
+// Reads one schedule entry; `layer` is returned without the first-child flag.
 __device__ __forceinline__ Step load_step(const Step *p) {
     const int4 raw = __ldg(reinterpret_cast<const int4 *>(p));
     Step s;
-    s.node = raw.x; s.layer = raw.y; s.wbits = (uint32_t)raw.z; s.index = raw.w;
+    s.node = raw.x; s.layer = raw.y & 0xff; s.wbits = (uint32_t)raw.z; s.index = raw.w;
     return s;
 }
 
@@ -119,6 +126,42 @@ __device__ __forceinline__ void fold(T (&acc)[LMAX][V], const T (&e)[V], int lay
                 T msg = e[q];
                 if (l < LMAX) { msg += acc[l < LMAX ? l : 0][q]; acc[l < LMAX ? l : 0][q] = T(0); }
                 acc[l - 1][q] += w * msg;
+            }
+        }
+    }
+}
+
+// The same recursion for NP patterns whose schedules visit the same layers in the same order (they
+// differ in which children are used and with what weights): one uniform branch on the layer, NP
+// independent dependency chains inside it.  This form never clears an accumulator: the first consumed
+// child of a parent ASSIGNS acc[layer-1] = w * message, later children add to it (`lf` carries the
+// layer in bits 0..7 and the first-child flag in bit 8).  acc must start at zero so that leaves, whose
+// own acc is never written, add nothing.
+template <typename T, int LMAX, int NP>
+__device__ __forceinline__ void fold_many(T (&acc)[NP][LMAX][4], const T (&e)[NP][4], int lf, const T (&w)[NP]) {
+    const int layer = lf & 0xff;
+    const bool first = (lf & 0x100) != 0;
+#pragma unroll
+    for (int l = 1; l <= LMAX; ++l) {
+        if (layer == l) {
+            if (first) {
+#pragma unroll
+                for (int p = 0; p < NP; ++p)
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        T msg = e[p][q];
+                        if (l < LMAX) msg += acc[p][l < LMAX ? l : 0][q];
+                        acc[p][l - 1][q] = w[p] * msg;
+                    }
+            } else {
+#pragma unroll
+                for (int p = 0; p < NP; ++p)
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        T msg = e[p][q];
+                        if (l < LMAX) msg += acc[p][l < LMAX ? l : 0][q];
+                        acc[p][l - 1][q] += w[p] * msg;
+                    }
             }
         }
     }
@@ -245,7 +288,7 @@ cr_fused_tma_kernel(const __grid_constant__ CUtensorMap tmap, const FusedArgs a)
 #pragma unroll
                         for (int j = 0; j < kMaxBoxRows; ++j) cj_next[j] = j < R ? __ldg(cf + j) : T(0);
                     }
-                    if (!mbar_wait(&full[stage], phase, &flags[1])) { ok = false; break; }
+                    if (!mbar_wait_warp(&full[stage], phase, &flags[1])) { ok = false; break; }
                     const T *src = ring + (size_t)stage * stage_elems + (size_t)box * R * BOXW + within;
 #pragma unroll
                     for (int j = 0; j < kMaxBoxRows; ++j) {
@@ -279,27 +322,40 @@ cr_fused_tma_kernel(const __grid_constant__ CUtensorMap tmap, const FusedArgs a)
 // K4b: fused aggregation, a batch of straggler patterns over the same slots
 // ------------------------------------------------------------------------------------------------
 //
-// The coded gradient e_v of a node does not depend on the straggler pattern, so a CTA (tile of 128
-// columns, each consumer warp a full tile row of float4s) first forms e_v for every node of the union
-// of consumed nodes -- warp w takes nodes w, w+NCW, .. -- into shared memory E[n_union][128], then
-// replays every pattern's post-order schedule from E (warp w takes patterns w, w+NCW, ..) and writes
-// one output tile per pattern.  The slots are read from HBM once for the whole batch; the producer
-// warp keeps prefetching the next tile's rows while patterns are replayed.
+// The coded gradient e_v of a node does not depend on the straggler pattern, so the slots are read
+// from HBM once for the whole batch.  One persistent CTA per SM works on tiles of 128 columns with
+// two kinds of warps:
+//   * NLW loader warps each own a PRIVATE ring of `stages` TMA boxes (R slot rows x 128 columns) that
+//     only they fill and drain, in order: after consuming box q a loader's lane 0 issues box
+//     q + stages into the buffer it has just read (a single serial producer thread for all rings could
+//     not keep up: each of its waits costs several hundred nanoseconds).  Loader w forms e_v (a full
+//     tile row of float4s per warp) for union nodes w, w+NLW, .. and stores it in the tile's E buffer
+//     in shared memory, E[buf][n_union][128];
+//   * NRW replay warps replay every pattern's post-order schedule from E (warp r takes pattern groups
+//     r, r+NRW, ..) and write one output tile per pattern.
+// E is double buffered (when it fits), so the loaders stream tile t+1 while tile t is replayed and HBM
+// never idles; loaders and replayers hand the buffers over with two mbarriers per buffer.
 //
-// Every consumer warp has a PRIVATE ring of `stages` buffers that only it drains, in order.  (With one
-// ring shared by warps that each take every NCW-th box, a warp can reach a buffer whose previous box --
-// another warp's -- has not landed yet, since TMA completions are unordered; a parity wait cannot tell
-// "one phase behind" from "done", the warp would read early and release the buffer twice.)
-// Box number q of warp w (counted over the whole kernel) lives in buffer w*stages + q % stages with
-// phase (q / stages) & 1; producer and consumer derive q from (tile, node, chunk) the same way.
+// Why private rings: with one ring shared by warps that each take every NLW-th box, a warp can reach a
+// buffer whose previous box -- another warp's -- has not landed yet, since TMA completions are
+// unordered; a parity wait cannot tell "one phase behind" from "done", the warp would read early and
+// release the buffer twice.  Box number q of a loader (counted over the whole kernel) lives in its
+// buffer q % stages with phase (q / stages) & 1.  Every warp passes every phase of every barrier it
+// waits on, in order, so no wait can alias.
 
 struct BatchArgs {
     const void *coeff;
     const Step *steps;
     const int32_t *pat_off;
     const int32_t *unodes;
+    const uint32_t *wtab;  // distinct weight bit patterns of the batch
+    int n_wtab;
     int n_union, batch;
     int m, R, cpn, stages;
+    int same_shape;  // every pattern's schedule has the same length and layer sequence
+    int sched_smem;  // bytes of shared memory set aside for the staged schedules (0: replay reads them from global)
+    int nst;         // same_shape: entries per schedule
+    int nbuf;        // E buffers: 2, or 1 when two do not fit
     long long d;
     long long ntiles;
     void *out;
@@ -307,91 +363,96 @@ struct BatchArgs {
     int *status;
 };
 
-template <typename T, int LMAX, int NCW>
-__global__ void __launch_bounds__((NCW + 1) * 32, 1)
+template <typename T, int LMAX, int NLW, int NRW>
+__global__ void __launch_bounds__((NLW + NRW) * 32, 1)
 cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchArgs a) {
     constexpr int TILE = 128;
+    constexpr int NP = LMAX <= 4 ? 4 : 2;  // patterns replayed together by one warp
     typedef typename Vec4<T>::type V4;
 
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    const int R = a.R, S = a.stages, NS = NCW * a.stages;
+    const int R = a.R, S = a.stages, NS = NLW * a.stages;
     const size_t stage_elems = (size_t)R * TILE;
+    const size_t e_elems = (size_t)a.n_union * TILE;
     T *ring = reinterpret_cast<T *>(smem_raw);
-    T *E = ring + (size_t)NS * stage_elems;
-    uint64_t *full = reinterpret_cast<uint64_t *>(E + (size_t)a.n_union * TILE);
-    uint64_t *empty = full + NS;
-    volatile int *flags = reinterpret_cast<volatile int *>(empty + NS);
+    T *E = ring + (size_t)NS * stage_elems;  // [nbuf][n_union][TILE]
+    // staged schedules (same-shape batches with a weight table): lf[nst] = layer | first-child flag of
+    // every step, ent[nst][batch_pad] = position of the node in E (bits 0..11) | index of the decode
+    // weight in the table (bits 12..) per step and pattern, wtab_s[n_wtab] = the table
+    int *lf = reinterpret_cast<int *>(E + (size_t)a.nbuf * e_elems);
+    const int batch_pad = (a.batch + NP - 1) / NP * NP;
+    uint32_t *ent = reinterpret_cast<uint32_t *>(reinterpret_cast<unsigned char *>(lf) + (((size_t)a.nst * 4 + 15) & ~(size_t)15));
+    uint32_t *wtab_s = ent + (((size_t)a.nst * batch_pad + 3) & ~(size_t)3);
+    const int pos_mask = a.n_wtab ? 0xfff : 0x7fffffff;
+    uint64_t *full = reinterpret_cast<uint64_t *>(reinterpret_cast<unsigned char *>(lf) + a.sched_smem);
+    uint64_t *e_full = full + NS;    // [2] E buffer written by all loaders
+    uint64_t *e_free = e_full + 2;   // [2] E buffer released by all replayers
+    volatile int *flags = reinterpret_cast<volatile int *>(e_free + 2);  // [0] someone gave up, [1] never set
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
-        for (int s = 0; s < NS; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        flags[0] = 0; flags[1] = 0; flags[2] = 0;
+        for (int s = 0; s < NS; ++s) mbar_init(&full[s], 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(&e_full[b], NLW); mbar_init(&e_free[b], NRW); }
+        flags[0] = 0; flags[1] = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (a.sched_smem) {
+        for (int k = tid; k < a.nst; k += blockDim.x) lf[k] = __ldg(&a.steps[k].layer);
+        for (int idx = tid; idx < a.nst * batch_pad; idx += blockDim.x) {
+            const int k = idx / batch_pad, b = min(idx - k * batch_pad, a.batch - 1);  // padding repeats the last pattern
+            ent[idx] = (uint32_t)__ldg(&a.steps[__ldg(&a.pat_off[b]) + k].index);
+        }
+        for (int i = tid; i < a.n_wtab; i += blockDim.x) wtab_s[i] = __ldg(&a.wtab[i]);
     }
     __syncthreads();
 
     const T *coeff = reinterpret_cast<const T *>(a.coeff);
     const uint32_t stage_bytes = (uint32_t)(stage_elems * sizeof(T));
 
-    if (warp == NCW) {
-        if (lane == 0) {
-            bool ok = true;
-            unsigned tiles_done = 0;
-            int u_stop = 0, c_stop = 0;  // where issuing stopped if a wait gave up
-            for (long long tile = blockIdx.x; tile < a.ntiles && ok; tile += gridDim.x) {
-                const int x0 = (int)(tile * TILE);
-                for (int u = 0; u < a.n_union && ok; ++u) {
-                    const int w = u % NCW;
-                    const unsigned nodes_w = (unsigned)(a.n_union - w + NCW - 1) / NCW;  // nodes of warp w per tile
-                    const unsigned q0 = (tiles_done * nodes_w + (unsigned)(u / NCW)) * (unsigned)a.cpn;
-                    const int row0 = __ldg(&a.unodes[u]) * a.m;
-                    for (int c = 0; c < a.cpn; ++c) {
-                        const unsigned q = q0 + (unsigned)c;
-                        const int stage = w * S + (int)(q % (unsigned)S);
-                        const uint32_t phase = (q / (unsigned)S) & 1u;
-                        if (!mbar_wait(&empty[stage], phase ^ 1u, &flags[0])) { ok = false; u_stop = u; c_stop = c; break; }
-                        mbar_expect_tx(&full[stage], stage_bytes);
-                        tma_load_2d(ring + (size_t)stage * stage_elems, &tmap, x0, row0 + c * R, &full[stage]);
-                    }
-                }
-                if (ok) ++tiles_done;
-            }
-            if (!ok) {
-                // give up: flag it, then wait (bounded) for the last `stages` boxes issued to every
-                // ring, so that no copy lands in shared memory after the CTA has gone
-                flags[1] = 1;
-                atomicExch(a.status, 1);
-                for (int w = 0; w < NCW; ++w) {
-                    const unsigned nodes_w = (unsigned)(a.n_union - w + NCW - 1) / NCW;
-                    const unsigned before = u_stop > w ? (unsigned)(u_stop - w + NCW - 1) / NCW : 0u;  // nodes of w below u_stop
-                    const unsigned issued = (tiles_done * nodes_w + before) * (unsigned)a.cpn + (u_stop % NCW == w ? (unsigned)c_stop : 0u);
-                    for (unsigned q = issued > (unsigned)S ? issued - (unsigned)S : 0u; q < issued; ++q)
-                        mbar_wait(&full[w * S + (int)(q % (unsigned)S)], (q / (unsigned)S) & 1u, &flags[2]);
-                }
-            }
-        }
-    } else {
+    if (warp < NLW) {
+        // ---------------- loaders: stream their boxes, coded gradients of the union nodes -> E[buf] ----------------
         bool ok = true;
-        const unsigned nodes_w = (unsigned)(a.n_union - warp + NCW - 1) / NCW;
-        unsigned tiles_done = 0;
-        for (long long tile = blockIdx.x; tile < a.ntiles; tile += gridDim.x, ++tiles_done) {
-            // phase 1: coded gradients of the union nodes -> E.  The coefficients of a box are
-            // fetched before the wait on its data.
-            for (int u = warp; u < a.n_union && ok; u += NCW) {
+        const unsigned nodes_w = (unsigned)(a.n_union - warp + NLW - 1) / NLW;   // union nodes of this loader per tile
+        const unsigned my_tiles = blockIdx.x < a.ntiles ? (unsigned)((a.ntiles - 1 - blockIdx.x) / gridDim.x + 1) : 0u;
+        const unsigned total_boxes = my_tiles * nodes_w * (unsigned)a.cpn;
+        T *my_ring = ring + (size_t)warp * S * stage_elems;
+        uint64_t *my_full = full + warp * S;
+        // cursor of the next box to issue: (tile number of this CTA, node number of this loader, chunk)
+        unsigned issued = 0, it_t = 0, it_n = 0, it_c = 0;
+        auto issue_next = [&]() {   // lane 0 only
+            const int slot = (int)(issued % (unsigned)S);
+            const long long tile = (long long)blockIdx.x + (long long)it_t * gridDim.x;
+            const int u = warp + (int)it_n * NLW;
+            mbar_expect_tx(&my_full[slot], stage_bytes);
+            tma_load_2d(my_ring + (size_t)slot * stage_elems, &tmap, (int)(tile * TILE),
+                        __ldg(&a.unodes[u]) * a.m + (int)it_c * R, &my_full[slot]);
+            ++issued;
+            if (++it_c == (unsigned)a.cpn) { it_c = 0; if (++it_n == nodes_w) { it_n = 0; ++it_t; } }
+        };
+        if (lane == 0)
+            while (issued < total_boxes && issued < (unsigned)S) issue_next();
+        unsigned q = 0;  // next box to consume
+        unsigned t = 0;  // tiles handled by this CTA so far
+        for (long long tile = blockIdx.x; tile < a.ntiles && ok; tile += gridDim.x, ++t) {
+            const int buf = (int)(t % (unsigned)a.nbuf);
+            const unsigned use = t / (unsigned)a.nbuf;  // how many times this buffer has been filled before
+            // the buffer must have been released by the replay of its previous tile
+            if (!mbar_wait_warp(&e_free[buf], (use & 1u) ^ 1u, &flags[0])) { ok = false; break; }
+            T *Eb = E + (size_t)buf * e_elems;
+            for (int u = warp; u < a.n_union && ok; u += NLW) {
                 const int node = __ldg(&a.unodes[u]);
-                const unsigned q0 = (tiles_done * nodes_w + (unsigned)(u / NCW)) * (unsigned)a.cpn;
                 T e[4] = {T(0), T(0), T(0), T(0)};
-                for (int c = 0; c < a.cpn; ++c) {
-                    const unsigned q = q0 + (unsigned)c;
-                    const int stage = warp * S + (int)(q % (unsigned)S);
+                for (int c = 0; c < a.cpn; ++c, ++q) {
+                    const int slot = (int)(q % (unsigned)S);
                     const uint32_t phase = (q / (unsigned)S) & 1u;
+                    // the coefficients of a box are fetched before the wait on its data
                     const T *cf = coeff + (size_t)node * a.m + c * R;
                     T cj[kMaxBoxRows];
 #pragma unroll
                     for (int j = 0; j < kMaxBoxRows; ++j) cj[j] = j < R ? __ldg(cf + j) : T(0);
-                    if (!mbar_wait(&full[stage], phase, &flags[1])) { ok = false; break; }
-                    const T *src = ring + (size_t)stage * stage_elems + lane * 4;
+                    if (!mbar_wait_warp(&my_full[slot], phase, &flags[0])) { ok = false; break; }
+                    const T *src = my_ring + (size_t)slot * stage_elems + lane * 4;
 #pragma unroll
                     for (int j = 0; j < kMaxBoxRows; ++j) {
                         if (j < R) {
@@ -399,50 +460,131 @@ cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchA
                             e[0] += cj[j] * v.x; e[1] += cj[j] * v.y; e[2] += cj[j] * v.z; e[3] += cj[j] * v.w;
                         }
                     }
+                    // every lane has read the box: refill its buffer with box q + stages
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(&empty[stage]);
-                }
-                V4 o; o.x = e[0]; o.y = e[1]; o.z = e[2]; o.w = e[3];
-                *reinterpret_cast<V4 *>(E + (size_t)u * TILE + lane * 4) = o;
-            }
-            // flags[0] is written only by consumers and only before this barrier, so every consumer
-            // warp reads the same value after it and they leave together
-            if (!ok) { flags[0] = 1; atomicExch(a.status, 1); }
-            consumer_barrier(NCW * 32);
-            if (flags[0]) break;
-            // phase 2: replay every pattern's schedule from E.  Lane i fetches entry i of the
-            // pattern's schedule (one coalesced load per 32 entries); entries are then broadcast
-            // with shuffles.
-            const long long gcol = tile * TILE + lane * 4;
-            for (int b = warp; b < a.batch; b += NCW) {
-                T acc[LMAX][4];
-#pragma unroll
-                for (int l = 0; l < LMAX; ++l)
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) acc[l][q] = T(0);
-                const int k0 = __ldg(&a.pat_off[b]), k1 = __ldg(&a.pat_off[b + 1]);
-                for (int kb = k0; kb < k1; kb += 32) {
-                    int4 mine = make_int4(0, 0, 0, 0);
-                    if (kb + lane < k1) mine = __ldg(reinterpret_cast<const int4 *>(&a.steps[kb + lane]));
-                    const int cnt = k1 - kb < 32 ? k1 - kb : 32;
-                    for (int i = 0; i < cnt; ++i) {
-                        const int layer = __shfl_sync(0xffffffffu, mine.y, i);
-                        const uint32_t wb = (uint32_t)__shfl_sync(0xffffffffu, mine.z, i);
-                        const int idx = __shfl_sync(0xffffffffu, mine.w, i);
-                        const V4 v = *reinterpret_cast<const V4 *>(E + (size_t)idx * TILE + lane * 4);
-                        const T e[4] = {v.x, v.y, v.z, v.w};
-                        fold<T, LMAX, 4>(acc, e, layer, weight_of<T>(wb));
+                    if (lane == 0 && issued < total_boxes) {
+                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                        issue_next();
                     }
                 }
-                if (gcol < a.d) {
-                    V4 o;
-                    o.x = finish<T>(acc[0][0], a.shift); o.y = finish<T>(acc[0][1], a.shift);
-                    o.z = finish<T>(acc[0][2], a.shift); o.w = finish<T>(acc[0][3], a.shift);
-                    *reinterpret_cast<V4 *>(reinterpret_cast<T *>(a.out) + (size_t)b * a.d + gcol) = o;
+                V4 o; o.x = e[0]; o.y = e[1]; o.z = e[2]; o.w = e[3];
+                *reinterpret_cast<V4 *>(Eb + (size_t)u * TILE + lane * 4) = o;
+            }
+            if (!ok) break;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&e_full[buf]);
+        }
+        if (!ok) {
+            // give up: flag it, then wait (bounded) for this loader's copies still in flight, so that
+            // none lands in shared memory after the CTA has gone
+            flags[0] = 1;
+            atomicExch(a.status, 1);
+            const unsigned in_flight_end = __shfl_sync(0xffffffffu, issued, 0);
+            for (unsigned b = q; b < in_flight_end; ++b)
+                mbar_wait(&my_full[b % (unsigned)S], (b / (unsigned)S) & 1u, &flags[1]);
+        }
+    } else {
+        // ---------------- replayers: every pattern's schedule from E[buf] ----------------
+        const int rw = warp - NLW;
+        bool ok = true;
+        unsigned t = 0;
+        for (long long tile = blockIdx.x; tile < a.ntiles; tile += gridDim.x, ++t) {
+            const int buf = (int)(t % (unsigned)a.nbuf);
+            const unsigned use = t / (unsigned)a.nbuf;
+            if (!mbar_wait_warp(&e_full[buf], use & 1u, &flags[0])) { ok = false; break; }
+            const T *Eb = E + (size_t)buf * e_elems;
+            const long long gcol = tile * TILE + lane * 4;
+            if (a.sched_smem) {
+                // NP patterns at a time per warp: their schedules visit the same layers, so one
+                // branch per step serves NP independent chains.  Step entries come from the staged
+                // table (broadcast shared-memory loads); the loop is unrolled by two so that the E rows
+                // of the next step are in flight while the current one is folded.
+                const int nst = a.nst;
+                for (int g = rw; g * NP < a.batch; g += NRW) {
+                    T acc[NP][LMAX][4];
+#pragma unroll
+                    for (int p = 0; p < NP; ++p)
+#pragma unroll
+                        for (int l = 0; l < LMAX; ++l)
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) acc[p][l][q] = T(0);
+                    const uint32_t *mine = ent + g * NP;
+                    auto fetch = [&](int k, int &lfk, T (&e)[NP][4], T (&w)[NP]) {
+                        lfk = lf[k];
+                        uint32_t en[NP];
+                        if (NP == 4) {
+                            const uint4 t4 = *reinterpret_cast<const uint4 *>(mine + (size_t)k * batch_pad);
+                            en[0] = t4.x; en[1] = t4.y; en[NP - 2] = t4.z; en[NP - 1] = t4.w;
+                        } else {
+                            const uint2 t2 = *reinterpret_cast<const uint2 *>(mine + (size_t)k * batch_pad);
+                            en[0] = t2.x; en[1] = t2.y;
+                        }
+#pragma unroll
+                        for (int p = 0; p < NP; ++p) {
+                            w[p] = weight_of<T>(wtab_s[en[p] >> 12]);
+                            const V4 v = *reinterpret_cast<const V4 *>(Eb + (size_t)(en[p] & 0xfffu) * TILE + lane * 4);
+                            e[p][0] = v.x; e[p][1] = v.y; e[p][2] = v.z; e[p][3] = v.w;
+                        }
+                    };
+                    int lfA, lfB;
+                    T eA[NP][4], wA[NP], eB[NP][4], wB[NP];
+                    fetch(0, lfA, eA, wA);
+                    for (int k = 0; k < nst; k += 2) {
+                        if (k + 1 < nst) fetch(k + 1, lfB, eB, wB);
+                        fold_many<T, LMAX, NP>(acc, eA, lfA, wA);
+                        if (k + 1 < nst) {
+                            if (k + 2 < nst) fetch(k + 2, lfA, eA, wA);
+                            fold_many<T, LMAX, NP>(acc, eB, lfB, wB);
+                        }
+                    }
+                    if (gcol < a.d) {
+#pragma unroll
+                        for (int p = 0; p < NP; ++p) {
+                            const int b = g * NP + p;
+                            if (b < a.batch) {
+                                V4 o;
+                                o.x = finish<T>(acc[p][0][0], a.shift); o.y = finish<T>(acc[p][0][1], a.shift);
+                                o.z = finish<T>(acc[p][0][2], a.shift); o.w = finish<T>(acc[p][0][3], a.shift);
+                                *reinterpret_cast<V4 *>(reinterpret_cast<T *>(a.out) + (size_t)b * a.d + gcol) = o;
+                            }
+                        }
+                    }
+                }
+            } else {
+                // General case, one pattern at a time: lane i fetches entry i of the pattern's schedule
+                // (one coalesced load per 32 entries); entries are broadcast with shuffles.
+                for (int b = rw; b < a.batch; b += NRW) {
+                    T acc[LMAX][4];
+#pragma unroll
+                    for (int l = 0; l < LMAX; ++l)
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) acc[l][q] = T(0);
+                    const int k0 = __ldg(&a.pat_off[b]), k1 = __ldg(&a.pat_off[b + 1]);
+                    for (int kb = k0; kb < k1; kb += 32) {
+                        int4 mine = make_int4(0, 0, 0, 0);
+                        if (kb + lane < k1) mine = __ldg(reinterpret_cast<const int4 *>(&a.steps[kb + lane]));
+                        const int cnt = k1 - kb < 32 ? k1 - kb : 32;
+                        for (int i = 0; i < cnt; ++i) {
+                            const int layer = __shfl_sync(0xffffffffu, mine.y, i) & 0xff;
+                            const uint32_t wb = (uint32_t)__shfl_sync(0xffffffffu, mine.z, i);
+                            const int idx = __shfl_sync(0xffffffffu, mine.w, i) & pos_mask;
+                            const V4 v = *reinterpret_cast<const V4 *>(Eb + (size_t)idx * TILE + lane * 4);
+                            const T e[4] = {v.x, v.y, v.z, v.w};
+                            fold<T, LMAX, 4>(acc, e, layer, weight_of<T>(wb));
+                        }
+                    }
+                    if (gcol < a.d) {
+                        V4 o;
+                        o.x = finish<T>(acc[0][0], a.shift); o.y = finish<T>(acc[0][1], a.shift);
+                        o.z = finish<T>(acc[0][2], a.shift); o.w = finish<T>(acc[0][3], a.shift);
+                        *reinterpret_cast<V4 *>(reinterpret_cast<T *>(a.out) + (size_t)b * a.d + gcol) = o;
+                    }
                 }
             }
-            consumer_barrier(NCW * 32);  // E is rewritten by the next tile
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&e_free[buf]);  // this warp has finished reading E[buf]
         }
+        if (!ok) { flags[0] = 1; atomicExch(a.status, 1); }
     }
 }
 
@@ -787,23 +929,32 @@ cudaError_t launch_fused_tma(const AggArgs &a, const DeviceInfo &dev, const Tuni
     return err;
 }
 
-template <typename T, int LMAX, int NCW>
+template <typename T, int LMAX, int NLW, int NRW>
 static cudaError_t run_batch(const CUtensorMap &map, const BatchArgs &ba, int grid, size_t smem, cudaStream_t stream) {
-    auto kern = cr_fused_batch_tma_kernel<T, LMAX, NCW>;
+    auto kern = cr_fused_batch_tma_kernel<T, LMAX, NLW, NRW>;
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
-    kern<<<grid, (NCW + 1) * 32, smem, stream>>>(map, ba);
+    kern<<<grid, (NLW + NRW) * 32, smem, stream>>>(map, ba);
     return cudaGetLastError();
 }
 
-template <typename T, int NCW>
+template <typename T, int NLW, int NRW>
 static cudaError_t run_batch_l(int lmax, const CUtensorMap &map, const BatchArgs &ba, int grid, size_t smem,
                                cudaStream_t stream) {
     switch (lmax) {
-        case 2: return run_batch<T, 2, NCW>(map, ba, grid, smem, stream);
-        case 4: return run_batch<T, 4, NCW>(map, ba, grid, smem, stream);
-        default: return run_batch<T, 8, NCW>(map, ba, grid, smem, stream);
+        case 2: return run_batch<T, 2, NLW, NRW>(map, ba, grid, smem, stream);
+        case 4: return run_batch<T, 4, NLW, NRW>(map, ba, grid, smem, stream);
+        default: return run_batch<T, 8, NLW, NRW>(map, ba, grid, smem, stream);
     }
+}
+
+template <typename T>
+static cudaError_t run_batch_w(int nlw, int nrw, int lmax, const CUtensorMap &map, const BatchArgs &ba, int grid,
+                               size_t smem, cudaStream_t stream) {
+    if (nlw == 6) return nrw == 4 ? run_batch_l<T, 6, 4>(lmax, map, ba, grid, smem, stream)
+                                  : run_batch_l<T, 6, 8>(lmax, map, ba, grid, smem, stream);
+    return nrw == 4 ? run_batch_l<T, 4, 4>(lmax, map, ba, grid, smem, stream)
+                    : run_batch_l<T, 4, 8>(lmax, map, ba, grid, smem, stream);
 }
 
 cudaError_t launch_fused_batch_tma(const AggArgs &a, const DeviceInfo &dev, const Tuning &tune, EncodeTiledFn encode,
@@ -811,33 +962,52 @@ cudaError_t launch_fused_batch_tma(const AggArgs &a, const DeviceInfo &dev, cons
     *done = false;
     if (!encode || !tma_eligible(a)) return cudaSuccess;
     const int tile = 128;
-    const int ncw = (tune.ncw == 2 || tune.ncw == 4 || tune.ncw == 8) ? tune.ncw : 4;
-    const size_t e_bytes = (size_t)a.n_union * tile * 4;
-    const size_t usable = (size_t)dev.smem_per_sm - 2048;
-    // Shared memory = E + ncw private rings of `stages` boxes of R rows.  Prefer two CTAs per SM (one
-    // replays patterns while the other streams), at least 2 boxes per ring, boxes as tall as fit.
-    int ctas = tune.ctas_per_sm ? tune.ctas_per_sm : 2, stages = 0, R = 0;
-    for (; ctas >= 1 && !stages; --ctas) {
-        const size_t budget = std::min(usable / ctas - 1024, (size_t)dev.smem_optin);
-        if (budget <= e_bytes + 256) continue;
-        const size_t ring_budget = budget - e_bytes - 256;
-        const int want_stages = tune.stages ? tune.stages : 3;
-        for (int depth = want_stages; depth >= 2 && !stages; --depth) {
-            // tallest box (a divisor of m, at most kMaxBoxRows) such that ncw * depth boxes fit
-            const int cap = (int)std::min<size_t>(kMaxBoxRows, ring_budget / ((size_t)ncw * depth * tile * 4));
-            if (cap < 1) continue;
-            const int r = tune.rows && a.m % tune.rows == 0 && tune.rows <= cap ? tune.rows : rows_per_box(a.m, cap);
-            if (r * 4 < std::min(a.m, 8) && depth > 2) continue;  // prefer taller boxes over a third buffer
-            R = r; stages = depth;
-        }
-        if (stages) break;
+    const int nrw = tune.ncw == 4 ? 4 : 8;  // replay warps
+    // same-shape batches stage their schedules in shared memory (layer word per step, one 4-byte entry
+    // per step and pattern, patterns padded to the replay group size, the weight table) when small
+    const int lmax = pick_lmax(a.L);
+    const int np = lmax <= 4 ? 4 : 2;
+    const int nst = a.same_shape && a.batch > 0 ? a.total_steps / a.batch : 0;
+    size_t sched_bytes = 0;
+    if (a.same_shape && nst > 0 && a.n_wtab > 0) {
+        const size_t want = (((size_t)nst * 4 + 15) & ~(size_t)15) +
+                            (((size_t)nst * ((a.batch + np - 1) / np * np) + 3) & ~(size_t)3) * 4 +
+                            (((size_t)a.n_wtab * 4 + 15) & ~(size_t)15);
+        if (want <= 24 * 1024) sched_bytes = (want + 15) & ~(size_t)15;
     }
-    if (!stages) return cudaSuccess;  // union too large for shared memory: caller falls back
+    const size_t e_one = (size_t)a.n_union * tile * 4;
+    const size_t budget = (size_t)dev.smem_optin - 512;   // barriers and flags take the rest
+    // Shared memory = nbuf x E + staged schedules + one private ring of `stages` boxes of R rows per
+    // loader warp.  Measured on B200 (d = 2^22, m = 16, 120 nodes, 64 patterns): six loaders with two
+    // boxes of 8 KB each stream at the copy bandwidth; four loaders reach 90 % of it, boxes of 4 KB two
+    // thirds, a third box per loader adds nothing.  So: boxes as tall as fit come first, then the
+    // second E buffer, then six loaders rather than four.
+    int nbuf = 0, stages = 0, R = 0, nlw = 0;
+    const int want_loaders = tune.ctas_per_sm == 4 ? 4 : 6;
+    for (int try_buf = 2; try_buf >= 1 && !nbuf; --try_buf) {
+        if (budget <= try_buf * e_one + sched_bytes) continue;
+        const size_t ring_budget = budget - try_buf * e_one - sched_bytes;
+        const int want_stages = tune.stages ? tune.stages : 2;
+        int best_r = 0, best_depth = 0, best_lw = 0;
+        for (int lw = want_loaders; lw >= 4; lw -= 2) {
+            for (int depth = want_stages; depth >= 2; --depth) {
+                const int cap = (int)std::min<size_t>(kMaxBoxRows, ring_budget / ((size_t)lw * depth * tile * 4));
+                if (cap < 1) continue;
+                const int r = tune.rows && a.m % tune.rows == 0 && tune.rows <= cap ? tune.rows : rows_per_box(a.m, cap);
+                if (r > best_r) { best_r = r; best_depth = depth; best_lw = lw; }
+            }
+        }
+        // two buffers only if they do not cost more than half of the box height one buffer allows
+        if (best_r && (try_buf == 1 || 2 * best_r >= std::min(a.m, kMaxBoxRows))) {
+            nbuf = try_buf; R = best_r; stages = best_depth; nlw = best_lw;
+        }
+    }
+    if (!nbuf) return cudaSuccess;  // union too large for shared memory: caller falls back
     const size_t stage_bytes = (size_t)R * tile * 4;
-    const size_t smem = (size_t)ncw * stages * stage_bytes + e_bytes + (size_t)ncw * stages * 16 + 32;
+    const size_t smem = (size_t)nlw * stages * stage_bytes + nbuf * e_one + sched_bytes + (size_t)nlw * stages * 8 + 64 + 16;
     if (smem > (size_t)dev.smem_optin) return cudaSuccess;
     const long long ntiles = (a.d + tile - 1) / tile;
-    const int grid = (int)std::min<long long>(ntiles, (long long)dev.sm_count * ctas);
+    const int grid = (int)std::min<long long>(ntiles, (long long)dev.sm_count);
     // box counters are 32-bit
     if ((ntiles / grid + 1) * (long long)a.n_union * (a.m / R) >= (1ll << 31)) return cudaSuccess;
 
@@ -846,19 +1016,11 @@ cudaError_t launch_fused_batch_tma(const AggArgs &a, const DeviceInfo &dev, cons
 
     BatchArgs ba;
     ba.coeff = a.coeff; ba.steps = a.steps; ba.pat_off = a.pat_off; ba.unodes = a.unodes; ba.n_union = a.n_union;
-    ba.batch = a.batch; ba.m = a.m; ba.R = R; ba.cpn = a.m / R; ba.stages = stages; ba.d = a.d; ba.ntiles = ntiles;
-    ba.out = a.out; ba.shift = a.shift; ba.status = a.status;
-    const int lmax = pick_lmax(a.L);
-    cudaError_t err;
-    if (a.is_int) {
-        err = ncw == 2 ? run_batch_l<int, 2>(lmax, map, ba, grid, smem, stream)
-            : ncw == 8 ? run_batch_l<int, 8>(lmax, map, ba, grid, smem, stream)
-                       : run_batch_l<int, 4>(lmax, map, ba, grid, smem, stream);
-    } else {
-        err = ncw == 2 ? run_batch_l<float, 2>(lmax, map, ba, grid, smem, stream)
-            : ncw == 8 ? run_batch_l<float, 8>(lmax, map, ba, grid, smem, stream)
-                       : run_batch_l<float, 4>(lmax, map, ba, grid, smem, stream);
-    }
+    ba.batch = a.batch; ba.same_shape = a.same_shape; ba.m = a.m; ba.R = R; ba.cpn = a.m / R; ba.stages = stages;
+    ba.d = a.d; ba.ntiles = ntiles; ba.out = a.out; ba.shift = a.shift; ba.status = a.status;
+    ba.sched_smem = (int)sched_bytes; ba.nst = nst; ba.nbuf = nbuf; ba.wtab = a.wtab; ba.n_wtab = a.n_wtab;
+    const cudaError_t err = a.is_int ? run_batch_w<int>(nlw, nrw, lmax, map, ba, grid, smem, stream)
+                                     : run_batch_w<float>(nlw, nrw, lmax, map, ba, grid, smem, stream);
     if (err == cudaSuccess) { *done = true; ++*launches; }
     return err;
 }

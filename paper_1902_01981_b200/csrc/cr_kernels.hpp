@@ -11,16 +11,17 @@ namespace cr {
 // One consumed node of an expanded straggler pattern, as the kernels read it (16 bytes).
 struct Step {
     int32_t node;    // flat node index: its slots are rows node*m .. node*m+m-1 of G_slots
-    int32_t layer;   // 1..L
+    int32_t layer;   // bits 0..7: layer 1..L; bit 8: first consumed child of its parent
     uint32_t wbits;  // decode weight of the node's message at its parent: float bits (CR_F32) or int32 (CR_I32)
-    int32_t index;   // batch kernel: position of the node in the union list; otherwise unused
+    int32_t index;   // batch kernel: position of the node in the union list (bits 0..11) and, when the batch
+                     // has a weight table, the index of wbits in it (bits 12..); otherwise unused
 };
 
 // Tuning of the TMA kernels; 0 selects the built-in choice.
 struct Tuning {
     int ncw = 0;          // consumer warps per CTA (single-pattern kernel: tile = 128 * ncw columns)
     int stages = 0;       // depth of the shared-memory ring
-    int ctas_per_sm = 0;  // persistent CTAs per SM
+    int ctas_per_sm = 0;  // persistent CTAs per SM (batch kernel, always one CTA per SM: loader warps, 4 or 6)
     int rows = 0;         // slot rows per TMA box (must divide m)
 };
 
@@ -36,6 +37,8 @@ struct AggArgs {
     const Step *steps;    // device: all patterns' steps, concatenated
     const int32_t *pat_off;  // device [batch+1]: pattern b owns steps pat_off[b] .. pat_off[b+1]-1
     const int32_t *unodes;   // device [n_union]: union of used nodes (batch kernel)
+    const uint32_t *wtab;    // device [n_wtab]: distinct weight bit patterns of the batch (n_wtab = 0: none)
+    int n_wtab;
     int n_union;
     int batch;
     int total_steps;
@@ -47,6 +50,7 @@ struct AggArgs {
     int shift;            // CR_I32: arithmetic right shift applied at the root
     int *status;          // device status word (bounded waits)
     int is_int;
+    int same_shape;       // batch > 1: all patterns' schedules share length and layer sequence
 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,

@@ -174,7 +174,10 @@ static bool decode_table(int n, int s, int code, const std::vector<double> &B, s
             for (int k = 0; k < n; ++k)
                 for (int t = 0; t < q; ++t) At[(size_t)k * q + t] = B[(size_t)U[t] * n + k];
             if (!least_squares(At, n, q, ones, sol)) return false;
-            for (int t = 0; t < q; ++t) a[U[t]] = sol[t];
+            // weights that are pure rounding noise of the solve (a survivor that is not needed) are zero
+            double big = 0.0;
+            for (int t = 0; t < q; ++t) big = std::max(big, std::fabs(sol[t]));
+            for (int t = 0; t < q; ++t) a[U[t]] = std::fabs(sol[t]) <= 1e-13 * big ? 0.0 : sol[t];
         }
         double amp = 0.0;
         for (int j = 0; j < n; ++j) amp += std::fabs(a[j]) * rownorm[j];
@@ -210,9 +213,9 @@ bool HostPlan::mask_ok(uint32_t mask) const { return (mask >> n) == 0 && popcoun
 
 cr_status_t HostPlan::expand(const uint32_t *masks, std::vector<UsedNode> &out) const {
     // Iterative post-order walk.  A frame is a parent (layer, index in layer) and the next child to visit.
-    struct Frame { int layer, index, next; double weight; };
+    struct Frame { int layer, index, next; double weight; bool first; int seen; };
     std::vector<Frame> stack;
-    stack.push_back({0, 0, 0, 0.0});
+    stack.push_back({0, 0, 0, 0.0, true, 0});
     while (!stack.empty()) {
         Frame &f = stack.back();
         const int group = f.layer == 0 ? 0 : layer_offset[f.layer] + f.index + 1;
@@ -224,17 +227,19 @@ cr_status_t HostPlan::expand(const uint32_t *masks, std::vector<UsedNode> &out) 
         while (j < n && a[j] == 0.0) ++j;
         if (j == n) {
             // all used children done: emit this parent itself (not the master)
-            if (f.layer > 0) out.push_back({layer_offset[f.layer] + f.index, f.layer, f.weight});
+            if (f.layer > 0) out.push_back({layer_offset[f.layer] + f.index, f.layer, f.weight, f.first});
             stack.pop_back();
             continue;
         }
         f.next = j + 1;
+        const bool child_first = f.seen == 0;
+        ++f.seen;
         const int cl = f.layer + 1, ci = f.index * n + j;
         if (cl == L) {
-            out.push_back({layer_offset[cl] + ci, cl, a[j]});
+            out.push_back({layer_offset[cl] + ci, cl, a[j], child_first});
         } else {
             const double w = a[j];
-            stack.push_back({cl, ci, 0, w});  // invalidates f
+            stack.push_back({cl, ci, 0, w, child_first, 0});  // invalidates f
         }
     }
     return CR_OK;

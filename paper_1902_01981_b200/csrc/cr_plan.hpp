@@ -23,6 +23,7 @@ struct UsedNode {
     int32_t node;
     int32_t layer;
     double weight;
+    bool first;  // first consumed child of its parent (in visiting order)
 };
 
 struct HostPlan {

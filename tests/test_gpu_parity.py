@@ -133,6 +133,30 @@ def test_random_patterns_medium_trees(cfg, batch, flags):
         B.cr_plan_destroy(plan)
 
 
+def test_batch_of_patterns_with_different_shapes():
+    """An explicit code whose decode rows use two or three children depending on the straggler:
+    the patterns of one batch then have schedules of different lengths."""
+    Bx = np.array([[1, 1, 0, 0], [0, 0, 1, 1], [1, 0, 2, 0], [0, 1, 0, 2]], dtype=np.float64)
+    n, L, s, d = 4, 2, 1, 6000
+    P = O.partition_quantum(n, L, s)
+    plan = B.cr_plan_create(n, L, s, P, d, code=B.CR_CODE_EXPLICIT, B_explicit=np.stack([Bx, Bx]), device=0)
+    try:
+        code = O.Code(n, L, s, [Bx, Bx], kind="solve")
+        local, _ = O.allocate(n, L, s, P, code.B_levels)
+        assert B.slot_partitions(plan).tolist() == [[p for p, _ in pairs] for pairs in local]
+        G = inputs.partition_gradients(P, d, seed=17)
+        G_dev = slots_on_device(plan, G, torch)
+        masks = inputs.straggler_masks(n, L, s, 24, seed=19)
+        lengths = {len(B.cr_plan_expand(plan, masks[b])[0]) for b in range(24)}
+        assert len(lengths) > 1
+        for flags in FUSED_VARIANTS:
+            got = run_aggregate(plan, G_dev, masks, d, flags)
+            for b in range(24):
+                assert rel_l2(got[b], O.execute(code, local, G, masks[b])) <= REL_L2_BAR
+    finally:
+        B.cr_plan_destroy(plan)
+
+
 def test_fused_matches_unfused_closely():
     cfg = tree(5, 2, 2, "cyclic", 1 << 16)
     plan = make_plan(cfg)
