@@ -38,7 +38,8 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the timed kernel, from the ncu capture
 # summarised under profiles/ (absent = no capture of the current kernel on that workload).
 # cfg4: 917.4 MB measured at d = 2^21, scaled by 8 to d = 2^24 (traffic is proportional to d).
-NCU_TRAFFIC_BYTES = {("cfg4", "f32", 1 << 24): 8 * 917.37e6}
+# cfg5: 2083.3 MB measured at d = 2^18, scaled by 16 to d = 2^22.
+NCU_TRAFFIC_BYTES = {("cfg4", "f32", 1 << 24): 8 * 917.37e6, ("cfg5", "f32", 1 << 22): 16 * 2083.3e6}
 
 
 def peak_hbm():
@@ -155,6 +156,16 @@ def oracle_sample(cfg, d_sample: int, steps: int, warmup: int, G=None):
     return float(np.mean(times)), float(np.mean(nbytes)), last, masks[-1]
 
 
+def calibrated_columns(cfg, steps: int, seconds: float, max_cols: int) -> int:
+    """Largest power-of-two column count (>= 4096, <= max_cols) for which `steps` oracle steps take
+    about `seconds`, from one timed step on 4096 columns."""
+    sec, _, _, _ = oracle_sample(cfg, 4096, 1, 0)
+    cols = 4096
+    while cols * 2 <= max_cols and sec * (cols * 2 / 4096.0) * steps <= seconds:
+        cols *= 2
+    return cols
+
+
 def host_threads() -> int:
     try:
         return len(os.sched_getaffinity(0))
@@ -167,15 +178,8 @@ def run_reference(args, cfg):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    # bounded sample: about a minute of oracle time for the whole run at ~0.8 GB/s of algorithmic bytes
-    n_used = sum((cfg["n"] - cfg["s"]) ** l for l in range(1, cfg["L"] + 1))
-    m = cfg["P"] * (cfg["s"] + 1) ** cfg["L"] // sum(cfg["n"] ** l * (cfg["s"] + 1) ** (cfg["L"] - l)
-                                                      for l in range(1, cfg["L"] + 1))
-    per_col = 4 * (m * n_used + 1) * cfg.get("batch", 1)
-    budget_cols = int(60.0 * 0.8e9 / ((args.steps + args.warmup) * per_col))
-    d_sample = 4096
-    while d_sample * 2 <= min(budget_cols, args.ref_columns, cfg["d"]):
-        d_sample *= 2
+    # bounded sample: calibrate the oracle on 4096 columns, then size the sample for about a minute
+    d_sample = calibrated_columns(cfg, args.steps + args.warmup, 60.0, min(args.ref_columns, cfg["d"]))
     sec, nbytes, _, _ = oracle_sample(cfg, d_sample, args.steps, args.warmup)
     value = nbytes / sec / 1e9
     sample = f"first {d_sample} of {cfg['d']} columns, every step a fresh straggler pattern"
@@ -362,7 +366,7 @@ def run_ours(args, cfg):
                     "avg_launch_ms": avg_launch * 1e3, "best_launch_ms": float(per.min()) * 1e3}
         cpu = None
         if not args.no_cpu_baseline:
-            d_sample = min(d, args.cpu_columns)
+            d_sample = calibrated_columns(cfg, args.cpu_steps + 1, 15.0, min(d, args.cpu_columns))
             sec, nbytes, last, last_masks = oracle_sample(
                 cfg, d_sample, args.cpu_steps, 1, np.ascontiguousarray(G_parts[:, :d_sample])) \
                 if not is_int else (None, None, None, None)
