@@ -396,13 +396,96 @@ def run_ours(args, cfg):
         dist.destroy_process_group()
 
 
+def run_linreg(args, cfg):
+    """End-to-end gradient-descent step of a linear-regression workload (cfg1, cfg3): partial gradients of
+    every node's slots, fused aggregation under a fresh straggler pattern, model update.  One GPU."""
+    import torch
+    from paper_1902_01981_b200 import binding as B
+    from paper_1902_01981_b200 import build as cr_build
+    cr_build.build()
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(0)
+    code_id = {"printed_3_1": B.CR_CODE_PAPER_3_1, "cyclic": B.CR_CODE_CYCLIC_RANDOM,
+               "repetition": B.CR_CODE_FRACTIONAL_REPETITION}[cfg["code"]]
+    n, L, s, P, d, rows = cfg["n"], cfg["L"], cfg["s"], cfg["P"], cfg["d"], cfg["rows"]
+    plan = B.cr_plan_create(n, L, s, P, d, code=code_id, device=0)
+    N, m, groups = B.cr_plan_num_nodes(plan), B.cr_plan_load(plan), B.cr_plan_num_groups(plan)
+    X, y, w_star = inputs.linreg_partitions(P, rows, d, cfg["seed"], cfg["x_std"], cfg["noise_std"])
+    X_dev, y_dev = torch.from_numpy(X).cuda(), torch.from_numpy(y).cuda()
+    w_dev = torch.zeros(d, device="cuda")
+    G_slots = torch.zeros((N, m, d), device="cuda")
+    ws = torch.empty(max(16, B.cr_partial_gradients_workspace_bytes(plan, rows)), dtype=torch.uint8, device="cuda")
+    out = torch.zeros((1, d), device="cuda")
+    total = min(args.steps + args.warmup, 256)
+    masks = inputs.straggler_masks(n, L, s, total, cfg.get("mask_seed", 1))
+    lr_eff = cfg["lr"] / P if args.workload == "cfg3" else cfg["lr"]
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if X.nbytes <= 126e6 else None
+    stream = torch.cuda.current_stream()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+
+    def step(i, events=None):
+        if events:
+            events[0].record(stream)
+        B.cr_partial_gradients(plan, X_dev, y_dev, rows, w_dev, G_slots, ws, stream)
+        if events:
+            events[1].record(stream)
+        B.cr_aggregate(plan, G_slots, masks[i % total], out, B.CR_AGG_FUSED, None, stream)
+        w_dev.sub_(out[0], alpha=lr_eff)
+        if events:
+            events[2].record(stream)
+
+    for i in range(args.warmup):
+        step(i)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.wait_first_sample()
+    n0 = B.cr_plan_launch_count(plan)
+    t0 = time.time()
+    for i in range(args.steps):
+        if flush is not None:
+            flush.fill_(i & 0xff)
+        step(args.warmup + i, ev[i])
+    torch.cuda.synchronize()
+    t1 = time.time()
+    launches = B.cr_plan_launch_count(plan) - n0
+    clocks = sampler.stop((t0, t1))
+    t_grad = np.array([e[0].elapsed_time(e[1]) for e in ev]) * 1e-3
+    t_step = np.array([e[0].elapsed_time(e[2]) for e in ev]) * 1e-3
+    elapsed = float(t_step.sum())
+    # algorithmic bytes: every (node, slot) reads its partition once; the aggregation reads the consumed slots
+    grad_bytes = 4.0 * rows * d * N * m
+    agg_bytes = float(np.mean([B.cr_aggregate_bytes(plan, masks[i])[0] for i in range(total)]))
+    step_bytes = grad_bytes + agg_bytes
+    peak, peak_kind = peak_hbm()
+    achieved = grad_bytes / float(t_grad.mean()) / 1e9
+    w_final = w_dev.cpu().numpy()
+    line = {
+        "metric": METRIC, "value": step_bytes * args.steps / elapsed / 1e9, "unit": UNIT, "n_gpus": 1,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": elapsed / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{args.workload}: linear regression n={n} L={L} s={s} P={P} rows={rows} d={d}, "
+                               "step = partial gradients of all N*m slots + fused aggregation + model update",
+                   "l2": "inputs larger than L2 (no flush needed)" if flush is None else "L2 flushed between steps"},
+        "iterations_per_s": args.steps / elapsed,
+        "roofline": {"bound": "hbm", "kernel": "partial gradients", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "algorithmic_bytes_per_launch": grad_bytes, "avg_launch_ms": float(t_grad.mean()) * 1e3,
+                     "aggregate_ms": float((t_step - t_grad).mean()) * 1e3},
+        "cpu_baseline": None, "e2e": None, "gpu_launches": int(launches), "clocks": clocks,
+        "normalized_error_rate": float(np.sum((w_final - w_star) ** 2) / np.sum(w_star ** 2)),
+    }
+    print(json.dumps(line), flush=True)
+    B.cr_plan_destroy(plan)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=2000)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg4", choices=[k for k, v in inputs.CONFIGS.items() if v["kind"] == "aggregate"])
+    ap.add_argument("--workload", default="cfg4", choices=list(inputs.CONFIGS))
     ap.add_argument("--dtype", default="f32", choices=["f32", "int32"])
     ap.add_argument("--d", type=int, default=0, help="override the gradient length (profiling on a small case)")
     ap.add_argument("--tune", default="", help="consumer_warps,stages,ctas_per_sm,rows_per_box (0 = auto)")
@@ -422,7 +505,12 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     if args.gpus != world and world > 1:
         args.gpus = world
-    if args.impl == "reference":
+    if cfg["kind"] == "linreg":
+        if args.impl == "reference":
+            print(json.dumps({"impl": "reference", "unavailable": "the reference arm times aggregation workloads only"}))
+        else:
+            run_linreg(args, cfg)
+    elif args.impl == "reference":
         run_reference(args, cfg)
     else:
         run_ours(args, cfg)

@@ -143,8 +143,12 @@ cr_status_t cr_plan_device_status(cr_plan_t *plan);
  * Linear-regression instance of Eq. (g): for every node v and slot j holding partition p,
  *   G_slots[v][j][:] = X_p^T (X_p w - y_p).
  * X [P][rows][d], y [P][rows], w [d], G_slots [N][m][d]: device pointers, fp32, row-major.
- * workspace: device scratch of at least cr_partial_gradients_workspace_bytes(plan, rows) bytes
- * (residuals, one per node, slot and row).  CR_F32 plans only. */
+ * Two kernels serve it: when d % 4 == 0, d <= 8192 and X, w, G_slots are 16-byte aligned, a one-pass
+ * kernel (row blocks staged by TMA bulk copies, a cluster of CTAs per slot, reduction through
+ * distributed shared memory) that needs no scratch; otherwise a two-pass kernel pair that keeps the
+ * residuals (one per node, slot and row) in `workspace`, device scratch of at least
+ * cr_partial_gradients_workspace_bytes(plan, rows) bytes (CR_ERR_OOM if it is needed and missing).
+ * CR_F32 plans only. */
 size_t cr_partial_gradients_workspace_bytes(const cr_plan_t *plan, int32_t rows);
 cr_status_t cr_partial_gradients(cr_plan_t *plan, const float *X, const float *y, int32_t rows,
                                  const float *w, float *G_slots, void *workspace,

@@ -336,10 +336,18 @@ cr_status_t cr_partial_gradients(cr_plan_t *plan, const float *X, const float *y
     if (st != CR_OK) return st;
     if (!X || !y || !w || !G_slots || rows < 1) return CR_ERR_INVALID_ARG;
     if (plan->hp.dtype != CR_F32) return CR_ERR_DTYPE;
-    if (!workspace || workspace_bytes < cr_partial_gradients_workspace_bytes(plan, rows)) return CR_ERR_OOM;
-    cudaError_t e = cr::launch_partial_gradients(X, y, w, plan->d_part, plan->hp.N * plan->hp.m, rows, plan->hp.d,
-                                                 reinterpret_cast<float *>(workspace), G_slots,
-                                                 reinterpret_cast<cudaStream_t>(stream), &plan->launches);
+    const int items = plan->hp.N * plan->hp.m;
+    cudaError_t e;
+    if (cr::partial_fused_eligible(X, w, G_slots, plan->hp.d, items)) {
+        // one pass over X, no scratch
+        e = cr::launch_partial_gradients_fused(X, y, w, plan->d_part, items, rows, plan->hp.d, G_slots, plan->d_status,
+                                               plan->dev, reinterpret_cast<cudaStream_t>(stream), &plan->launches);
+    } else {
+        if (!workspace || workspace_bytes < cr_partial_gradients_workspace_bytes(plan, rows)) return CR_ERR_OOM;
+        e = cr::launch_partial_gradients_two_pass(X, y, w, plan->d_part, items, rows, plan->hp.d,
+                                                  reinterpret_cast<float *>(workspace), G_slots,
+                                                  reinterpret_cast<cudaStream_t>(stream), &plan->launches);
+    }
     if (e != cudaSuccess) { note_cuda(e, "cr_partial_gradients"); return CR_ERR_CUDA; }
     return CR_OK;
 }
@@ -593,7 +601,7 @@ cr_status_t cr_partial_gradients_static(cr_plan_t *plan, const float *X, const f
         }
         scratch = g_static_ptr[plan->device];
     }
-    cudaError_t e = cr::launch_partial_gradients(X, y, w, plan->d_part, plan->hp.N * plan->hp.m, rows, plan->hp.d,
+    cudaError_t e = cr::launch_partial_gradients_two_pass(X, y, w, plan->d_part, plan->hp.N * plan->hp.m, rows, plan->hp.d,
                                                  scratch, G_slots, reinterpret_cast<cudaStream_t>(stream),
                                                  &plan->launches);
     if (e != cudaSuccess) { note_cuda(e, "cr_partial_gradients_static"); return CR_ERR_CUDA; }

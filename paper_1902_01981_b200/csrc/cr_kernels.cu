@@ -7,6 +7,8 @@
 // or shared memory; only the root tile is written.
 #include "cr_kernels.hpp"
 
+#include <cooperative_groups.h>
+
 #include <algorithm>
 #include <cstdio>
 
@@ -828,6 +830,185 @@ cr_xt_r_kernel(const float *__restrict__ X, const int32_t *__restrict__ part, co
 }
 
 // ------------------------------------------------------------------------------------------------
+// K1 (one pass): X_p^T (X_p w - y_p) with every X element read from HBM once
+// ------------------------------------------------------------------------------------------------
+//
+// A cluster of `csplit` CTAs owns one (node, slot) item; CTA c takes a contiguous range of the
+// partition's rows.  A block of RB consecutive rows is one contiguous piece of X, so it is staged with a
+// single bulk copy (TMA, no tensor map) into a ring of shared-memory buffers.  Per block: pass A forms
+// the residuals r = X_b w - y_b (warp-shuffle reduction, then across the 8 warps through shared
+// memory), pass B adds r^T X_b to the thread's column accumulators, both from shared memory.  Thread t
+// owns columns 4t + 1024k .. +3 (k < KPT), so d <= 1024 * KPT.  At the end the CTAs of the cluster add
+// their partial gradients through distributed shared memory, each CTA reducing and storing one slice
+// of the columns: deterministic, no atomics, no scratch in global memory.
+
+struct PgArgs {
+    const float *X;
+    const float *y;
+    const float *w;
+    const int32_t *part;
+    float *G;
+    int rows;
+    int rows_per_cta;
+    int RB;
+    int stages;
+    long long d;
+    int *status;
+};
+
+__device__ __forceinline__ void bulk_load_1d(void *smem_dst, const void *gsrc, uint32_t bytes, uint64_t *bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
+        : "memory");
+}
+
+template <int KPT>
+__global__ void __launch_bounds__(256, 1)
+cr_partial_fused_kernel(const PgArgs a) {
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    constexpr int RG = 4;  // rows handled together in pass A
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const long long d = a.d;
+    const int RB = a.RB, S = a.stages;
+    const size_t stage_elems = (size_t)RB * d;
+    float *ring = reinterpret_cast<float *>(smem_raw);
+    float *gpart = ring + (size_t)S * stage_elems;          // [d] this CTA's partial gradient
+    float *red = gpart + d;                                 // [RB][8] per-warp partial residuals
+    float *rfin = red + (size_t)RB * 8;                     // [RB] residuals of the block
+    uint64_t *full = reinterpret_cast<uint64_t *>(rfin + ((RB + 3) & ~3));
+    volatile int *flags = reinterpret_cast<volatile int *>(full + S);
+
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) mbar_init(&full[s], 1);
+        flags[0] = 0; flags[1] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    const long long item = blockIdx.y;
+    const int p = __ldg(&a.part[item]);
+    const int r0 = min(a.rows, (int)blockIdx.x * a.rows_per_cta);
+    const int r1 = min(a.rows, r0 + a.rows_per_cta);
+    const int nblocks = (r1 - r0 + RB - 1) / RB;
+    const float *Xp = a.X + ((size_t)p * a.rows + r0) * d;
+    const float *yp = a.y + (size_t)p * a.rows + r0;
+
+    float4 wv[KPT], acc[KPT];
+#pragma unroll
+    for (int k = 0; k < KPT; ++k) {
+        const long long col = 4ll * tid + 1024ll * k;
+        wv[k] = col < d ? __ldg(reinterpret_cast<const float4 *>(a.w + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+
+    int issued = 0;
+    auto issue = [&](int blk) {  // thread 0 only
+        const int nr = min(RB, (r1 - r0) - blk * RB);
+        const uint32_t bytes = (uint32_t)((size_t)nr * d * sizeof(float));
+        mbar_expect_tx(&full[blk % S], bytes);
+        bulk_load_1d(ring + (size_t)(blk % S) * stage_elems, Xp + (size_t)blk * RB * d, bytes, &full[blk % S]);
+    };
+    if (tid == 0)
+        for (; issued < nblocks && issued < S - 1; ++issued) issue(issued);
+
+    int done = 0;
+    for (int blk = 0; blk < nblocks; ++blk) {
+        const int nr = min(RB, (r1 - r0) - blk * RB);
+        // label of this thread's row, fetched before the wait so that its latency hides behind it
+        const float yv = tid < nr ? __ldg(yp + (size_t)blk * RB + tid) : 0.f;
+        // all threads have left the previous block once this barrier is passed, so its buffer is free
+        const int ok = __syncthreads_and(mbar_wait(&full[blk % S], (uint32_t)((blk / S) & 1), &flags[1]) ? 1 : 0);
+        if (!ok) break;
+        if (tid == 0 && issued < nblocks) {
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            issue(issued);
+            ++issued;
+        }
+        const float *Xb = ring + (size_t)(blk % S) * stage_elems;
+        // pass A: residual partials, RG rows at a time
+        for (int rg = 0; rg < nr; rg += RG) {
+            float part[RG];
+#pragma unroll
+            for (int i = 0; i < RG; ++i) part[i] = 0.f;
+#pragma unroll
+            for (int k = 0; k < KPT; ++k) {
+                const long long col = 4ll * tid + 1024ll * k;
+                if (col < d) {
+#pragma unroll
+                    for (int i = 0; i < RG; ++i) {
+                        if (rg + i < nr) {
+                            const float4 x = *reinterpret_cast<const float4 *>(Xb + (size_t)(rg + i) * d + col);
+                            part[i] += x.x * wv[k].x + x.y * wv[k].y + x.z * wv[k].z + x.w * wv[k].w;
+                        }
+                    }
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < RG; ++i) {
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) part[i] += __shfl_xor_sync(0xffffffffu, part[i], o);
+                if (lane == 0 && rg + i < nr) red[(rg + i) * 8 + warp] = part[i];
+            }
+        }
+        __syncthreads();
+        if (tid < nr) {
+            float r = -yv;
+#pragma unroll
+            for (int w8 = 0; w8 < 8; ++w8) r += red[tid * 8 + w8];
+            rfin[tid] = r;
+        }
+        __syncthreads();
+        // pass B: acc += r[row] * X_b[row, cols]
+        for (int row = 0; row < nr; ++row) {
+            const float r = rfin[row];
+#pragma unroll
+            for (int k = 0; k < KPT; ++k) {
+                const long long col = 4ll * tid + 1024ll * k;
+                if (col < d) {
+                    const float4 x = *reinterpret_cast<const float4 *>(Xb + (size_t)row * d + col);
+                    acc[k].x += r * x.x; acc[k].y += r * x.y; acc[k].z += r * x.z; acc[k].w += r * x.w;
+                }
+            }
+        }
+        ++done;
+    }
+    if (done < nblocks) {
+        // a wait gave up: report it and wait (bounded) for the copies still in flight; the cluster
+        // reduction below still runs so that the other CTAs of the cluster are not left waiting
+        if (tid == 0) {
+            flags[1] = 1;
+            atomicExch(a.status, 1);
+            for (int b = done; b < issued; ++b) mbar_wait(&full[b % S], (uint32_t)((b / S) & 1), &flags[0]);
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int k = 0; k < KPT; ++k) {
+        const long long col = 4ll * tid + 1024ll * k;
+        if (col < d) *reinterpret_cast<float4 *>(gpart + col) = acc[k];
+    }
+    cluster.sync();
+    {
+        const unsigned C = cluster.num_blocks(), rank = cluster.block_rank();
+        const long long vecs = d / 4;
+        const long long per = (vecs + C - 1) / C;
+        for (long long v = (long long)rank * per + tid; v < min(vecs, (long long)(rank + 1) * per); v += blockDim.x) {
+            float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (unsigned c = 0; c < C; ++c) {
+                const float4 x = *reinterpret_cast<const float4 *>(cluster.map_shared_rank(gpart, c) + v * 4);
+                sum.x += x.x; sum.y += x.y; sum.z += x.z; sum.w += x.w;
+            }
+            *reinterpret_cast<float4 *>(a.G + (size_t)item * d + v * 4) = sum;
+        }
+    }
+    cluster.sync();  // nobody leaves while its shared memory may still be read
+}
+
+// ------------------------------------------------------------------------------------------------
 // host side: launch wrappers
 // ------------------------------------------------------------------------------------------------
 
@@ -1115,9 +1296,9 @@ cudaError_t launch_decode(const void *M_child, const void *E_parent, const void 
     return err;
 }
 
-cudaError_t launch_partial_gradients(const float *X, const float *y, const float *w, const int32_t *part,
-                                     int items, int rows, int64_t d, float *resid, float *G,
-                                     cudaStream_t stream, int64_t *launches) {
+cudaError_t launch_partial_gradients_two_pass(const float *X, const float *y, const float *w, const int32_t *part,
+                                              int items, int rows, int64_t d, float *resid, float *G,
+                                              cudaStream_t stream, int64_t *launches) {
     const bool v4 = d % 4 == 0 && aligned16(X) && aligned16(w) && aligned16(G);
     const long long total_rows = (long long)items * rows;
     const long long want_blocks = (total_rows + 7) / 8;  // 8 warps per block
@@ -1135,6 +1316,55 @@ cudaError_t launch_partial_gradients(const float *X, const float *y, const float
         cr_xt_r_kernel<1><<<grid, 128, 0, stream>>>(X, part, resid, rows, d, G);
     }
     err = cudaGetLastError();
+    if (err == cudaSuccess) ++*launches;
+    return err;
+}
+
+template <int KPT>
+static cudaError_t run_partial_fused(const PgArgs &pa, int csplit, int items, size_t smem, cudaStream_t stream) {
+    auto kern = cr_partial_fused_kernel<KPT>;
+    cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (err != cudaSuccess) return err;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)csplit, (unsigned)items, 1);
+    cfg.blockDim = dim3(256, 1, 1);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)csplit;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kern, pa);
+}
+
+bool partial_fused_eligible(const float *X, const float *w, const float *G, int64_t d, int items) {
+    return d % 4 == 0 && d <= 8192 && aligned16(X) && aligned16(w) && aligned16(G) && items <= 65535;
+}
+
+cudaError_t launch_partial_gradients_fused(const float *X, const float *y, const float *w, const int32_t *part,
+                                           int items, int rows, int64_t d, float *G, int *status,
+                                           const DeviceInfo &dev, cudaStream_t stream, int64_t *launches) {
+    // blocks of about 32 KB, four buffers (three copies in flight: ~100 KB per SM)
+    const int RB = (int)std::max<int64_t>(1, std::min<int64_t>(32, (32 * 1024) / (d * 4)));
+    const int stages = 4;
+    // rows of one item are split over a cluster of up to 8 CTAs, each with at least 4 blocks of work
+    int csplit = 1;
+    while (csplit < 8 && rows / (csplit * 2) >= 4 * RB) csplit *= 2;
+    const int rows_per_cta = (rows + csplit - 1) / csplit;
+    const size_t smem = (size_t)stages * RB * d * 4 + (size_t)d * 4 + (size_t)RB * 8 * 4 + (size_t)((RB + 3) & ~3) * 4 +
+                        (size_t)stages * 8 + 16;
+    if (smem > (size_t)dev.smem_optin) return cudaErrorInvalidConfiguration;
+    PgArgs pa;
+    pa.X = X; pa.y = y; pa.w = w; pa.part = part; pa.G = G; pa.rows = rows; pa.rows_per_cta = rows_per_cta;
+    pa.RB = RB; pa.stages = stages; pa.d = d; pa.status = status;
+    cudaError_t err;
+    if (d <= 1024) err = run_partial_fused<1>(pa, csplit, items, smem, stream);
+    else if (d <= 2048) err = run_partial_fused<2>(pa, csplit, items, smem, stream);
+    else if (d <= 4096) err = run_partial_fused<4>(pa, csplit, items, smem, stream);
+    else err = run_partial_fused<8>(pa, csplit, items, smem, stream);
     if (err == cudaSuccess) ++*launches;
     return err;
 }

@@ -80,9 +80,16 @@ cudaError_t launch_decode(const void *M_child, const void *E_parent, const void 
                           cudaStream_t stream, int64_t *launches);
 
 // Partial gradients of linear regression, two passes over X: residuals r = X_p w - y_p into `resid`
-// ([items][rows]), then G[item][:] = X_p^T r.  part[item] is the partition of slot `item`.
-cudaError_t launch_partial_gradients(const float *X, const float *y, const float *w, const int32_t *part,
-                                     int items, int rows, int64_t d, float *resid, float *G,
-                                     cudaStream_t stream, int64_t *launches);
+// ([items][rows]), then G[item][:] = X_p^T r.  part[item] is the partition of slot `item`.  Any d.
+cudaError_t launch_partial_gradients_two_pass(const float *X, const float *y, const float *w, const int32_t *part,
+                                              int items, int rows, int64_t d, float *resid, float *G,
+                                              cudaStream_t stream, int64_t *launches);
+
+// The same in one pass over X (row blocks staged in shared memory, cluster reduction), no scratch;
+// needs d % 4 == 0, d <= 8192 and 16-byte aligned X, w, G (partial_fused_eligible).
+bool partial_fused_eligible(const float *X, const float *w, const float *G, int64_t d, int items);
+cudaError_t launch_partial_gradients_fused(const float *X, const float *y, const float *w, const int32_t *part,
+                                           int items, int rows, int64_t d, float *G, int *status,
+                                           const DeviceInfo &dev, cudaStream_t stream, int64_t *launches);
 
 }  // namespace cr
