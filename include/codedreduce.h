@@ -223,6 +223,12 @@ cr_status_t cr_aggregate_bytes(const cr_plan_t *plan, const uint32_t *masks_host
 cr_status_t cr_plan_tune(cr_plan_t *plan, int32_t consumer_warps, int32_t stages, int32_t ctas_per_sm,
                          int32_t rows_per_box);
 
+/* Launch shape of the one-pass partial-gradient kernel; 0 keeps the built-in choice for that field.
+ * block_kb = KB of X per staged row block (1..128), stages = row-block buffers per CTA (2..8),
+ * cluster = CTAs that share one (node, slot) item (1, 2, 4 or 8).  A shape that does not fit shared
+ * memory makes cr_partial_gradients return CR_ERR_CUDA. */
+cr_status_t cr_plan_tune_gradients(cr_plan_t *plan, int32_t block_kb, int32_t stages, int32_t cluster);
+
 /* Kernel launches enqueued by this plan's device calls so far. */
 int64_t cr_plan_launch_count(const cr_plan_t *plan);
 

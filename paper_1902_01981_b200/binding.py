@@ -73,6 +73,7 @@ _SIGNATURES = {
                                     C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
     "cr_aggregate_bytes": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(C.c_int64), C.POINTER(C.c_int32)]),
     "cr_plan_tune": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32]),
+    "cr_plan_tune_gradients": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32]),
     "cr_plan_launch_count": (C.c_int64, [C.c_void_p]),
 }
 
@@ -210,6 +211,10 @@ def cr_plan_device_status(plan: int) -> int:
 def cr_plan_tune(plan: int, consumer_warps: int = 0, stages: int = 0, ctas_per_sm: int = 0,
                  rows_per_box: int = 0) -> None:
     _check(lib().cr_plan_tune(plan, consumer_warps, stages, ctas_per_sm, rows_per_box), "cr_plan_tune")
+
+
+def cr_plan_tune_gradients(plan: int, block_kb: int = 0, stages: int = 0, cluster: int = 0) -> None:
+    _check(lib().cr_plan_tune_gradients(plan, block_kb, stages, cluster), "cr_plan_tune_gradients")
 
 
 # ------------------------------------------------------------------ device work

@@ -268,6 +268,13 @@ cr_status_t cr_plan_tune(cr_plan_t *plan, int32_t consumer_warps, int32_t stages
     return CR_OK;
 }
 
+cr_status_t cr_plan_tune_gradients(cr_plan_t *plan, int32_t block_kb, int32_t stages, int32_t cluster) {
+    if (!plan || block_kb < 0 || block_kb > 128 || stages < 0 || stages == 1 || stages > 8) return CR_ERR_INVALID_ARG;
+    if (cluster != 0 && cluster != 1 && cluster != 2 && cluster != 4 && cluster != 8) return CR_ERR_INVALID_ARG;
+    plan->tune.pg_block_kb = block_kb; plan->tune.pg_stages = stages; plan->tune.pg_cluster = cluster;
+    return CR_OK;
+}
+
 cr_status_t cr_plan_get_B(const cr_plan_t *plan, int32_t level, double *B, double *kappa, uint64_t *sub_seed) {
     if (!plan || !B || level < 0 || level >= plan->hp.L) return CR_ERR_INVALID_ARG;
     std::copy(plan->hp.B[level].begin(), plan->hp.B[level].end(), B);
@@ -341,7 +348,8 @@ cr_status_t cr_partial_gradients(cr_plan_t *plan, const float *X, const float *y
     if (cr::partial_fused_eligible(X, w, G_slots, plan->hp.d, items)) {
         // one pass over X, no scratch
         e = cr::launch_partial_gradients_fused(X, y, w, plan->d_part, items, rows, plan->hp.d, G_slots, plan->d_status,
-                                               plan->dev, reinterpret_cast<cudaStream_t>(stream), &plan->launches);
+                                               plan->dev, plan->tune, reinterpret_cast<cudaStream_t>(stream),
+                                               &plan->launches);
     } else {
         if (!workspace || workspace_bytes < cr_partial_gradients_workspace_bytes(plan, rows)) return CR_ERR_OOM;
         e = cr::launch_partial_gradients_two_pass(X, y, w, plan->d_part, items, rows, plan->hp.d,

@@ -23,6 +23,9 @@ struct Tuning {
     int stages = 0;       // depth of the shared-memory ring
     int ctas_per_sm = 0;  // persistent CTAs per SM (batch kernel, always one CTA per SM: loader warps, 4 or 6)
     int rows = 0;         // slot rows per TMA box (must divide m)
+    int pg_block_kb = 0;  // partial gradients: KB of X per staged row block
+    int pg_stages = 0;    // partial gradients: row-block buffers per CTA
+    int pg_cluster = 0;   // partial gradients: CTAs per (node, slot) item (1, 2, 4 or 8)
 };
 
 struct DeviceInfo {
@@ -90,6 +93,7 @@ cudaError_t launch_partial_gradients_two_pass(const float *X, const float *y, co
 bool partial_fused_eligible(const float *X, const float *w, const float *G, int64_t d, int items);
 cudaError_t launch_partial_gradients_fused(const float *X, const float *y, const float *w, const int32_t *part,
                                            int items, int rows, int64_t d, float *G, int *status,
-                                           const DeviceInfo &dev, cudaStream_t stream, int64_t *launches);
+                                           const DeviceInfo &dev, const Tuning &tune, cudaStream_t stream,
+                                           int64_t *launches);
 
 }  // namespace cr
