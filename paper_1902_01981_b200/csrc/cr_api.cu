@@ -503,6 +503,30 @@ cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *m
         return aggregate_unfused(plan, G_slots, masks_host, batch, g_out, (flags & CR_AGG_ALL_NODES) != 0, workspace, ex, s);
     }
 
+    cr::AggArgs a;
+    a.G = G_slots; a.coeff = plan->d_coeff;
+    a.steps = nullptr; a.pat_off = nullptr; a.unodes = nullptr; a.wtab = nullptr;
+    a.host_steps = ex.steps.data();
+    a.n_wtab = (int)ex.wtab.size();
+    a.n_union = (int)ex.unodes.size(); a.batch = batch; a.total_steps = (int)ex.steps.size();
+    a.m = hp.m; a.L = hp.L; a.d = hp.d; a.rows_total = (int64_t)hp.N * hp.m; a.out = g_out;
+    a.shift = hp.dtype == CR_I32 ? hp.int_shift : 0; a.status = plan->d_status; a.is_int = hp.dtype == CR_I32;
+    a.same_shape = 1;
+    for (int b = 1; b < batch && a.same_shape; ++b) {
+        const auto &p0 = ex.per_pattern[0], &pb = ex.per_pattern[b];
+        if (pb.size() != p0.size()) { a.same_shape = 0; break; }
+        for (size_t k = 0; k < p0.size(); ++k)
+            if (pb[k].layer != p0[k].layer) { a.same_shape = 0; break; }
+    }
+
+    // A single short pattern needs no staging: its schedule travels in the kernel parameters.
+    if (variant == CR_AGG_FUSED && batch == 1 && a.total_steps <= cr::inline_schedule_limit()) {
+        bool done = false;
+        cudaError_t e0 = cr::launch_fused_tma(a, plan->dev, plan->tune, plan->encode, s, &plan->launches, &done);
+        if (e0 != cudaSuccess) { note_cuda(e0, "cr_aggregate"); return CR_ERR_CUDA; }
+        if (done) return CR_OK;
+    }
+
     // staging layout: steps | pattern offsets | union nodes
     const size_t steps_bytes = align16(ex.steps.size() * sizeof(cr::Step));
     const size_t off_bytes = align16(ex.pat_off.size() * 4);
@@ -519,23 +543,11 @@ cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *m
     st = stage_commit(slot, total, s);
     if (st != CR_OK) return st;
 
-    cr::AggArgs a;
-    a.G = G_slots; a.coeff = plan->d_coeff;
     a.steps = reinterpret_cast<const cr::Step *>(slot->dev);
     a.pat_off = reinterpret_cast<const int32_t *>(slot->dev + steps_bytes);
     a.unodes = reinterpret_cast<const int32_t *>(slot->dev + steps_bytes + off_bytes);
     a.wtab = reinterpret_cast<const uint32_t *>(slot->dev + steps_bytes + off_bytes + nodes_bytes);
-    a.n_wtab = (int)ex.wtab.size();
-    a.n_union = (int)ex.unodes.size(); a.batch = batch; a.total_steps = (int)ex.steps.size();
-    a.m = hp.m; a.L = hp.L; a.d = hp.d; a.rows_total = (int64_t)hp.N * hp.m; a.out = g_out;
-    a.shift = hp.dtype == CR_I32 ? hp.int_shift : 0; a.status = plan->d_status; a.is_int = hp.dtype == CR_I32;
-    a.same_shape = 1;
-    for (int b = 1; b < batch && a.same_shape; ++b) {
-        const auto &p0 = ex.per_pattern[0], &pb = ex.per_pattern[b];
-        if (pb.size() != p0.size()) { a.same_shape = 0; break; }
-        for (size_t k = 0; k < p0.size(); ++k)
-            if (pb[k].layer != p0[k].layer) { a.same_shape = 0; break; }
-    }
+    a.host_steps = nullptr;
 
     cudaError_t e = cudaSuccess;
     if (variant == CR_AGG_UNCODED_SUM) {

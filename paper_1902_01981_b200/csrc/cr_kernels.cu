@@ -180,9 +180,15 @@ __device__ __forceinline__ void fold_many(T (&acc)[NP][LMAX][4], const T (&e)[NP
 // register recursion above.  Shared-memory layout of a stage: [box][R][BOXW] with BOXW = min(TILE,256)
 // (a TMA box is at most 256 elements wide).
 
+// Schedules of at most kInlineSteps entries travel inside the kernel parameters (constant bank), which
+// saves the host-to-device copy in front of short launches.
+constexpr int kInlineSteps = 96;
+
 struct FusedArgs {
     const void *coeff;
-    const Step *steps;
+    const Step *steps;      // device schedule, unless n_inline > 0
+    int n_inline;           // entries of steps_inline in use (0: read `steps`)
+    Step steps_inline[kInlineSteps];
     int n_steps;
     int m, R, cpn, stages;
     long long d;
@@ -230,7 +236,7 @@ cr_fused_tma_kernel(const __grid_constant__ CUtensorMap tmap, const FusedArgs a)
             for (long long tile = blockIdx.x; tile < a.ntiles && ok; tile += gridDim.x) {
                 const int x0 = (int)(tile * TILE);
                 for (int k = 0; k < a.n_steps && ok; ++k) {
-                    const int row0 = __ldg(&a.steps[k].node) * a.m;
+                    const int row0 = (a.n_inline ? a.steps_inline[k].node : __ldg(&a.steps[k].node)) * a.m;
                     for (int c = 0; c < a.cpn; ++c) {
                         if (!mbar_wait(&empty[stage], phase ^ 1u, &flags[0])) { ok = false; break; }
                         mbar_expect_tx(&full[stage], stage_bytes);
@@ -266,7 +272,11 @@ cr_fused_tma_kernel(const __grid_constant__ CUtensorMap tmap, const FusedArgs a)
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
-        Step st_next = load_step(&a.steps[0]);
+        auto step_at = [&](int k) {
+            if (a.n_inline) { Step t = a.steps_inline[k]; t.layer &= 0xff; return t; }
+            return load_step(&a.steps[k]);
+        };
+        Step st_next = step_at(0);
         T cj_next[kMaxBoxRows];
         {
             const T *cf = coeff + (size_t)st_next.node * a.m;
@@ -285,7 +295,7 @@ cr_fused_tma_kernel(const __grid_constant__ CUtensorMap tmap, const FusedArgs a)
                     {
                         int kn = k, cn = c + 1;
                         if (cn == a.cpn) { cn = 0; kn = k + 1 == a.n_steps ? 0 : k + 1; }
-                        st_next = load_step(&a.steps[kn]);
+                        st_next = step_at(kn);
                         const T *cf = coeff + (size_t)st_next.node * a.m + cn * R;
 #pragma unroll
                         for (int j = 0; j < kMaxBoxRows; ++j) cj_next[j] = j < R ? __ldg(cf + j) : T(0);
@@ -1019,6 +1029,8 @@ bool tma_eligible(const AggArgs &a) {
            a.rows_total < (1ll << 31);
 }
 
+int inline_schedule_limit() { return kInlineSteps; }
+
 static bool vec4_ok(const void *G, const void *out, int64_t d) { return d % 4 == 0 && aligned16(G) && aligned16(out); }
 
 static int pick_lmax(int L) { return L <= 2 ? 2 : (L <= 4 ? 4 : 8); }
@@ -1099,6 +1111,13 @@ cudaError_t launch_fused_tma(const AggArgs &a, const DeviceInfo &dev, const Tuni
     if (make_map(encode, &map, a, boxw, R) != CUDA_SUCCESS) return cudaSuccess;
 
     FusedArgs fa;
+    fa.n_inline = 0;
+    if (a.host_steps && a.total_steps <= kInlineSteps) {
+        fa.n_inline = a.total_steps;
+        for (int k = 0; k < a.total_steps; ++k) fa.steps_inline[k] = a.host_steps[k];
+    } else if (!a.steps) {
+        return cudaSuccess;  // no staged schedule and too long to inline: caller stages it and retries
+    }
     fa.coeff = a.coeff; fa.steps = a.steps; fa.n_steps = a.total_steps; fa.m = a.m; fa.R = R; fa.cpn = a.m / R;
     fa.stages = stages; fa.d = a.d; fa.ntiles = (a.d + tile - 1) / tile; fa.out = a.out; fa.shift = a.shift;
     fa.status = a.status;

@@ -37,7 +37,9 @@ struct DeviceInfo {
 struct AggArgs {
     const void *G;        // [N*m][d]
     const void *coeff;    // [N*m] element type T
-    const Step *steps;    // device: all patterns' steps, concatenated
+    const Step *steps;    // device: all patterns' steps, concatenated (may be null for launch_fused_tma
+                          // when host_steps is given and short enough to travel in the kernel parameters)
+    const Step *host_steps;  // host copy of the same entries, or null
     const int32_t *pat_off;  // device [batch+1]: pattern b owns steps pat_off[b] .. pat_off[b+1]-1
     const int32_t *unodes;   // device [n_union]: union of used nodes (batch kernel)
     const uint32_t *wtab;    // device [n_wtab]: distinct weight bit patterns of the batch (n_wtab = 0: none)
@@ -63,6 +65,8 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 // Each returns cudaSuccess or the first CUDA error; *launches is incremented per kernel launched.
 // `can_tma` tells whether d and the pointers meet the TMA alignment rules.
 bool tma_eligible(const AggArgs &a);
+// Longest single-pattern schedule that launch_fused_tma can pass inside the kernel parameters.
+int inline_schedule_limit();
 
 cudaError_t launch_fused_tma(const AggArgs &a, const DeviceInfo &dev, const Tuning &tune, EncodeTiledFn encode,
                              cudaStream_t stream, int64_t *launches, bool *done);
