@@ -873,12 +873,12 @@ __device__ __forceinline__ void bulk_load_1d(void *smem_dst, const void *gsrc, u
         : "memory");
 }
 
-template <int KPT>
+// RG = rows handled together in pass A (1, 2 or 4; at most the rows of a block).
+template <int KPT, int RG>
 __global__ void __launch_bounds__(256, 2)
 cr_partial_fused_kernel(const PgArgs a) {
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
-    constexpr int RG = 4;  // rows handled together in pass A
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const long long d = a.d;
@@ -1339,9 +1339,9 @@ cudaError_t launch_partial_gradients_two_pass(const float *X, const float *y, co
     return err;
 }
 
-template <int KPT>
-static cudaError_t run_partial_fused(const PgArgs &pa, int csplit, int items, size_t smem, cudaStream_t stream) {
-    auto kern = cr_partial_fused_kernel<KPT>;
+template <int KPT, int RG>
+static cudaError_t run_partial_fused_rg(const PgArgs &pa, int csplit, int items, size_t smem, cudaStream_t stream) {
+    auto kern = cr_partial_fused_kernel<KPT, RG>;
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
     cudaLaunchConfig_t cfg = {};
@@ -1359,6 +1359,13 @@ static cudaError_t run_partial_fused(const PgArgs &pa, int csplit, int items, si
     return cudaLaunchKernelEx(&cfg, kern, pa);
 }
 
+template <int KPT>
+static cudaError_t run_partial_fused(const PgArgs &pa, int csplit, int items, size_t smem, cudaStream_t stream) {
+    if (pa.RB >= 4) return run_partial_fused_rg<KPT, 4>(pa, csplit, items, smem, stream);
+    if (pa.RB >= 2) return run_partial_fused_rg<KPT, 2>(pa, csplit, items, smem, stream);
+    return run_partial_fused_rg<KPT, 1>(pa, csplit, items, smem, stream);
+}
+
 bool partial_fused_eligible(const float *X, const float *w, const float *G, int64_t d, int items) {
     return d % 4 == 0 && d <= 8192 && aligned16(X) && aligned16(w) && aligned16(G) && items <= 65535;
 }
@@ -1367,14 +1374,15 @@ cudaError_t launch_partial_gradients_fused(const float *X, const float *y, const
                                            int items, int rows, int64_t d, float *G, int *status,
                                            const DeviceInfo &dev, const Tuning &tune, cudaStream_t stream,
                                            int64_t *launches) {
-    // Measured on B200 (d = 4096, rows = 2048): blocks of 32 KB with three buffers per CTA leave room
-    // for two CTAs per SM, which hide each other's reduction latency: 5.8 TB/s against 3.1 TB/s for one
-    // CTA per SM with four buffers; smaller or larger blocks lose 20-40 %.
-    const int block_kb = tune.pg_block_kb ? tune.pg_block_kb : 32;
-    const int RB = (int)std::max<int64_t>(1, std::min<int64_t>(32, ((int64_t)block_kb * 1024) / (d * 4)));
-    int stages = tune.pg_stages ? tune.pg_stages : 3;
-    if (!tune.pg_stages && (size_t)stages * RB * d * 4 + (size_t)d * 4 + 2048 > ((size_t)dev.smem_per_sm - 2048) / 2 - 1024)
-        stages = 2;
+    // Measured on B200 (d = 4096, rows = 2048): two CTAs per SM hide each other's reduction latency
+    // (one CTA per SM with four buffers: 3.1 TB/s), and with two buffers per CTA the largest row block
+    // that still lets two CTAs share an SM is best (32 KB: 6.2 TB/s, 48 KB: 6.7 TB/s; 64 KB, which
+    // leaves one CTA per SM: 4.5 TB/s).
+    const size_t per_cta = (size_t)dev.smem_per_sm / 2 - 1024;
+    const int stages = tune.pg_stages ? tune.pg_stages : 2;
+    int64_t rb = tune.pg_block_kb ? ((int64_t)tune.pg_block_kb * 1024) / (d * 4)
+                                  : ((int64_t)per_cta - d * 4 - 512) / ((int64_t)stages * d * 4);
+    const int RB = (int)std::max<int64_t>(1, std::min<int64_t>(32, rb));
     // rows of one item are split over a cluster of up to 8 CTAs, each with at least 4 blocks of work
     int csplit = 1;
     while (csplit < 8 && rows / (csplit * 2) >= 4 * RB) csplit *= 2;
