@@ -94,8 +94,17 @@ enum {
     CR_AGG_UNFUSED = 2,      /* cr_encode + cr_decode per level through the workspace */
     CR_AGG_UNCODED_SUM = 3,  /* comparator: plain sum of the same used slots, all weights 1 */
     CR_AGG_VARIANT_MASK = 0xff,
-    CR_AGG_ALL_NODES = 0x100 /* CR_AGG_UNFUSED only: encode and decode every node, not just used ones */
+    CR_AGG_ALL_NODES = 0x100, /* CR_AGG_UNFUSED only: encode and decode every node, not just used ones */
+    CR_AGG_FROM_CODED = 0x200 /* the first buffer is E [N][d] (coded gradients of cr_coded_gradients or cr_encode),
+                                 not G_slots: the encode step is skipped.  Not with CR_AGG_UNFUSED. */
 };
+
+/* Per-sample loss whose gradient the workers compute (Eq. (g) leaves the loss generic; the paper's
+ * experiments use linear regression on synthetic data and logistic regression on real data, Section V). */
+typedef enum {
+    CR_LOSS_SQUARED = 0,  /* 1/2 (x.w - y)^2        : gradient X^T (X w - y) */
+    CR_LOSS_LOGISTIC = 1  /* log(1+e^{x.w}) - y x.w : gradient X^T (sigmoid(X w) - y), labels y in {0,1} */
+} cr_loss_t;
 
 /* ---- plan: CR.Allocate + the gradient-coding tables (host work, once) ------------------------
  * cr_plan_create builds the tree indexing, the per-level encoding matrices B (Section II-C), the
@@ -153,6 +162,22 @@ size_t cr_partial_gradients_workspace_bytes(const cr_plan_t *plan, int32_t rows)
 cr_status_t cr_partial_gradients(cr_plan_t *plan, const float *X, const float *y, int32_t rows,
                                  const float *w, float *G_slots, void *workspace,
                                  size_t workspace_bytes, void *stream);
+
+/* The same pass for either loss (cr_partial_gradients is the CR_LOSS_SQUARED case). */
+cr_status_t cr_partial_gradients_loss(cr_plan_t *plan, int32_t loss, const float *X, const float *y, int32_t rows,
+                                      const float *w, float *G_slots, void *workspace, size_t workspace_bytes,
+                                      void *stream);
+
+/* ---- CR.Execute, "all nodes compute their local partial CODED gradients" in one step -----------
+ * E[v][:] = g_{D(l,i)} = sum_j c_{v,j} * X_p^T r_p with p the partition of slot j of node v
+ * (Section III-A: D(l,i) carries the combining coefficients along with its data points), r_p the
+ * residuals of `loss` at w.  The slot gradients are never written: each node's cluster of CTAs walks
+ * the rows of all its m slots and scales the residuals by the slot's coefficient.  X [P][rows][d],
+ * y [P][rows], w [d], E [N][d]: device pointers, fp32.  Needs d % 4 == 0, d <= 8192 and 16-byte
+ * aligned X, w, E (CR_ERR_INVALID_ARG otherwise: use cr_partial_gradients_loss + cr_encode).  Feed E
+ * to cr_aggregate with CR_AGG_FROM_CODED, or to cr_decode level by level.  CR_F32 plans only. */
+cr_status_t cr_coded_gradients(cr_plan_t *plan, int32_t loss, const float *X, const float *y, int32_t rows,
+                               const float *w, float *E, void *stream);
 
 /* ---- the same partial-gradient pass for callers that cannot allocate device memory ----------------
  * (No counterpart in the paper: this is a packaging variant of cr_partial_gradients.)

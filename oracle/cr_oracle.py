@@ -441,6 +441,21 @@ def loss_linreg(X: np.ndarray, y: np.ndarray, w: np.ndarray) -> float:
     return 0.5 * float(r @ r)
 
 
+def partial_gradient_logistic(X: np.ndarray, y: np.ndarray, w: np.ndarray) -> np.ndarray:
+    """Gradient of the logistic loss sum_i [log(1 + exp(x_i.w)) - y_i x_i.w] over the rows of one
+    partition (labels y in {0, 1}): X^T (sigmoid(X w) - y), the instance of Eq. (g) used in the
+    paper's real-data experiment (Section V).  Pinned by a central finite difference of the loss and by
+    the closed form at w = 0."""
+    X = np.asarray(X, dtype=np.float64)
+    z = X @ np.asarray(w, dtype=np.float64)
+    return X.T @ (1.0 / (1.0 + np.exp(-z)) - np.asarray(y, dtype=np.float64))
+
+
+def loss_logistic(X: np.ndarray, y: np.ndarray, w: np.ndarray) -> float:
+    z = np.asarray(X, dtype=np.float64) @ np.asarray(w, dtype=np.float64)
+    return float(np.sum(np.logaddexp(0.0, z) - np.asarray(y, dtype=np.float64) * z))
+
+
 def normalized_error_rate(w: np.ndarray, w_star: np.ndarray) -> float:
     """||w - w*||^2 / ||w*||^2 (Eq. NER)."""
     w = w.astype(np.float64)

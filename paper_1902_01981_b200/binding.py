@@ -23,6 +23,8 @@ CR_CODE_CYCLIC_RANDOM, CR_CODE_FRACTIONAL_REPETITION, CR_CODE_PAPER_3_1, CR_CODE
 CR_F32, CR_I32 = 0, 1
 CR_AGG_FUSED, CR_AGG_FUSED_LDG, CR_AGG_UNFUSED, CR_AGG_UNCODED_SUM = 0, 1, 2, 3
 CR_AGG_ALL_NODES = 0x100
+CR_AGG_FROM_CODED = 0x200
+CR_LOSS_SQUARED, CR_LOSS_LOGISTIC = 0, 1
 
 
 class cr_plan_desc_t(C.Structure):
@@ -61,6 +63,10 @@ _SIGNATURES = {
     "cr_partial_gradients_workspace_bytes": (C.c_size_t, [C.c_void_p, C.c_int32]),
     "cr_partial_gradients": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
                                        C.c_void_p, C.c_size_t, C.c_void_p]),
+    "cr_partial_gradients_loss": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
+                                            C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
+    "cr_coded_gradients": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
+                                     C.c_void_p]),
     "cr_partial_gradients_static_capacity": (C.c_size_t, []),
     "cr_partial_gradients_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
                                               C.c_void_p]),
@@ -228,6 +234,19 @@ def cr_partial_gradients(plan: int, X, y, rows: int, w, G_slots, workspace, stre
                                       _dev_ptr(workspace),
                                       0 if workspace is None else workspace.numel() * workspace.element_size(),
                                       _stream_ptr(stream)), "cr_partial_gradients")
+
+
+def cr_partial_gradients_loss(plan: int, loss: int, X, y, rows: int, w, G_slots, workspace, stream=None) -> None:
+    _check(lib().cr_partial_gradients_loss(plan, loss, _dev_ptr(X), _dev_ptr(y), rows, _dev_ptr(w), _dev_ptr(G_slots),
+                                           _dev_ptr(workspace),
+                                           0 if workspace is None else workspace.numel() * workspace.element_size(),
+                                           _stream_ptr(stream)), "cr_partial_gradients_loss")
+
+
+def cr_coded_gradients(plan: int, loss: int, X, y, rows: int, w, E, stream=None) -> None:
+    """E[v] = coded gradient of node v (its slots' gradients combined with their coefficients)."""
+    _check(lib().cr_coded_gradients(plan, loss, _dev_ptr(X), _dev_ptr(y), rows, _dev_ptr(w), _dev_ptr(E),
+                                    _stream_ptr(stream)), "cr_coded_gradients")
 
 
 def cr_partial_gradients_static_capacity() -> int:

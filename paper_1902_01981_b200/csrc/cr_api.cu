@@ -49,6 +49,7 @@ struct cr_plan {
     cr::HostPlan hp;
     int device = -1;
     void *d_coeff = nullptr;     // [N*m] float or int32
+    void *d_ones = nullptr;      // [N] the value 1 in the plan's element type (aggregation of coded gradients)
     int32_t *d_part = nullptr;   // [N*m]
     int *d_status = nullptr;
     cr::DeviceInfo dev;
@@ -193,6 +194,7 @@ cr_status_t cr_plan_destroy(cr_plan_t *plan) {
             if (s.dev) cudaFree(s.dev);
         }
         if (plan->d_coeff) cudaFree(plan->d_coeff);
+        if (plan->d_ones) cudaFree(plan->d_ones);
         if (plan->d_part) cudaFree(plan->d_part);
         if (plan->d_status) cudaFree(plan->d_status);
     }
@@ -236,6 +238,11 @@ cr_status_t cr_plan_create(const cr_plan_desc_t *desc, cr_plan_t **out) {
         CR_CUDA_P(cudaMalloc(reinterpret_cast<void **>(&p->d_part), slots * 4));
         CR_CUDA_P(cudaMalloc(reinterpret_cast<void **>(&p->d_status), sizeof(int)));
         CR_CUDA_P(cudaMemcpy(p->d_coeff, coeff.data(), slots * 4, cudaMemcpyHostToDevice));
+        {
+            std::vector<uint32_t> ones((size_t)p->hp.N, weight_bits(p->hp, 1.0));
+            CR_CUDA_P(cudaMalloc(&p->d_ones, ones.size() * 4));
+            CR_CUDA_P(cudaMemcpy(p->d_ones, ones.data(), ones.size() * 4, cudaMemcpyHostToDevice));
+        }
         CR_CUDA_P(cudaMemcpy(p->d_part, part.data(), slots * 4, cudaMemcpyHostToDevice));
         CR_CUDA_P(cudaMemset(p->d_status, 0, sizeof(int)));
         // cuTensorMapEncodeTiled through the runtime, so that the library needs no link to libcuda
@@ -337,26 +344,51 @@ size_t cr_partial_gradients_workspace_bytes(const cr_plan_t *plan, int32_t rows)
     return (size_t)plan->hp.N * plan->hp.m * (size_t)rows * sizeof(float);
 }
 
-cr_status_t cr_partial_gradients(cr_plan_t *plan, const float *X, const float *y, int32_t rows, const float *w,
-                                 float *G_slots, void *workspace, size_t workspace_bytes, void *stream) {
+cr_status_t cr_partial_gradients_loss(cr_plan_t *plan, int32_t loss, const float *X, const float *y, int32_t rows,
+                                      const float *w, float *G_slots, void *workspace, size_t workspace_bytes,
+                                      void *stream) {
     cr_status_t st = check_device_plan(plan);
     if (st != CR_OK) return st;
-    if (!X || !y || !w || !G_slots || rows < 1) return CR_ERR_INVALID_ARG;
+    if (!X || !y || !w || !G_slots || rows < 1 || (loss != CR_LOSS_SQUARED && loss != CR_LOSS_LOGISTIC)) return CR_ERR_INVALID_ARG;
     if (plan->hp.dtype != CR_F32) return CR_ERR_DTYPE;
     const int items = plan->hp.N * plan->hp.m;
     cudaError_t e;
     if (cr::partial_fused_eligible(X, w, G_slots, plan->hp.d, items)) {
         // one pass over X, no scratch
-        e = cr::launch_partial_gradients_fused(X, y, w, plan->d_part, items, rows, plan->hp.d, G_slots, plan->d_status,
-                                               plan->dev, plan->tune, reinterpret_cast<cudaStream_t>(stream),
-                                               &plan->launches);
+        e = cr::launch_partial_gradients_fused(X, y, w, plan->d_part, nullptr, items, 1, rows, plan->hp.d, G_slots, loss,
+                                               plan->d_status, plan->dev, plan->tune,
+                                               reinterpret_cast<cudaStream_t>(stream), &plan->launches);
     } else {
         if (!workspace || workspace_bytes < cr_partial_gradients_workspace_bytes(plan, rows)) return CR_ERR_OOM;
         e = cr::launch_partial_gradients_two_pass(X, y, w, plan->d_part, items, rows, plan->hp.d,
-                                                  reinterpret_cast<float *>(workspace), G_slots,
+                                                  reinterpret_cast<float *>(workspace), G_slots, loss,
                                                   reinterpret_cast<cudaStream_t>(stream), &plan->launches);
     }
     if (e != cudaSuccess) { note_cuda(e, "cr_partial_gradients"); return CR_ERR_CUDA; }
+    return CR_OK;
+}
+
+cr_status_t cr_partial_gradients(cr_plan_t *plan, const float *X, const float *y, int32_t rows, const float *w,
+                                 float *G_slots, void *workspace, size_t workspace_bytes, void *stream) {
+    return cr_partial_gradients_loss(plan, CR_LOSS_SQUARED, X, y, rows, w, G_slots, workspace, workspace_bytes, stream);
+}
+
+cr_status_t cr_coded_gradients(cr_plan_t *plan, int32_t loss, const float *X, const float *y, int32_t rows,
+                               const float *w, float *E, void *stream) {
+    cr_status_t st = check_device_plan(plan);
+    if (st != CR_OK) return st;
+    if (!X || !y || !w || !E || rows < 1 || (loss != CR_LOSS_SQUARED && loss != CR_LOSS_LOGISTIC)) return CR_ERR_INVALID_ARG;
+    if (plan->hp.dtype != CR_F32) return CR_ERR_DTYPE;
+    if (!cr::partial_fused_eligible(X, w, E, plan->hp.d, plan->hp.N)) {
+        std::snprintf(g_last_error, sizeof(g_last_error),
+                      "cr_coded_gradients needs d %% 4 == 0, d <= 8192 and 16-byte aligned X, w, E");
+        return CR_ERR_INVALID_ARG;
+    }
+    cudaError_t e = cr::launch_partial_gradients_fused(X, y, w, plan->d_part, reinterpret_cast<const float *>(plan->d_coeff),
+                                                       plan->hp.N, plan->hp.m, rows, plan->hp.d, E, loss, plan->d_status,
+                                                       plan->dev, plan->tune, reinterpret_cast<cudaStream_t>(stream),
+                                                       &plan->launches);
+    if (e != cudaSuccess) { note_cuda(e, "cr_coded_gradients"); return CR_ERR_CUDA; }
     return CR_OK;
 }
 
@@ -490,8 +522,10 @@ cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *m
     const cr::HostPlan &hp = plan->hp;
     if (!G_slots || !masks_host || !g_out || batch < 1 || batch > (1 << 16)) return CR_ERR_INVALID_ARG;
     const uint32_t variant = flags & CR_AGG_VARIANT_MASK;
-    if (variant > CR_AGG_UNCODED_SUM || (flags & ~(uint32_t)(CR_AGG_VARIANT_MASK | CR_AGG_ALL_NODES)) != 0) return CR_ERR_INVALID_ARG;
+    if (variant > CR_AGG_UNCODED_SUM || (flags & ~(uint32_t)(CR_AGG_VARIANT_MASK | CR_AGG_ALL_NODES | CR_AGG_FROM_CODED)) != 0)
+        return CR_ERR_INVALID_ARG;
     if ((flags & CR_AGG_ALL_NODES) && variant != CR_AGG_UNFUSED) return CR_ERR_INVALID_ARG;
+    if ((flags & CR_AGG_FROM_CODED) && variant == CR_AGG_UNFUSED) return CR_ERR_INVALID_ARG;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
 
     Expanded ex;
@@ -510,6 +544,10 @@ cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *m
     a.n_wtab = (int)ex.wtab.size();
     a.n_union = (int)ex.unodes.size(); a.batch = batch; a.total_steps = (int)ex.steps.size();
     a.m = hp.m; a.L = hp.L; a.d = hp.d; a.rows_total = (int64_t)hp.N * hp.m; a.out = g_out;
+    if (flags & CR_AGG_FROM_CODED) {
+        // the input is E [N][d]: one row per node, already combined with the slot coefficients
+        a.m = 1; a.coeff = plan->d_ones; a.rows_total = hp.N;
+    }
     a.shift = hp.dtype == CR_I32 ? hp.int_shift : 0; a.status = plan->d_status; a.is_int = hp.dtype == CR_I32;
     a.same_shape = 1;
     for (int b = 1; b < batch && a.same_shape; ++b) {
@@ -622,7 +660,7 @@ cr_status_t cr_partial_gradients_static(cr_plan_t *plan, const float *X, const f
         scratch = g_static_ptr[plan->device];
     }
     cudaError_t e = cr::launch_partial_gradients_two_pass(X, y, w, plan->d_part, plan->hp.N * plan->hp.m, rows, plan->hp.d,
-                                                 scratch, G_slots, reinterpret_cast<cudaStream_t>(stream),
+                                                 scratch, G_slots, CR_LOSS_SQUARED, reinterpret_cast<cudaStream_t>(stream),
                                                  &plan->launches);
     if (e != cudaSuccess) { note_cuda(e, "cr_partial_gradients_static"); return CR_ERR_CUDA; }
     return CR_OK;

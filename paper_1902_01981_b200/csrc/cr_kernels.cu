@@ -780,7 +780,7 @@ template <int V>
 __global__ void __launch_bounds__(256)
 cr_residual_kernel(const float *__restrict__ X, const float *__restrict__ y, const float *__restrict__ w,
                    const int32_t *__restrict__ part, long long total_rows, int rows, long long d,
-                   float *__restrict__ resid) {
+                   float *__restrict__ resid, int loss) {
     const int lane = threadIdx.x & 31;
     const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
     for (long long idx = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; idx < total_rows; idx += warps) {
@@ -800,7 +800,10 @@ cr_residual_kernel(const float *__restrict__ X, const float *__restrict__ y, con
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
-        if (lane == 0) resid[idx] = acc - __ldg(&y[(size_t)p * rows + row]);
+        if (lane == 0) {
+            if (loss == 1) acc = 1.f / (1.f + expf(-acc));   // logistic: sigmoid of the score
+            resid[idx] = acc - __ldg(&y[(size_t)p * rows + row]);
+        }
     }
 }
 
@@ -857,9 +860,12 @@ struct PgArgs {
     const float *y;
     const float *w;
     const int32_t *part;
-    float *G;
+    const float *coeff;   // [N*m] slot coefficients, or null: every slot weighs 1
+    float *G;             // [items][d]
     int rows;
-    int rows_per_cta;
+    int slots_per_item;   // 1: an item is one (node, slot); m: an item is a node and its slots are
+                          //    combined with their coefficients (the coded gradient of the node)
+    int loss;             // 0: squared loss, r = X w - y; 1: logistic loss, r = sigmoid(X w) - y
     int RB;
     int stages;
     long long d;
@@ -899,13 +905,17 @@ cr_partial_fused_kernel(const PgArgs a) {
     }
     __syncthreads();
 
+    // The item's work is a list of row blocks: slot by slot, `bps` blocks of RB rows per slot (a block
+    // never straddles two slots, whose partitions lie apart).  CTA c of the cluster takes a contiguous
+    // share of the list.
     const long long item = blockIdx.y;
-    const int p = __ldg(&a.part[item]);
-    const int r0 = min(a.rows, (int)blockIdx.x * a.rows_per_cta);
-    const int r1 = min(a.rows, r0 + a.rows_per_cta);
-    const int nblocks = (r1 - r0 + RB - 1) / RB;
-    const float *Xp = a.X + ((size_t)p * a.rows + r0) * d;
-    const float *yp = a.y + (size_t)p * a.rows + r0;
+    const int spi = a.slots_per_item;
+    const int bps = (a.rows + RB - 1) / RB;
+    const int total_blocks = spi * bps;
+    const int per_cta = (total_blocks + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int b0 = min(total_blocks, (int)blockIdx.x * per_cta);
+    const int nblocks = min(total_blocks, b0 + per_cta) - b0;
+    auto block_rows = [&](int blk) { return min(RB, a.rows - ((b0 + blk) % bps) * RB); };
 
     float4 wv[KPT], acc[KPT];
 #pragma unroll
@@ -917,19 +927,24 @@ cr_partial_fused_kernel(const PgArgs a) {
 
     int issued = 0;
     auto issue = [&](int blk) {  // thread 0 only
-        const int nr = min(RB, (r1 - r0) - blk * RB);
-        const uint32_t bytes = (uint32_t)((size_t)nr * d * sizeof(float));
+        const int vb = b0 + blk;
+        const int p = __ldg(&a.part[item * spi + vb / bps]);
+        const uint32_t bytes = (uint32_t)((size_t)block_rows(blk) * d * sizeof(float));
         mbar_expect_tx(&full[blk % S], bytes);
-        bulk_load_1d(ring + (size_t)(blk % S) * stage_elems, Xp + (size_t)blk * RB * d, bytes, &full[blk % S]);
+        bulk_load_1d(ring + (size_t)(blk % S) * stage_elems, a.X + ((size_t)p * a.rows + (size_t)(vb % bps) * RB) * d,
+                     bytes, &full[blk % S]);
     };
     if (tid == 0)
         for (; issued < nblocks && issued < S - 1; ++issued) issue(issued);
 
     int done = 0;
     for (int blk = 0; blk < nblocks; ++blk) {
-        const int nr = min(RB, (r1 - r0) - blk * RB);
-        // label of this thread's row, fetched before the wait so that its latency hides behind it
-        const float yv = tid < nr ? __ldg(yp + (size_t)blk * RB + tid) : 0.f;
+        const int nr = block_rows(blk);
+        // label of this thread's row and weight of the slot, fetched before the wait so that their
+        // latency hides behind it
+        const long long slot = item * spi + (b0 + blk) / bps;
+        const float yv = tid < nr ? __ldg(a.y + (size_t)__ldg(&a.part[slot]) * a.rows + (size_t)((b0 + blk) % bps) * RB + tid) : 0.f;
+        const float scale = a.coeff ? __ldg(&a.coeff[slot]) : 1.f;
         // all threads have left the previous block once this barrier is passed, so its buffer is free
         const int ok = __syncthreads_and(mbar_wait(&full[blk % S], (uint32_t)((blk / S) & 1), &flags[1]) ? 1 : 0);
         if (!ok) break;
@@ -966,10 +981,11 @@ cr_partial_fused_kernel(const PgArgs a) {
         }
         __syncthreads();
         if (tid < nr) {
-            float r = -yv;
+            float z = 0.f;
 #pragma unroll
-            for (int w8 = 0; w8 < 8; ++w8) r += red[tid * 8 + w8];
-            rfin[tid] = r;
+            for (int w8 = 0; w8 < 8; ++w8) z += red[tid * 8 + w8];
+            if (a.loss == 1) z = 1.f / (1.f + expf(-z));
+            rfin[tid] = scale * (z - yv);
         }
         __syncthreads();
         // pass B: acc += r[row] * X_b[row, cols]
@@ -1316,14 +1332,14 @@ cudaError_t launch_decode(const void *M_child, const void *E_parent, const void 
 }
 
 cudaError_t launch_partial_gradients_two_pass(const float *X, const float *y, const float *w, const int32_t *part,
-                                              int items, int rows, int64_t d, float *resid, float *G,
+                                              int items, int rows, int64_t d, float *resid, float *G, int loss,
                                               cudaStream_t stream, int64_t *launches) {
     const bool v4 = d % 4 == 0 && aligned16(X) && aligned16(w) && aligned16(G);
     const long long total_rows = (long long)items * rows;
     const long long want_blocks = (total_rows + 7) / 8;  // 8 warps per block
     const int blocks = (int)std::min<long long>(want_blocks, 148 * 32);
-    if (v4) cr_residual_kernel<4><<<blocks, 256, 0, stream>>>(X, y, w, part, total_rows, rows, d, resid);
-    else cr_residual_kernel<1><<<blocks, 256, 0, stream>>>(X, y, w, part, total_rows, rows, d, resid);
+    if (v4) cr_residual_kernel<4><<<blocks, 256, 0, stream>>>(X, y, w, part, total_rows, rows, d, resid, loss);
+    else cr_residual_kernel<1><<<blocks, 256, 0, stream>>>(X, y, w, part, total_rows, rows, d, resid, loss);
     cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) return err;
     ++*launches;
@@ -1371,9 +1387,9 @@ bool partial_fused_eligible(const float *X, const float *w, const float *G, int6
 }
 
 cudaError_t launch_partial_gradients_fused(const float *X, const float *y, const float *w, const int32_t *part,
-                                           int items, int rows, int64_t d, float *G, int *status,
-                                           const DeviceInfo &dev, const Tuning &tune, cudaStream_t stream,
-                                           int64_t *launches) {
+                                           const float *coeff, int items, int slots_per_item, int rows, int64_t d,
+                                           float *G, int loss, int *status, const DeviceInfo &dev,
+                                           const Tuning &tune, cudaStream_t stream, int64_t *launches) {
     // Measured on B200 (d = 4096, rows = 2048): two CTAs per SM hide each other's reduction latency
     // (one CTA per SM with four buffers: 3.1 TB/s), and with two buffers per CTA the largest row block
     // that still lets two CTAs share an SM is best (32 KB: 6.2 TB/s, 48 KB: 6.7 TB/s; 64 KB, which
@@ -1383,17 +1399,17 @@ cudaError_t launch_partial_gradients_fused(const float *X, const float *y, const
     int64_t rb = tune.pg_block_kb ? ((int64_t)tune.pg_block_kb * 1024) / (d * 4)
                                   : ((int64_t)per_cta - d * 4 - 512) / ((int64_t)stages * d * 4);
     const int RB = (int)std::max<int64_t>(1, std::min<int64_t>(32, rb));
-    // rows of one item are split over a cluster of up to 8 CTAs, each with at least 4 blocks of work
+    // the row blocks of one item are split over a cluster of up to 8 CTAs, each with at least 4 blocks
+    const int item_blocks = slots_per_item * ((rows + RB - 1) / RB);
     int csplit = 1;
-    while (csplit < 8 && rows / (csplit * 2) >= 4 * RB) csplit *= 2;
+    while (csplit < 8 && item_blocks / (csplit * 2) >= 4) csplit *= 2;
     if (tune.pg_cluster) csplit = tune.pg_cluster;
-    const int rows_per_cta = (rows + csplit - 1) / csplit;
     const size_t smem = (size_t)stages * RB * d * 4 + (size_t)d * 4 + (size_t)RB * 8 * 4 + (size_t)((RB + 3) & ~3) * 4 +
                         (size_t)stages * 8 + 16;
     if (smem > (size_t)dev.smem_optin) return cudaErrorInvalidConfiguration;
     PgArgs pa;
-    pa.X = X; pa.y = y; pa.w = w; pa.part = part; pa.G = G; pa.rows = rows; pa.rows_per_cta = rows_per_cta;
-    pa.RB = RB; pa.stages = stages; pa.d = d; pa.status = status;
+    pa.X = X; pa.y = y; pa.w = w; pa.part = part; pa.coeff = coeff; pa.G = G; pa.rows = rows;
+    pa.slots_per_item = slots_per_item; pa.loss = loss; pa.RB = RB; pa.stages = stages; pa.d = d; pa.status = status;
     cudaError_t err;
     if (d <= 1024) err = run_partial_fused<1>(pa, csplit, items, smem, stream);
     else if (d <= 2048) err = run_partial_fused<2>(pa, csplit, items, smem, stream);

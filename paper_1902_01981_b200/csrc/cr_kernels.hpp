@@ -88,16 +88,20 @@ cudaError_t launch_decode(const void *M_child, const void *E_parent, const void 
 
 // Partial gradients of linear regression, two passes over X: residuals r = X_p w - y_p into `resid`
 // ([items][rows]), then G[item][:] = X_p^T r.  part[item] is the partition of slot `item`.  Any d.
+// loss: 0 squared, 1 logistic (r = sigmoid(X_p w) - y_p).
 cudaError_t launch_partial_gradients_two_pass(const float *X, const float *y, const float *w, const int32_t *part,
-                                              int items, int rows, int64_t d, float *resid, float *G,
+                                              int items, int rows, int64_t d, float *resid, float *G, int loss,
                                               cudaStream_t stream, int64_t *launches);
 
 // The same in one pass over X (row blocks staged in shared memory, cluster reduction), no scratch;
 // needs d % 4 == 0, d <= 8192 and 16-byte aligned X, w, G (partial_fused_eligible).
 bool partial_fused_eligible(const float *X, const float *w, const float *G, int64_t d, int items);
+// slots_per_item = 1: G[item] for every (node, slot) item; slots_per_item = m with `coeff`: item = node,
+// G[node] = sum_j coeff[node*m+j] * (gradient of slot j), the node's coded gradient.
+// loss: 0 squared (r = X w - y), 1 logistic (r = sigmoid(X w) - y).
 cudaError_t launch_partial_gradients_fused(const float *X, const float *y, const float *w, const int32_t *part,
-                                           int items, int rows, int64_t d, float *G, int *status,
-                                           const DeviceInfo &dev, const Tuning &tune, cudaStream_t stream,
-                                           int64_t *launches);
+                                           const float *coeff, int items, int slots_per_item, int rows, int64_t d,
+                                           float *G, int loss, int *status, const DeviceInfo &dev,
+                                           const Tuning &tune, cudaStream_t stream, int64_t *launches);
 
 }  // namespace cr

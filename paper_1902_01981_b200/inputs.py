@@ -52,6 +52,22 @@ def linreg_partitions(P: int, rows: int, d: int, seed: int, x_std: float = 1.0,
     return X, y, w_star
 
 
+def logistic_partitions(P: int, rows: int, d: int, seed: int, x_std: float = 1.0):
+    """P partitions of a two-class data set: X [P, rows, d] fp32 ~ N(0, x_std^2), labels y [P, rows]
+    in {0, 1} drawn with probability 1 / (1 + exp(-x . w_star)), w_star [d] fp32 ~ N(0, I)."""
+    rng = _rng(seed)
+    w_star = rng.standard_normal(d, dtype=np.float32)
+    X = rng.standard_normal((P, rows, d), dtype=np.float32)
+    if x_std != 1.0:
+        X *= np.float32(x_std)
+    u = rng.random((P, rows))
+    y = np.empty((P, rows), dtype=np.float32)
+    for p in range(P):
+        z = X[p].astype(np.float64) @ w_star.astype(np.float64)
+        y[p] = (u[p] < 1.0 / (1.0 + np.exp(-z))).astype(np.float32)
+    return X, y, w_star
+
+
 def model_vector(d: int, seed: int) -> np.ndarray:
     """A start model w_0 ~ N(0, I), fp32."""
     return _rng(seed).standard_normal(d, dtype=np.float32)
@@ -110,6 +126,10 @@ CONFIGS = {
                  batch=1, exactly_s=True, seed=0, mask_seed=1),
     "cfg5": dict(n=3, L=4, s=1, P=195, d=1 << 22, code="printed_3_1", kind="aggregate", std=1.0, iters=5,
                  batch=64, exactly_s=False, seed=0, mask_seed=1, int_bound=1 << 10),
+    # shaped like the paper's logistic-regression run: 6552 samples, p = 5001 (padded to 5004 so that rows
+    # are 16-byte multiples), (12,2) tree with one straggler per group: 168 partitions of 39 samples
+    "cfg_logit": dict(n=12, L=2, s=1, P=168, d=5004, rows=39, code="cyclic", kind="logistic", x_std=1.0 / 70.0,
+                      iters=20, lr=0.5, seed=0, mask_seed=1),
     "cfg_rep": dict(n=4, L=2, s=1, P=24, d=1 << 20, code="repetition", kind="aggregate", std=1.0, iters=20,
                     batch=1, exactly_s=False, seed=0, mask_seed=1, int_bound=1 << 10),
 }

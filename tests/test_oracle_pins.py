@@ -328,6 +328,23 @@ def test_partial_gradient_is_the_derivative_of_the_loss():
     assert O.normalized_error_rate(w_star, w_star) == 0.0
 
 
+def test_logistic_gradient_is_the_derivative_of_the_loss():
+    X, y, _ = inputs.logistic_partitions(1, 15, 6, seed=4)
+    X, y = X[0].astype(np.float64), y[0].astype(np.float64)
+    assert set(np.unique(y)) <= {0.0, 1.0}
+    w = inputs.model_vector(6, seed=5).astype(np.float64)
+    g = O.partial_gradient_logistic(X, y, w)
+    h = 1e-5
+    for k in range(6):
+        e = np.zeros(6)
+        e[k] = h
+        fd = (O.loss_logistic(X, y, w + e) - O.loss_logistic(X, y, w - e)) / (2 * h)
+        assert abs(fd - g[k]) <= 1e-7 * max(1.0, abs(g[k]))
+    # at w = 0 every sample has probability 1/2
+    assert np.allclose(O.partial_gradient_logistic(X, y, np.zeros(6)), X.T @ (0.5 - y), atol=1e-13)
+    assert abs(O.loss_logistic(X, y, np.zeros(6)) - 15 * np.log(2.0)) < 1e-12
+
+
 # ------------------------------------------------- planted-mistake checks
 
 def test_pins_catch_planted_mistakes(monkeypatch):
