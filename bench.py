@@ -411,15 +411,22 @@ def run_linreg(args, cfg):
     n, L, s, P, d, rows = cfg["n"], cfg["L"], cfg["s"], cfg["P"], cfg["d"], cfg["rows"]
     plan = B.cr_plan_create(n, L, s, P, d, code=code_id, device=0)
     N, m, groups = B.cr_plan_num_nodes(plan), B.cr_plan_load(plan), B.cr_plan_num_groups(plan)
-    X, y, w_star = inputs.linreg_partitions(P, rows, d, cfg["seed"], cfg["x_std"], cfg["noise_std"])
+    logistic = cfg["kind"] == "logistic"
+    loss = B.CR_LOSS_LOGISTIC if logistic else B.CR_LOSS_SQUARED
+    if logistic:
+        X, y, w_star = inputs.logistic_partitions(P, rows, d, cfg["seed"], cfg["x_std"])
+    else:
+        X, y, w_star = inputs.linreg_partitions(P, rows, d, cfg["seed"], cfg["x_std"], cfg["noise_std"])
     X_dev, y_dev = torch.from_numpy(X).cuda(), torch.from_numpy(y).cuda()
+    E_coded = torch.zeros((N, d), device="cuda")
+    coded = args.coded and d % 4 == 0 and d <= 8192
     w_dev = torch.zeros(d, device="cuda")
     G_slots = torch.zeros((N, m, d), device="cuda")
     ws = torch.empty(max(16, B.cr_partial_gradients_workspace_bytes(plan, rows)), dtype=torch.uint8, device="cuda")
     out = torch.zeros((1, d), device="cuda")
     total = min(args.steps + args.warmup, 256)
     masks = inputs.straggler_masks(n, L, s, total, cfg.get("mask_seed", 1))
-    lr_eff = cfg["lr"] / P if args.workload == "cfg3" else cfg["lr"]
+    lr_eff = cfg["lr"] if args.workload == "cfg1" else cfg["lr"] / P
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if X.nbytes <= 126e6 else None
     stream = torch.cuda.current_stream()
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
@@ -427,10 +434,16 @@ def run_linreg(args, cfg):
     def step(i, events=None):
         if events:
             events[0].record(stream)
-        B.cr_partial_gradients(plan, X_dev, y_dev, rows, w_dev, G_slots, ws, stream)
+        if coded:
+            B.cr_coded_gradients(plan, loss, X_dev, y_dev, rows, w_dev, E_coded, stream)
+        else:
+            B.cr_partial_gradients_loss(plan, loss, X_dev, y_dev, rows, w_dev, G_slots, ws, stream)
         if events:
             events[1].record(stream)
-        B.cr_aggregate(plan, G_slots, masks[i % total], out, B.CR_AGG_FUSED, None, stream)
+        if coded:
+            B.cr_aggregate(plan, E_coded, masks[i % total], out, B.CR_AGG_FUSED | B.CR_AGG_FROM_CODED, None, stream)
+        else:
+            B.cr_aggregate(plan, G_slots, masks[i % total], out, B.CR_AGG_FUSED, None, stream)
         w_dev.sub_(out[0], alpha=lr_eff)
         if events:
             events[2].record(stream)
@@ -464,8 +477,10 @@ def run_linreg(args, cfg):
         "metric": METRIC, "value": step_bytes * args.steps / elapsed / 1e9, "unit": UNIT, "n_gpus": 1,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": elapsed / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": f"{args.workload}: linear regression n={n} L={L} s={s} P={P} rows={rows} d={d}, "
-                               "step = partial gradients of all N*m slots + fused aggregation + model update",
+        "config": {"workload": f"{args.workload}: {'logistic' if logistic else 'linear'} regression n={n} L={L} s={s} "
+                               f"P={P} rows={rows} d={d}, step = "
+                               + ("coded gradients of all N nodes (slot gradients never written)" if coded
+                                  else "partial gradients of all N*m slots") + " + fused aggregation + model update",
                    "l2": "inputs larger than L2 (no flush needed)" if flush is None else "L2 flushed between steps"},
         "iterations_per_s": args.steps / elapsed,
         "roofline": {"bound": "hbm", "kernel": "partial gradients", "achieved": achieved, "peak": peak, "unit": "GB/s",
@@ -489,6 +504,7 @@ def main():
     ap.add_argument("--dtype", default="f32", choices=["f32", "int32"])
     ap.add_argument("--d", type=int, default=0, help="override the gradient length (profiling on a small case)")
     ap.add_argument("--tune", default="", help="consumer_warps,stages,ctas_per_sm,rows_per_box (0 = auto)")
+    ap.add_argument("--coded", action="store_true", help="regression workloads: gradient + encode in one kernel")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extras", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -505,7 +521,7 @@ def main():
     world = int(os.environ.get("WORLD_SIZE", "1"))
     if args.gpus != world and world > 1:
         args.gpus = world
-    if cfg["kind"] == "linreg":
+    if cfg["kind"] in ("linreg", "logistic"):
         if args.impl == "reference":
             print(json.dumps({"impl": "reference", "unavailable": "the reference arm times aggregation workloads only"}))
         else:

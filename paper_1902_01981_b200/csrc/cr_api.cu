@@ -277,7 +277,7 @@ cr_status_t cr_plan_tune(cr_plan_t *plan, int32_t consumer_warps, int32_t stages
 
 cr_status_t cr_plan_tune_gradients(cr_plan_t *plan, int32_t block_kb, int32_t stages, int32_t cluster) {
     if (!plan || block_kb < 0 || block_kb > 128 || stages < 0 || stages == 1 || stages > 8) return CR_ERR_INVALID_ARG;
-    if (cluster != 0 && cluster != 1 && cluster != 2 && cluster != 4 && cluster != 8) return CR_ERR_INVALID_ARG;
+    if (cluster != 0 && cluster != 1 && cluster != 2 && cluster != 4 && cluster != 8 && cluster != 16) return CR_ERR_INVALID_ARG;
     plan->tune.pg_block_kb = block_kb; plan->tune.pg_stages = stages; plan->tune.pg_cluster = cluster;
     return CR_OK;
 }

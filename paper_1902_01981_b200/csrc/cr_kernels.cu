@@ -1102,7 +1102,8 @@ cudaError_t launch_fused_tma(const AggArgs &a, const DeviceInfo &dev, const Tuni
                              cudaStream_t stream, int64_t *launches, bool *done) {
     *done = false;
     if (!encode || !tma_eligible(a) || a.batch != 1) return cudaSuccess;
-    int ncw = tune.ncw ? tune.ncw : 4;
+    // Short vectors give few column tiles: halve the tile so that more CTAs take part.
+    int ncw = tune.ncw ? tune.ncw : ((a.d + 511) / 512 < 3ll * dev.sm_count ? 2 : 4);
     if (ncw != 2 && ncw != 4 && ncw != 8) ncw = 4;
     const int tile = ncw * 128;
     const int boxw = tile < 256 ? tile : 256;
@@ -1117,6 +1118,11 @@ cudaError_t launch_fused_tma(const AggArgs &a, const DeviceInfo &dev, const Tuni
     int ctas = tune.ctas_per_sm ? tune.ctas_per_sm : 3;
     int stages = tune.stages ? tune.stages
                              : std::max(2, std::min(8, (int)((36 * 1024 + stage_bytes / 2) / stage_bytes)));
+    // With fewer tiles than resident CTAs the launch is bound by the latency of each box, not by HBM:
+    // deepen every CTA's ring so that about as many boxes are in flight as a full grid would have.
+    const long long tiles_now = (a.d + tile - 1) / tile;
+    if (!tune.stages && tiles_now < (long long)dev.sm_count * ctas)
+        stages = (int)std::min<long long>(8, std::max<long long>(stages, ((long long)dev.sm_count * ctas * stages + tiles_now - 1) / tiles_now));
     const size_t usable = (size_t)dev.smem_per_sm - 2048;  // leave room for the per-CTA reserve
     while (ctas > 1 && ((size_t)stages * stage_bytes + 1024 + 256) * ctas > usable) --ctas;
     while (stages > 2 && (size_t)stages * stage_bytes + 256 > (size_t)dev.smem_optin) --stages;
@@ -1360,6 +1366,10 @@ static cudaError_t run_partial_fused_rg(const PgArgs &pa, int csplit, int items,
     auto kern = cr_partial_fused_kernel<KPT, RG>;
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
+    if (csplit > 8) {
+        err = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        if (err != cudaSuccess) return err;
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)csplit, (unsigned)items, 1);
     cfg.blockDim = dim3(256, 1, 1);
@@ -1403,6 +1413,8 @@ cudaError_t launch_partial_gradients_fused(const float *X, const float *y, const
     const int item_blocks = slots_per_item * ((rows + RB - 1) / RB);
     int csplit = 1;
     while (csplit < 8 && item_blocks / (csplit * 2) >= 4) csplit *= 2;
+    // few items (coded gradients of a small tree): a cluster of 16 fills more of the GPU
+    if (csplit == 8 && items * 8 < 2 * dev.sm_count && item_blocks / 16 >= 4) csplit = 16;
     if (tune.pg_cluster) csplit = tune.pg_cluster;
     const size_t smem = (size_t)stages * RB * d * 4 + (size_t)d * 4 + (size_t)RB * 8 * 4 + (size_t)((RB + 3) & ~3) * 4 +
                         (size_t)stages * 8 + 16;
