@@ -182,7 +182,7 @@ __device__ __forceinline__ void fold_many(T (&acc)[NP][LMAX][4], const T (&e)[NP
 
 // Schedules of at most kInlineSteps entries travel inside the kernel parameters (constant bank), which
 // saves the host-to-device copy in front of short launches.
-constexpr int kInlineSteps = 96;
+constexpr int kInlineSteps = 160;
 
 struct FusedArgs {
     const void *coeff;

@@ -130,6 +130,12 @@ CONFIGS = {
     # are 16-byte multiples), (12,2) tree with one straggler per group: 168 partitions of 39 samples
     "cfg_logit": dict(n=12, L=2, s=1, P=168, d=5004, rows=39, code="cyclic", kind="logistic", x_std=1.0 / 70.0,
                       iters=20, lr=0.5, seed=0, mask_seed=1),
+    # the trees of the paper's clusters at a large gradient: (12,2) = 156 workers (stated for CR) and
+    # (4,3) = 84 workers (the only regular tree with 84 nodes), one straggler per sibling group
+    "cfg_tree12": dict(n=12, L=2, s=1, P=168, d=1 << 22, code="cyclic", kind="aggregate", std=1.0, iters=20,
+                       batch=1, exactly_s=True, seed=0, mask_seed=1),
+    "cfg_tree43": dict(n=4, L=3, s=1, P=112, d=1 << 22, code="cyclic", kind="aggregate", std=1.0, iters=20,
+                       batch=1, exactly_s=True, seed=0, mask_seed=1),
     "cfg_rep": dict(n=4, L=2, s=1, P=24, d=1 << 20, code="repetition", kind="aggregate", std=1.0, iters=20,
                     batch=1, exactly_s=False, seed=0, mask_seed=1, int_bound=1 << 10),
 }

@@ -92,6 +92,15 @@ def test_cfg5_deep_tree_batch_int32_bit_exact():
         assert np.array_equal(O.execute_integer(code, local, G_cols, masks[0]), want)
 
 
+@pytest.mark.parametrize("name", ["cfg_tree12", "cfg_tree43"])
+def test_paper_cluster_trees_d_2_22(name):
+    """The (12,2) and (4,3) trees of the paper's 156- and 84-worker clusters at d = 2^22."""
+    cfg = inputs.CONFIGS[name]
+    for it, (code, local, got, G_cols, masks) in enumerate(aggregate_full(cfg, B.CR_F32, 4)):
+        assert rel_l2(got[0], O.execute(code, local, G_cols, masks[0])) <= REL_L2_BAR
+        assert rel_l2(got[0], O.full_gradient(G_cols)) <= REL_L2_BAR
+
+
 @pytest.mark.parametrize("dtype", [B.CR_F32, B.CR_I32])
 def test_repetition_code_d_2_20(dtype):
     cfg = inputs.CONFIGS["cfg_rep"]
