@@ -144,6 +144,18 @@ cr_status_t cr_plan_get_decode(const cr_plan_t *plan, int32_t level, uint32_t st
  * message enters its parent.  capacity >= N always suffices; *count receives the length. */
 cr_status_t cr_plan_expand(const cr_plan_t *plan, const uint32_t *masks, int32_t capacity,
                            int32_t *nodes, int32_t *layers, double *weights, int32_t *count);
+/* Which children each parent ends up not waiting for, from the workers' computation times: the
+ * run-time model of Section III-C.  compute_time[v] (host, N doubles, >= 0) is the time node v needs
+ * for its local coded gradient (the paper draws it from the shifted exponential of Eq. (comp_model));
+ * a parent receives one message at a time (single-port model), each taking t_c, in the order in which
+ * its children's messages become ready (ties: lower index first); a node's message is ready once it
+ * holds n-s children messages and its own gradient (leaves: their own gradient).  The s children of
+ * every group whose messages would come last are marked in masks_out[num_groups] (host), ready to be
+ * passed to cr_aggregate; *t_total (may be NULL) receives the time at which the master holds its n-s
+ * messages, i.e. one sample of T_CR of Theorem 2.  Host work only. */
+cr_status_t cr_latency_masks(const cr_plan_t *plan, const double *compute_time, double t_c, uint32_t *masks_out,
+                             double *t_total);
+
 /* Sticky status word written by bounded device-side waits: CR_OK, or CR_ERR_TIMEOUT if a kernel of
  * this plan ever gave up waiting for a copy.  Synchronises the device. */
 cr_status_t cr_plan_device_status(cr_plan_t *plan);

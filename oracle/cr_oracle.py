@@ -464,6 +464,56 @@ def normalized_error_rate(w: np.ndarray, w_star: np.ndarray) -> float:
 
 
 # --------------------------------------------------------------------------
+# Run-time model (Section III-C): shifted-exponential computation, single-port communication
+# --------------------------------------------------------------------------
+
+
+def expected_order_statistic(n: int, s: int, load_points: float, a: float, mu: float) -> float:
+    """E[T_(n-s)] = (r d / mu) (H_n - H_s) + a r d for n i.i.d. shifted exponentials with shift
+    a r d and rate mu / (r d) (Appendix D); load_points = r d."""
+    H = lambda k: sum(1.0 / i for i in range(1, k + 1))
+    return load_points / mu * (H(n) - H(s)) + a * load_points
+
+
+def latency_trial(n: int, L: int, s: int, compute_time, t_c: float):
+    """One run of CR.Execute on the clock.  A leaf's message is ready when its computation ends.  A parent
+    listens to one child at a time (single-port model, a message takes t_c), serving children in the
+    order in which their messages become ready (ties: lower index), and stops after n-s messages; its own
+    message is ready when it has those and its own computation has ended.  Returns (masks, T): per
+    sibling group the bit mask of the s children not waited for, and the time at which the master has
+    its n-s messages.  Pinned by hand-worked cases, by the order-statistic mean of Appendix D (t_c = 0)
+    and by elementary bounds."""
+    ready = {}
+    masks = [0] * num_groups(n, L)
+
+    def serve(l, i):
+        """Time at which parent (l, i) holds n-s messages; records its group's mask."""
+        kids = []
+        for j in range(1, n + 1):
+            c = n * (i - 1) + j
+            kids.append((message_ready(l + 1, c), j - 1))
+        kids.sort()                       # by ready time, then by index
+        port_free = 0.0
+        got = 0.0
+        for rank, (t_ready, j) in enumerate(kids):
+            if rank < n - s:
+                port_free = max(t_ready, port_free) + t_c
+                got = port_free
+            else:
+                masks[group_of_parent(n, l, i)] |= 1 << j
+        return got
+
+    def message_ready(l, i):
+        if (l, i) not in ready:
+            own = float(compute_time[flat_index(n, l, i)])
+            ready[(l, i)] = own if l == L else max(serve(l, i), own)
+        return ready[(l, i)]
+
+    total = serve(0, 1)
+    return masks, total
+
+
+# --------------------------------------------------------------------------
 # Integer-exact mode
 # --------------------------------------------------------------------------
 

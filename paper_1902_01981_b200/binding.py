@@ -59,6 +59,7 @@ _SIGNATURES = {
     "cr_plan_get_decode": (C.c_int, [C.c_void_p, C.c_int32, C.c_uint32, C.c_void_p]),
     "cr_plan_expand": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
                                  C.POINTER(C.c_int32)]),
+    "cr_latency_masks": (C.c_int, [C.c_void_p, C.c_void_p, C.c_double, C.c_void_p, C.POINTER(C.c_double)]),
     "cr_plan_device_status": (C.c_int, [C.c_void_p]),
     "cr_partial_gradients_workspace_bytes": (C.c_size_t, [C.c_void_p, C.c_int32]),
     "cr_partial_gradients": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
@@ -208,6 +209,17 @@ def cr_plan_expand(plan: int, masks):
                                 weights.ctypes.data, C.byref(count)), "cr_plan_expand")
     k = count.value
     return nodes[:k].copy(), layers[:k].copy(), weights[:k].copy()
+
+
+def cr_latency_masks(plan: int, compute_time, t_c: float):
+    """(masks uint32 [groups], T_CR) for one vector of per-node computation times."""
+    ct = np.ascontiguousarray(np.asarray(compute_time, dtype=np.float64))
+    if ct.size != cr_plan_num_nodes(plan):
+        raise ValueError("one computation time per node is needed")
+    masks = np.zeros(cr_plan_num_groups(plan), dtype=np.uint32)
+    total = C.c_double()
+    _check(lib().cr_latency_masks(plan, ct.ctypes.data, t_c, masks.ctypes.data, C.byref(total)), "cr_latency_masks")
+    return masks, total.value
 
 
 def cr_plan_device_status(plan: int) -> int:

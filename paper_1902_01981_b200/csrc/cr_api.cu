@@ -319,6 +319,16 @@ cr_status_t cr_plan_expand(const cr_plan_t *plan, const uint32_t *masks, int32_t
     return CR_OK;
 }
 
+cr_status_t cr_latency_masks(const cr_plan_t *plan, const double *compute_time, double t_c, uint32_t *masks_out,
+                             double *t_total) {
+    if (!plan || !compute_time || !masks_out || !(t_c >= 0.0)) return CR_ERR_INVALID_ARG;
+    for (int v = 0; v < plan->hp.N; ++v)
+        if (!(compute_time[v] >= 0.0)) return CR_ERR_INVALID_ARG;
+    const double t = plan->hp.latency_masks(compute_time, t_c, masks_out);
+    if (t_total) *t_total = t;
+    return CR_OK;
+}
+
 cr_status_t cr_plan_device_status(cr_plan_t *plan) {
     cr_status_t st = check_device_plan(plan);
     if (st != CR_OK) return st;

@@ -245,6 +245,43 @@ cr_status_t HostPlan::expand(const uint32_t *masks, std::vector<UsedNode> &out) 
     return CR_OK;
 }
 
+double HostPlan::latency_masks(const double *compute_time, double t_c, uint32_t *masks_out) const {
+    // ready[v] = time at which node v's message is ready for upload.  Layers are handled bottom-up, so
+    // the children of a parent are ready before the parent is looked at.
+    std::vector<double> ready(N, 0.0);
+    for (int v = layer_offset[L]; v < N; ++v) ready[v] = compute_time[v];
+    double master_done = 0.0;
+    for (int l = L - 1; l >= 0; --l) {
+        const int parents = nodes_in_layer(l);
+        for (int i = 0; i < parents; ++i) {
+            const int first_child = layer_offset[l + 1] + i * n;
+            // the parent's single port serves its children in the order in which their messages become
+            // ready (ties: lower index first); a transfer takes t_c
+            std::vector<int> order(n);
+            for (int j = 0; j < n; ++j) order[j] = j;
+            std::stable_sort(order.begin(), order.end(),
+                             [&](int x, int y) { return ready[first_child + x] < ready[first_child + y]; });
+            double port_free = 0.0, got_enough = 0.0;
+            uint32_t mask = 0;
+            for (int k = 0; k < n; ++k) {
+                const int j = order[k];
+                if (k < n - s) {
+                    const double start = std::max(ready[first_child + j], port_free);
+                    port_free = start + t_c;
+                    got_enough = port_free;   // arrival of the (k+1)-th message
+                } else {
+                    mask |= 1u << j;          // the parent no longer waits for these
+                }
+            }
+            const int group = l == 0 ? 0 : layer_offset[l] + i + 1;
+            masks_out[group] = mask;
+            if (l == 0) master_done = got_enough;
+            else ready[layer_offset[l] + i] = std::max(got_enough, compute_time[layer_offset[l] + i]);
+        }
+    }
+    return master_done;
+}
+
 cr_status_t build_host_plan(const cr_plan_desc_t &desc, HostPlan &hp) {
     hp = HostPlan();
     const int n = desc.n, L = desc.L, s = desc.s;

@@ -47,6 +47,11 @@ struct HostPlan {
     const double *decode_row(int level, uint32_t mask) const { return &decode[level][(size_t)mask * n]; }
     bool mask_ok(uint32_t mask) const;
 
+    // Straggler pattern of one iteration from per-node computation times under the single-port model
+    // (Section III-C): see cr_latency_masks in codedreduce.h.  masks_out[groups], returns the time at
+    // which the master holds n-s messages.
+    double latency_masks(const double *compute_time, double t_c, uint32_t *masks_out) const;
+
     // Post-order expansion of one pattern.  Returns CR_OK, CR_ERR_UNDECODABLE_MASK or CR_ERR_INVALID_ARG.
     cr_status_t expand(const uint32_t *masks, std::vector<UsedNode> &out) const;
 };

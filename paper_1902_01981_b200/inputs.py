@@ -100,6 +100,12 @@ def straggler_masks(n: int, L: int, s: int, batch: int, seed: int,
     return masks
 
 
+def shifted_exponential_times(count: int, load_points: float, a: float, mu: float, seed: int, trials: int = 1):
+    """Computation times T with P[T <= t] = 1 - exp(-(mu / d_i)(t - a d_i)), t >= a d_i, for d_i =
+    load_points data points per worker; shape [trials, count], float64."""
+    return a * load_points + _rng(seed).exponential(load_points / mu, size=(trials, count))
+
+
 def replicate_into_slots(G_parts: np.ndarray, slot_partition: np.ndarray) -> np.ndarray:
     """Copy partition gradients into per-node slots: out[v, j] = G_parts[slot_partition[v, j]].
 

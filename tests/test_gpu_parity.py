@@ -157,6 +157,24 @@ def test_batch_of_patterns_with_different_shapes():
         B.cr_plan_destroy(plan)
 
 
+def test_masks_from_the_run_time_model():
+    """Straggler patterns produced by the shifted-exponential / single-port model feed the aggregation."""
+    cfg = tree(4, 3, 1, "cyclic", 3000)
+    plan = make_plan(cfg)
+    try:
+        code, local = check_slot_table(plan, cfg)
+        G = inputs.partition_gradients(cfg["P"], cfg["d"], seed=2)
+        G_dev = slots_on_device(plan, G, torch)
+        times = inputs.shifted_exponential_times(O.num_nodes(4, 3), 20.0, 0.01, 1.0, seed=5, trials=8)
+        masks = np.stack([B.cr_latency_masks(plan, t, 0.05)[0] for t in times])
+        assert [O.latency_trial(4, 3, 1, t, 0.05)[0] for t in times] == masks.tolist()
+        got = run_aggregate(plan, G_dev, masks, cfg["d"], B.CR_AGG_FUSED)
+        for b in range(8):
+            assert rel_l2(got[b], O.execute(code, local, G, masks[b])) <= REL_L2_BAR
+    finally:
+        B.cr_plan_destroy(plan)
+
+
 def test_fused_matches_unfused_closely():
     cfg = tree(5, 2, 2, "cyclic", 1 << 16)
     plan = make_plan(cfg)
