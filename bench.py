@@ -494,6 +494,93 @@ def run_linreg(args, cfg):
     B.cr_plan_destroy(plan)
 
 
+def run_multi(args, cfg):
+    """Partial gradients of --models K models in one pass over a regression workload (tensor-core path),
+    timed beside K passes of the single-model kernel.  One GPU; X is rounded to TF32-representable values."""
+    import torch
+    from paper_1902_01981_b200 import binding as B
+    from paper_1902_01981_b200 import build as cr_build
+    cr_build.build()
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(0)
+    code_id = {"printed_3_1": B.CR_CODE_PAPER_3_1, "cyclic": B.CR_CODE_CYCLIC_RANDOM,
+               "repetition": B.CR_CODE_FRACTIONAL_REPETITION}[cfg["code"]]
+    n, L, s, P, d, rows, K = cfg["n"], cfg["L"], cfg["s"], cfg["P"], cfg["d"], cfg["rows"], args.models
+    plan = B.cr_plan_create(n, L, s, P, d, code=code_id, device=0)
+    N, m = B.cr_plan_num_nodes(plan), B.cr_plan_load(plan)
+    logistic = cfg["kind"] == "logistic"
+    loss = B.CR_LOSS_LOGISTIC if logistic else B.CR_LOSS_SQUARED
+    if logistic:
+        X, y, _ = inputs.logistic_partitions(P, rows, d, cfg["seed"], cfg["x_std"])
+    else:
+        X, y, _ = inputs.linreg_partitions(P, rows, d, cfg["seed"], cfg["x_std"], cfg["noise_std"])
+    X = inputs.tf32_representable(X)
+    W = inputs.model_matrix(K, d, cfg["seed"] + 1)
+    X_dev, y_dev, W_dev = torch.from_numpy(X).cuda(), torch.from_numpy(y).cuda(), torch.from_numpy(W).cuda()
+    G = torch.zeros((K, N, m, d), device="cuda")
+    ws = torch.empty(B.cr_partial_gradients_multi_workspace_bytes(plan, rows), dtype=torch.uint8, device="cuda")
+    ws1 = torch.empty(max(16, B.cr_partial_gradients_workspace_bytes(plan, rows)), dtype=torch.uint8, device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if X.nbytes <= 126e6 else None
+    stream = torch.cuda.current_stream()
+
+    def timed(fn, steps):
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(steps)]
+        for i in range(steps):
+            if flush is not None:
+                flush.fill_(i & 0xff)
+            ev[i][0].record(stream)
+            fn()
+            ev[i][1].record(stream)
+        torch.cuda.synchronize()
+        return np.array([e[0].elapsed_time(e[1]) for e in ev]) * 1e-3
+
+    def multi():
+        B.cr_partial_gradients_multi(plan, loss, X_dev, y_dev, rows, W_dev, K, G, ws, None, stream)
+
+    def singles():
+        for k in range(K):
+            B.cr_partial_gradients_loss(plan, loss, X_dev, y_dev, rows, W_dev[k], G[k], ws1, stream)
+
+    steps = min(args.steps, 50)
+    timed(multi, args.warmup)
+    sampler = ClockSampler(0)
+    sampler.wait_first_sample()
+    n0 = B.cr_plan_launch_count(plan)
+    t0 = time.time()
+    t_multi = timed(multi, steps)
+    t1 = time.time()
+    launches = B.cr_plan_launch_count(plan) - n0
+    clocks = sampler.stop((t0, t1))
+    B.cr_plan_device_status(plan)
+    timed(singles, 1)
+    t_single = timed(singles, max(1, steps // 10))
+    # algorithmic bytes: each (node, slot) item reads its partition once per contraction and writes K gradients
+    items = N * m
+    nbytes = 4.0 * items * (2.0 * rows * d + K * d)
+    flops = 2.0 * 2.0 * rows * d * K * items
+    peak, peak_kind = peak_hbm()
+    sec = float(t_multi.mean())
+    achieved = nbytes / sec / 1e9
+    line = {
+        "metric": METRIC, "value": achieved, "unit": UNIT, "n_gpus": 1, "steps": steps, "warmup": args.warmup,
+        "ms_per_step": sec * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "tf32",
+        "data": "synthetic",
+        "config": {"workload": f"{args.workload}: partial gradients of K={K} models, n={n} L={L} s={s} P={P} rows={rows} "
+                               f"d={d} ({items} slot items), X TF32-representable",
+                   "l2": "inputs larger than L2 (no flush needed)" if flush is None else "L2 flushed between steps"},
+        "roofline": {"bound": "hbm", "kernel": "cr_tc_residual_kernel + cr_tc_gradient_kernel", "achieved": achieved,
+                     "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                     "traffic": None, "algorithmic_bytes_per_launch": nbytes, "avg_launch_ms": sec * 1e3,
+                     "tensor_tflops": flops / sec / 1e12},
+        "k_single_model_passes_ms": float(t_single.mean()) * 1e3,
+        "speedup_over_single_model_passes": float(t_single.mean()) / sec,
+        "cpu_baseline": None, "e2e": None, "gpu_launches": int(launches), "clocks": clocks,
+    }
+    print(json.dumps(line), flush=True)
+    B.cr_plan_destroy(plan)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -505,6 +592,7 @@ def main():
     ap.add_argument("--d", type=int, default=0, help="override the gradient length (profiling on a small case)")
     ap.add_argument("--tune", default="", help="consumer_warps,stages,ctas_per_sm,rows_per_box (0 = auto)")
     ap.add_argument("--coded", action="store_true", help="regression workloads: gradient + encode in one kernel")
+    ap.add_argument("--models", type=int, default=0, help="regression workloads: gradients of K models per pass (1..32)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-extras", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -524,6 +612,8 @@ def main():
     if cfg["kind"] in ("linreg", "logistic"):
         if args.impl == "reference":
             print(json.dumps({"impl": "reference", "unavailable": "the reference arm times aggregation workloads only"}))
+        elif args.models:
+            run_multi(args, cfg)
         else:
             run_linreg(args, cfg)
     elif args.impl == "reference":

@@ -191,6 +191,26 @@ cr_status_t cr_partial_gradients_loss(cr_plan_t *plan, int32_t loss, const float
 cr_status_t cr_coded_gradients(cr_plan_t *plan, int32_t loss, const float *X, const float *y, int32_t rows,
                                const float *w, float *E, void *stream);
 
+/* ---- partial gradients of K models in one pass (tensor cores) ----------------------------------
+ * Eq. (g) evaluated at K <= 32 models w_1..w_K at once (the candidates of a line search, several step
+ * sizes, an ensemble): for every node v, slot j with partition p and every k,
+ *   G_multi[k][v][j][:] = X_p^T (link(X_p w_k) - y_p),   link = identity or sigmoid by `loss`.
+ * With K columns the two products are dense contractions and run on the tensor cores (tcgen05,
+ * kind::tf32, fp32 accumulation in tensor memory).  Precision: the tensor core reads the upper 19 bits
+ * of each fp32 of X, so results carry fp32 accuracy only for X whose values are TF32-representable
+ * (low 13 mantissa bits zero); otherwise X is in effect truncated to TF32.  W and the residuals are
+ * split into two TF32 terms and are not truncated.
+ * X [P][rows][d], y [P][rows], W [K][d], G_multi [K][N][m][d], R_out [N][m][rows][K] or NULL
+ * (the residuals, for inspection): device pointers, fp32.  `workspace`: device scratch of at least
+ * cr_partial_gradients_multi_workspace_bytes(plan, rows) bytes (CR_ERR_OOM if smaller).  Needs
+ * d % 4 == 0, d >= 32, 1 <= K <= 32, N*m <= 65535 and 16-byte aligned X, G_multi, workspace
+ * (CR_ERR_INVALID_ARG otherwise).  Each G_multi[k] is a G_slots buffer for cr_aggregate.  CR_F32
+ * plans only. */
+size_t cr_partial_gradients_multi_workspace_bytes(const cr_plan_t *plan, int32_t rows);
+cr_status_t cr_partial_gradients_multi(cr_plan_t *plan, int32_t loss, const float *X, const float *y, int32_t rows,
+                                       const float *W, int32_t K, float *G_multi, float *R_out, void *workspace,
+                                       size_t workspace_bytes, void *stream);
+
 /* ---- the same partial-gradient pass for callers that cannot allocate device memory ----------------
  * (No counterpart in the paper: this is a packaging variant of cr_partial_gradients.)
  * Some callers have no way to provide the residual workspace: a host thread that runs inside a

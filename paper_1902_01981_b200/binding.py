@@ -68,6 +68,9 @@ _SIGNATURES = {
                                             C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
     "cr_coded_gradients": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
                                      C.c_void_p]),
+    "cr_partial_gradients_multi_workspace_bytes": (C.c_size_t, [C.c_void_p, C.c_int32]),
+    "cr_partial_gradients_multi": (C.c_int, [C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
+                                             C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]),
     "cr_partial_gradients_static_capacity": (C.c_size_t, []),
     "cr_partial_gradients_static": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
                                               C.c_void_p]),
@@ -259,6 +262,19 @@ def cr_coded_gradients(plan: int, loss: int, X, y, rows: int, w, E, stream=None)
     """E[v] = coded gradient of node v (its slots' gradients combined with their coefficients)."""
     _check(lib().cr_coded_gradients(plan, loss, _dev_ptr(X), _dev_ptr(y), rows, _dev_ptr(w), _dev_ptr(E),
                                     _stream_ptr(stream)), "cr_coded_gradients")
+
+
+def cr_partial_gradients_multi_workspace_bytes(plan: int, rows: int) -> int:
+    return lib().cr_partial_gradients_multi_workspace_bytes(plan, rows)
+
+
+def cr_partial_gradients_multi(plan: int, loss: int, X, y, rows: int, W, K: int, G_multi, workspace, R_out=None,
+                               stream=None) -> None:
+    """G_multi[k][v][j] = partial gradient of slot j of node v at model W[k], K <= 32 models in one pass."""
+    nbytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    _check(lib().cr_partial_gradients_multi(plan, loss, _dev_ptr(X), _dev_ptr(y), rows, _dev_ptr(W), K,
+                                            _dev_ptr(G_multi), _dev_ptr(R_out), _dev_ptr(workspace), nbytes,
+                                            _stream_ptr(stream)), "cr_partial_gradients_multi")
 
 
 def cr_partial_gradients_static_capacity() -> int:

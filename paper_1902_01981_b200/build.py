@@ -10,7 +10,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libcodedreduce.so")
-SOURCES = ["cr_plan.cpp", "cr_kernels.cu", "cr_api.cu"]
+SOURCES = ["cr_plan.cpp", "cr_kernels.cu", "cr_tc.cu", "cr_api.cu"]
 HEADERS = ["cr_plan.hpp", "cr_kernels.hpp"]
 
 

@@ -402,6 +402,34 @@ cr_status_t cr_coded_gradients(cr_plan_t *plan, int32_t loss, const float *X, co
     return CR_OK;
 }
 
+size_t cr_partial_gradients_multi_workspace_bytes(const cr_plan_t *plan, int32_t rows) {
+    if (!plan || rows < 1) return 0;
+    return cr::multi_model_workspace_bytes(plan->hp.N * plan->hp.m, rows, plan->hp.d);
+}
+
+cr_status_t cr_partial_gradients_multi(cr_plan_t *plan, int32_t loss, const float *X, const float *y, int32_t rows,
+                                       const float *W, int32_t K, float *G_multi, float *R_out, void *workspace,
+                                       size_t workspace_bytes, void *stream) {
+    cr_status_t st = check_device_plan(plan);
+    if (st != CR_OK) return st;
+    if (!X || !y || !W || !G_multi || rows < 1 || (loss != CR_LOSS_SQUARED && loss != CR_LOSS_LOGISTIC)) return CR_ERR_INVALID_ARG;
+    if (plan->hp.dtype != CR_F32) return CR_ERR_DTYPE;
+    if (!plan->encode) return CR_ERR_CUDA;
+    const int items = plan->hp.N * plan->hp.m;
+    if (!workspace || workspace_bytes < cr::multi_model_workspace_bytes(items, rows, plan->hp.d)) return CR_ERR_OOM;
+    if (!cr::multi_model_eligible(X, G_multi, workspace, plan->hp.d, rows, K, items)) {
+        std::snprintf(g_last_error, sizeof(g_last_error),
+                      "cr_partial_gradients_multi needs d %% 4 == 0, d >= 32, 1 <= K <= 32, N*m <= 65535 and 16-byte "
+                      "aligned X, G_multi, workspace");
+        return CR_ERR_INVALID_ARG;
+    }
+    cudaError_t e = cr::launch_partial_gradients_multi(X, y, W, K, plan->d_part, items, plan->hp.P, rows, plan->hp.d,
+                                                       G_multi, R_out, loss, workspace, plan->d_status, plan->encode,
+                                                       reinterpret_cast<cudaStream_t>(stream), &plan->launches);
+    if (e != cudaSuccess) { note_cuda(e, "cr_partial_gradients_multi"); return CR_ERR_CUDA; }
+    return CR_OK;
+}
+
 cr_status_t cr_encode(cr_plan_t *plan, const void *G_slots, void *E, void *stream) {
     cr_status_t st = check_device_plan(plan);
     if (st != CR_OK) return st;

@@ -104,4 +104,13 @@ cudaError_t launch_partial_gradients_fused(const float *X, const float *y, const
                                            float *G, int loss, int *status, const DeviceInfo &dev,
                                            const Tuning &tune, cudaStream_t stream, int64_t *launches);
 
+// Partial gradients of K <= 32 models at once on the tensor cores (cr_tc.cu): G [K][items][d]; R_out
+// optional [items][rows][K]; workspace of multi_model_workspace_bytes bytes.
+size_t multi_model_workspace_bytes(int items, int rows, int64_t d);
+bool multi_model_eligible(const float *X, const float *G, const void *workspace, int64_t d, int rows, int K, int items);
+cudaError_t launch_partial_gradients_multi(const float *X, const float *y, const float *W, int K, const int32_t *part,
+                                           int items, int P, int rows, int64_t d, float *G, float *R_out, int loss,
+                                           void *workspace, int *status, EncodeTiledFn encode, cudaStream_t stream,
+                                           int64_t *launches);
+
 }  // namespace cr

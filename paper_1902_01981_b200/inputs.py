@@ -73,6 +73,22 @@ def model_vector(d: int, seed: int) -> np.ndarray:
     return _rng(seed).standard_normal(d, dtype=np.float32)
 
 
+def model_matrix(K: int, d: int, seed: int, spread: float = 0.1) -> np.ndarray:
+    """K models around one start model, as a line search or an ensemble would hold them:
+    W[k] = w_0 + spread * N(0, I), fp32, shape [K, d]."""
+    rng = _rng(seed)
+    w0 = rng.standard_normal(d, dtype=np.float32)
+    return (w0[None, :] + np.float32(spread) * rng.standard_normal((K, d), dtype=np.float32)).astype(np.float32)
+
+
+def tf32_representable(x: np.ndarray) -> np.ndarray:
+    """Rounds fp32 values to the nearest value with a 10-bit mantissa (TF32), returned as fp32: the low
+    13 mantissa bits are zero, so a tensor core reads these numbers without loss."""
+    bits = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32)
+    rounded = (bits + np.uint32(0x1000)) & np.uint32(0xFFFFE000)
+    return rounded.view(np.float32)
+
+
 def group_count(n: int, L: int) -> int:
     """Sibling groups of an (n, L) tree: one per parent, the master included."""
     return sum(n ** l for l in range(L))
