@@ -199,7 +199,9 @@ cr_status_t cr_coded_gradients(cr_plan_t *plan, int32_t loss, const float *X, co
  * kind::tf32, fp32 accumulation in tensor memory).  Precision: the tensor core reads the upper 19 bits
  * of each fp32 of X, so results carry fp32 accuracy only for X whose values are TF32-representable
  * (low 13 mantissa bits zero); otherwise X is in effect truncated to TF32.  W and the residuals are
- * split into two TF32 terms and are not truncated.
+ * split into two TF32 terms and are not truncated.  The tensor core's fp32 accumulator truncates on
+ * every addition; the kernels spread each sum over 8 accumulators, which keeps the relative L2 error
+ * against exact arithmetic under 1e-5 for d <= 32768 and rows <= 16384 (it grows linearly beyond).
  * X [P][rows][d], y [P][rows], W [K][d], G_multi [K][N][m][d], R_out [N][m][rows][K] or NULL
  * (the residuals, for inspection): device pointers, fp32.  `workspace`: device scratch of at least
  * cr_partial_gradients_multi_workspace_bytes(plan, rows) bytes (CR_ERR_OOM if smaller).  Needs

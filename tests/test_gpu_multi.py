@@ -39,18 +39,12 @@ def oracle_parts(loss, X, y, w):
     return np.stack([fn(X[p], y[p], w) for p in range(X.shape[0])])
 
 
-def test_tf32_representable_inputs():
-    x = inputs.partition_gradients(4, 1000, 3)
-    r = inputs.tf32_representable(x)
-    assert (r.view(np.uint32) & 0x1FFF).max() == 0
-    assert np.abs(r - x).max() <= np.abs(x).max() * 2.0 ** -11
-
-
 CASES = [dict(n=3, L=1, s=1, P=6, d=256, code="printed_3_1", rows=64, K=3),      # one row tile, two column tiles
          dict(n=3, L=1, s=1, P=6, d=1000, code="printed_3_1", rows=200, K=32),   # ragged rows and columns, all models
          dict(n=3, L=2, s=1, P=15, d=36, code="printed_3_1", rows=9, K=1),       # smallest shapes
          dict(n=4, L=2, s=1, P=24, d=5004, code="cyclic", rows=39, K=8),         # shape of the logistic run
-         dict(n=4, L=2, s=1, P=48, d=4096, code="cyclic", rows=512, K=16)]
+         dict(n=4, L=2, s=1, P=48, d=4096, code="cyclic", rows=512, K=16),
+         dict(n=3, L=1, s=1, P=6, d=16384, code="printed_3_1", rows=24, K=2)]     # long contraction over d
 
 
 @pytest.mark.parametrize("loss", [B.CR_LOSS_SQUARED, B.CR_LOSS_LOGISTIC])
