@@ -89,7 +89,10 @@ typedef struct {
 
 /* Variants of cr_aggregate (low byte of `flags`) and option bits. */
 enum {
-    CR_AGG_FUSED = 0,        /* one kernel, TMA-staged tiles, all levels in registers/shared memory */
+    CR_AGG_FUSED = 0,        /* one kernel, TMA-staged tiles, all levels in registers/shared memory (single
+                                patterns whose TMA boxes would be 4 KB or less -- trees with m = 4 slot rows
+                                per node, and CR_AGG_FROM_CODED -- take the plain-load kernel unless
+                                cr_plan_tune fixed a TMA shape) */
     CR_AGG_FUSED_LDG = 1,    /* same dataflow with plain 128-bit loads (any d, any alignment) */
     CR_AGG_UNFUSED = 2,      /* cr_encode + cr_decode per level through the workspace */
     CR_AGG_UNCODED_SUM = 3,  /* comparator: plain sum of the same used slots, all weights 1 */
@@ -287,6 +290,12 @@ cr_status_t cr_plan_tune(cr_plan_t *plan, int32_t consumer_warps, int32_t stages
  * cluster = CTAs that share one (node, slot) item (1, 2, 4 or 8).  A shape that does not fit shared
  * memory makes cr_partial_gradients return CR_ERR_CUDA. */
 cr_status_t cr_plan_tune_gradients(cr_plan_t *plan, int32_t block_kb, int32_t stages, int32_t cluster);
+
+/* Order in which the partial-gradient kernels launch the (node, slot) items, and ring depth of the
+ * second kernel of cr_partial_gradients_multi; 0 keeps the built-in choice for that field.
+ * item_order: 1 = by node, then slot; 2 = grouped by partition (items that hold the same partition
+ * run side by side and share its rows through L2).  multi_stages: 2..4 (2 lets two CTAs share an SM). */
+cr_status_t cr_plan_tune_items(cr_plan_t *plan, int32_t item_order, int32_t multi_stages);
 
 /* Kernel launches enqueued by this plan's device calls so far. */
 int64_t cr_plan_launch_count(const cr_plan_t *plan);

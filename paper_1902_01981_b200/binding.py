@@ -84,6 +84,7 @@ _SIGNATURES = {
     "cr_aggregate_bytes": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(C.c_int64), C.POINTER(C.c_int32)]),
     "cr_plan_tune": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32]),
     "cr_plan_tune_gradients": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32]),
+    "cr_plan_tune_items": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32]),
     "cr_plan_launch_count": (C.c_int64, [C.c_void_p]),
 }
 
@@ -236,6 +237,10 @@ def cr_plan_tune(plan: int, consumer_warps: int = 0, stages: int = 0, ctas_per_s
 
 def cr_plan_tune_gradients(plan: int, block_kb: int = 0, stages: int = 0, cluster: int = 0) -> None:
     _check(lib().cr_plan_tune_gradients(plan, block_kb, stages, cluster), "cr_plan_tune_gradients")
+
+
+def cr_plan_tune_items(plan: int, item_order: int = 0, multi_stages: int = 0) -> None:
+    _check(lib().cr_plan_tune_items(plan, item_order, multi_stages), "cr_plan_tune_items")
 
 
 # ------------------------------------------------------------------ device work

@@ -51,6 +51,7 @@ struct cr_plan {
     void *d_coeff = nullptr;     // [N*m] float or int32
     void *d_ones = nullptr;      // [N] the value 1 in the plan's element type (aggregation of coded gradients)
     int32_t *d_part = nullptr;   // [N*m]
+    int32_t *d_order = nullptr;  // [N*m] slot items sorted by partition: launch order of the gradient kernels
     int *d_status = nullptr;
     cr::DeviceInfo dev;
     cr::Tuning tune;
@@ -196,6 +197,7 @@ cr_status_t cr_plan_destroy(cr_plan_t *plan) {
         if (plan->d_coeff) cudaFree(plan->d_coeff);
         if (plan->d_ones) cudaFree(plan->d_ones);
         if (plan->d_part) cudaFree(plan->d_part);
+        if (plan->d_order) cudaFree(plan->d_order);
         if (plan->d_status) cudaFree(plan->d_status);
     }
     delete plan;
@@ -244,6 +246,15 @@ cr_status_t cr_plan_create(const cr_plan_desc_t *desc, cr_plan_t **out) {
             CR_CUDA_P(cudaMemcpy(p->d_ones, ones.data(), ones.size() * 4, cudaMemcpyHostToDevice));
         }
         CR_CUDA_P(cudaMemcpy(p->d_part, part.data(), slots * 4, cudaMemcpyHostToDevice));
+        {
+            // items that hold the same partition compute the same gradient from the same rows of X:
+            // launched side by side, they fetch those rows from HBM once and share them through L2
+            std::vector<int32_t> order(slots);
+            for (size_t i = 0; i < slots; ++i) order[i] = (int32_t)i;
+            std::stable_sort(order.begin(), order.end(), [&](int32_t a, int32_t b) { return part[a] < part[b]; });
+            CR_CUDA_P(cudaMalloc(reinterpret_cast<void **>(&p->d_order), slots * 4));
+            CR_CUDA_P(cudaMemcpy(p->d_order, order.data(), slots * 4, cudaMemcpyHostToDevice));
+        }
         CR_CUDA_P(cudaMemset(p->d_status, 0, sizeof(int)));
         // cuTensorMapEncodeTiled through the runtime, so that the library needs no link to libcuda
         void *fn = nullptr;
@@ -279,6 +290,12 @@ cr_status_t cr_plan_tune_gradients(cr_plan_t *plan, int32_t block_kb, int32_t st
     if (!plan || block_kb < 0 || block_kb > 128 || stages < 0 || stages == 1 || stages > 8) return CR_ERR_INVALID_ARG;
     if (cluster != 0 && cluster != 1 && cluster != 2 && cluster != 4 && cluster != 8 && cluster != 16) return CR_ERR_INVALID_ARG;
     plan->tune.pg_block_kb = block_kb; plan->tune.pg_stages = stages; plan->tune.pg_cluster = cluster;
+    return CR_OK;
+}
+
+cr_status_t cr_plan_tune_items(cr_plan_t *plan, int32_t item_order, int32_t multi_stages) {
+    if (!plan || item_order < 0 || item_order > 2 || multi_stages < 0 || multi_stages == 1 || multi_stages > 4) return CR_ERR_INVALID_ARG;
+    plan->tune.pg_order = item_order; plan->tune.tc_stages = multi_stages;
     return CR_OK;
 }
 
@@ -365,7 +382,7 @@ cr_status_t cr_partial_gradients_loss(cr_plan_t *plan, int32_t loss, const float
     cudaError_t e;
     if (cr::partial_fused_eligible(X, w, G_slots, plan->hp.d, items)) {
         // one pass over X, no scratch
-        e = cr::launch_partial_gradients_fused(X, y, w, plan->d_part, nullptr, items, 1, rows, plan->hp.d, G_slots, loss,
+        e = cr::launch_partial_gradients_fused(X, y, w, plan->d_part, plan->tune.pg_order == 2 ? plan->d_order : nullptr, nullptr, items, 1, rows, plan->hp.d, G_slots, loss,
                                                plan->d_status, plan->dev, plan->tune,
                                                reinterpret_cast<cudaStream_t>(stream), &plan->launches);
     } else {
@@ -394,7 +411,7 @@ cr_status_t cr_coded_gradients(cr_plan_t *plan, int32_t loss, const float *X, co
                       "cr_coded_gradients needs d %% 4 == 0, d <= 8192 and 16-byte aligned X, w, E");
         return CR_ERR_INVALID_ARG;
     }
-    cudaError_t e = cr::launch_partial_gradients_fused(X, y, w, plan->d_part, reinterpret_cast<const float *>(plan->d_coeff),
+    cudaError_t e = cr::launch_partial_gradients_fused(X, y, w, plan->d_part, nullptr, reinterpret_cast<const float *>(plan->d_coeff),
                                                        plan->hp.N, plan->hp.m, rows, plan->hp.d, E, loss, plan->d_status,
                                                        plan->dev, plan->tune, reinterpret_cast<cudaStream_t>(stream),
                                                        &plan->launches);
@@ -423,8 +440,8 @@ cr_status_t cr_partial_gradients_multi(cr_plan_t *plan, int32_t loss, const floa
                       "aligned X, G_multi, workspace");
         return CR_ERR_INVALID_ARG;
     }
-    cudaError_t e = cr::launch_partial_gradients_multi(X, y, W, K, plan->d_part, items, plan->hp.P, rows, plan->hp.d,
-                                                       G_multi, R_out, loss, workspace, plan->d_status, plan->encode,
+    cudaError_t e = cr::launch_partial_gradients_multi(X, y, W, K, plan->d_part, plan->tune.pg_order == 1 ? nullptr : plan->d_order, items, plan->hp.P, rows, plan->hp.d,
+                                                       G_multi, R_out, loss, workspace, plan->d_status, plan->tune, plan->encode,
                                                        reinterpret_cast<cudaStream_t>(stream), &plan->launches);
     if (e != cudaSuccess) { note_cuda(e, "cr_partial_gradients_multi"); return CR_ERR_CUDA; }
     return CR_OK;
@@ -595,8 +612,17 @@ cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *m
             if (pb[k].layer != p0[k].layer) { a.same_shape = 0; break; }
     }
 
+    // Four slot rows per node make TMA boxes of 4 KB, and a coded gradient (one row per node) boxes of
+    // 1 KB: too small for the copy engine to keep HBM busy (measured at d = 2^22 on the (12,2) tree:
+    // 6.0-6.6 TB/s with m = 4, 1.7 TB/s from coded gradients).  The plain-load kernel, which for these
+    // two shapes requests the rows of the next schedule entries before it folds the current ones,
+    // reaches 7.4 and 7.0 TB/s there.  Unless the caller fixed a TMA launch shape, single patterns of
+    // these shapes take that kernel.
+    const bool prefer_plain = batch == 1 && (a.m == 4 || a.m == 1) && hp.d % 4 == 0 && !plan->tune.ncw &&
+                              !plan->tune.stages && !plan->tune.ctas_per_sm && !plan->tune.rows;
+
     // A single short pattern needs no staging: its schedule travels in the kernel parameters.
-    if (variant == CR_AGG_FUSED && batch == 1 && a.total_steps <= cr::inline_schedule_limit()) {
+    if (variant == CR_AGG_FUSED && !prefer_plain && batch == 1 && a.total_steps <= cr::inline_schedule_limit()) {
         bool done = false;
         cudaError_t e0 = cr::launch_fused_tma(a, plan->dev, plan->tune, plan->encode, s, &plan->launches, &done);
         if (e0 != cudaSuccess) { note_cuda(e0, "cr_aggregate"); return CR_ERR_CUDA; }
@@ -630,7 +656,7 @@ cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *m
         e = cr::launch_uncoded_sum(a, s, &plan->launches);
     } else {
         bool done = false;
-        if (variant == CR_AGG_FUSED) {
+        if (variant == CR_AGG_FUSED && !prefer_plain) {
             if (batch == 1) e = cr::launch_fused_tma(a, plan->dev, plan->tune, plan->encode, s, &plan->launches, &done);
             else e = cr::launch_fused_batch_tma(a, plan->dev, plan->tune, plan->encode, s, &plan->launches, &done);
         }

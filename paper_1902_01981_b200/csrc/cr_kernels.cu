@@ -632,7 +632,11 @@ template <> struct Loader<int, 4> {
     }
 };
 
-template <typename T, int LMAX, int V>
+// PIPE = 4 (m == 4): the four slot rows of the next node are requested before the current node is
+// combined and folded, so that eight row loads per thread are in flight instead of four.
+// PIPE = 1 (m == 1, aggregation of coded gradients): the rows of four schedule entries are requested
+// at once, and the next four before these are folded.
+template <typename T, int LMAX, int V, int PIPE>
 __global__ void __launch_bounds__(256)
 cr_fused_ldg_kernel(const T *__restrict__ G, const T *__restrict__ coeff, const Step *__restrict__ steps,
                     const int32_t *__restrict__ pat_off, int m, long long d, T *__restrict__ out, int shift) {
@@ -645,6 +649,62 @@ cr_fused_ldg_kernel(const T *__restrict__ G, const T *__restrict__ coeff, const 
     for (int l = 0; l < LMAX; ++l)
 #pragma unroll
         for (int q = 0; q < V; ++q) acc[l][q] = T(0);
+    if constexpr (PIPE == 1) {
+        T cur[4][V], nxt[4][V];
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (k0 + j < k1) Loader<T, V>::load(G + (size_t)__ldg(&steps[k0 + j].node) * d + col, cur[j]);
+#pragma unroll 2
+        for (int k = k0; k < k1; k += 4) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (k + 4 + j < k1) Loader<T, V>::load(G + (size_t)__ldg(&steps[k + 4 + j].node) * d + col, nxt[j]);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                if (k + j < k1) {
+                    const Step st = load_step(&steps[k + j]);
+                    const T c = __ldg(coeff + st.node);
+                    T e[V];
+#pragma unroll
+                    for (int q = 0; q < V; ++q) e[q] = c * cur[j][q];
+                    fold<T, LMAX, V>(acc, e, st.layer, weight_of<T>(st.wbits));
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+#pragma unroll
+                for (int q = 0; q < V; ++q) cur[j][q] = nxt[j][q];
+        }
+    } else if constexpr (PIPE == 4) {
+        T cur[4][V], nxt[4][V];
+        Step st = k0 < k1 ? load_step(&steps[k0]) : Step{0, 0, 0u, 0};
+        if (k0 < k1) {
+            const T *row = G + (size_t)st.node * 4 * d + col;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) Loader<T, V>::load(row + (size_t)j * d, cur[j]);
+        }
+#pragma unroll 2
+        for (int k = k0; k < k1; ++k) {
+            Step sn = st;
+            if (k + 1 < k1) {
+                sn = load_step(&steps[k + 1]);
+                const T *row = G + (size_t)sn.node * 4 * d + col;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) Loader<T, V>::load(row + (size_t)j * d, nxt[j]);
+            }
+            const T *cf = coeff + (size_t)st.node * 4;
+            const T c0 = __ldg(cf), c1 = __ldg(cf + 1), c2 = __ldg(cf + 2), c3 = __ldg(cf + 3);
+            T e[V];
+#pragma unroll
+            for (int q = 0; q < V; ++q) e[q] = c0 * cur[0][q] + c1 * cur[1][q] + c2 * cur[2][q] + c3 * cur[3][q];
+            fold<T, LMAX, V>(acc, e, st.layer, weight_of<T>(st.wbits));
+            st = sn;
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+#pragma unroll
+                for (int q = 0; q < V; ++q) cur[j][q] = nxt[j][q];
+        }
+    } else
     for (int k = k0; k < k1; ++k) {
         const Step st = load_step(&steps[k]);
         const T *row = G + (size_t)st.node * m * d + col;
@@ -860,6 +920,8 @@ struct PgArgs {
     const float *y;
     const float *w;
     const int32_t *part;
+    const int32_t *order; // [items] or null: cluster y works on item order[y] (items that read the same
+                          // partition launched next to each other share its rows through L2)
     const float *coeff;   // [N*m] slot coefficients, or null: every slot weighs 1
     float *G;             // [items][d]
     int rows;
@@ -908,7 +970,7 @@ cr_partial_fused_kernel(const PgArgs a) {
     // The item's work is a list of row blocks: slot by slot, `bps` blocks of RB rows per slot (a block
     // never straddles two slots, whose partitions lie apart).  CTA c of the cluster takes a contiguous
     // share of the list.
-    const long long item = blockIdx.y;
+    const long long item = a.order ? (long long)__ldg(&a.order[blockIdx.y]) : (long long)blockIdx.y;
     const int spi = a.slots_per_item;
     const int bps = (a.rows + RB - 1) / RB;
     const int total_blocks = spi * bps;
@@ -1254,10 +1316,26 @@ static cudaError_t run_ldg(const AggArgs &a, cudaStream_t stream) {
     const T *G = reinterpret_cast<const T *>(a.G);
     const T *cf = reinterpret_cast<const T *>(a.coeff);
     T *out = reinterpret_cast<T *>(a.out);
+    if (a.m == 4 && V == 4) {
+        switch (pick_lmax(a.L)) {
+            case 2: cr_fused_ldg_kernel<T, 2, V, 4><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift); break;
+            case 4: cr_fused_ldg_kernel<T, 4, V, 4><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift); break;
+            default: cr_fused_ldg_kernel<T, 8, V, 4><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift); break;
+        }
+        return cudaGetLastError();
+    }
+    if (a.m == 1 && V == 4) {
+        switch (pick_lmax(a.L)) {
+            case 2: cr_fused_ldg_kernel<T, 2, V, 1><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift); break;
+            case 4: cr_fused_ldg_kernel<T, 4, V, 1><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift); break;
+            default: cr_fused_ldg_kernel<T, 8, V, 1><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift); break;
+        }
+        return cudaGetLastError();
+    }
     switch (pick_lmax(a.L)) {
-        case 2: cr_fused_ldg_kernel<T, 2, V><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift); break;
-        case 4: cr_fused_ldg_kernel<T, 4, V><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift); break;
-        default: cr_fused_ldg_kernel<T, 8, V><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift); break;
+        case 2: cr_fused_ldg_kernel<T, 2, V, 0><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift); break;
+        case 4: cr_fused_ldg_kernel<T, 4, V, 0><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift); break;
+        default: cr_fused_ldg_kernel<T, 8, V, 0><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift); break;
     }
     return cudaGetLastError();
 }
@@ -1397,7 +1475,8 @@ bool partial_fused_eligible(const float *X, const float *w, const float *G, int6
 }
 
 cudaError_t launch_partial_gradients_fused(const float *X, const float *y, const float *w, const int32_t *part,
-                                           const float *coeff, int items, int slots_per_item, int rows, int64_t d,
+                                           const int32_t *order, const float *coeff, int items, int slots_per_item,
+                                           int rows, int64_t d,
                                            float *G, int loss, int *status, const DeviceInfo &dev,
                                            const Tuning &tune, cudaStream_t stream, int64_t *launches) {
     // Measured on B200 (d = 4096, rows = 2048): two CTAs per SM hide each other's reduction latency
@@ -1420,7 +1499,7 @@ cudaError_t launch_partial_gradients_fused(const float *X, const float *y, const
                         (size_t)stages * 8 + 16;
     if (smem > (size_t)dev.smem_optin) return cudaErrorInvalidConfiguration;
     PgArgs pa;
-    pa.X = X; pa.y = y; pa.w = w; pa.part = part; pa.coeff = coeff; pa.G = G; pa.rows = rows;
+    pa.X = X; pa.y = y; pa.w = w; pa.part = part; pa.order = slots_per_item == 1 ? order : nullptr; pa.coeff = coeff; pa.G = G; pa.rows = rows;
     pa.slots_per_item = slots_per_item; pa.loss = loss; pa.RB = RB; pa.stages = stages; pa.d = d; pa.status = status;
     cudaError_t err;
     if (d <= 1024) err = run_partial_fused<1>(pa, csplit, items, smem, stream);

@@ -26,6 +26,8 @@ struct Tuning {
     int pg_block_kb = 0;  // partial gradients: KB of X per staged row block
     int pg_stages = 0;    // partial gradients: row-block buffers per CTA
     int pg_cluster = 0;   // partial gradients: CTAs per (node, slot) item (1, 2, 4 or 8)
+    int pg_order = 0;     // partial gradients: launch order of the items: 1 (node, slot), 2 grouped by partition
+    int tc_stages = 0;    // multi-model gradients: ring depth of the X^T R kernel (2..4)
 };
 
 struct DeviceInfo {
@@ -98,9 +100,11 @@ cudaError_t launch_partial_gradients_two_pass(const float *X, const float *y, co
 bool partial_fused_eligible(const float *X, const float *w, const float *G, int64_t d, int items);
 // slots_per_item = 1: G[item] for every (node, slot) item; slots_per_item = m with `coeff`: item = node,
 // G[node] = sum_j coeff[node*m+j] * (gradient of slot j), the node's coded gradient.
-// loss: 0 squared (r = X w - y), 1 logistic (r = sigmoid(X w) - y).
+// loss: 0 squared (r = X w - y), 1 logistic (r = sigmoid(X w) - y).  `order` ([items], may be null;
+// used when slots_per_item = 1): the order in which the items are launched.
 cudaError_t launch_partial_gradients_fused(const float *X, const float *y, const float *w, const int32_t *part,
-                                           const float *coeff, int items, int slots_per_item, int rows, int64_t d,
+                                           const int32_t *order, const float *coeff, int items, int slots_per_item,
+                                           int rows, int64_t d,
                                            float *G, int loss, int *status, const DeviceInfo &dev,
                                            const Tuning &tune, cudaStream_t stream, int64_t *launches);
 
@@ -109,8 +113,9 @@ cudaError_t launch_partial_gradients_fused(const float *X, const float *y, const
 size_t multi_model_workspace_bytes(int items, int rows, int64_t d);
 bool multi_model_eligible(const float *X, const float *G, const void *workspace, int64_t d, int rows, int K, int items);
 cudaError_t launch_partial_gradients_multi(const float *X, const float *y, const float *W, int K, const int32_t *part,
-                                           int items, int P, int rows, int64_t d, float *G, float *R_out, int loss,
-                                           void *workspace, int *status, EncodeTiledFn encode, cudaStream_t stream,
-                                           int64_t *launches);
+                                           const int32_t *order, int items, int P, int rows, int64_t d, float *G,
+                                           float *R_out, int loss,
+                                           void *workspace, int *status, const Tuning &tune, EncodeTiledFn encode,
+                                           cudaStream_t stream, int64_t *launches);
 
 }  // namespace cr

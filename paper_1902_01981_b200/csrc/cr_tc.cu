@@ -201,6 +201,7 @@ __global__ void cr_tc_split_models_kernel(const float *__restrict__ W, int K, lo
 struct TcResidualArgs {
     const float *y;        // [P][rows]
     const int32_t *part;   // [items]
+    const int32_t *order;  // [items] or null: launch order of the items (same partition side by side)
     float *Rh, *Rl;        // [items][rows_pad][32]
     float *R_out;          // optional [items][rows][K]
     int rows, rows_pad, K, loss, stages;
@@ -226,7 +227,7 @@ cr_tc_residual_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_con
     volatile int *flags = reinterpret_cast<volatile int *>(tmem_slot + 1);   // [0] someone gave up, [1] never set
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int item = blockIdx.y;
+    const int item = a.order ? __ldg(&a.order[blockIdx.y]) : (int)blockIdx.y;
     const int row0 = blockIdx.x * kTileM;
     const int p = __ldg(&a.part[item]);
 
@@ -343,6 +344,7 @@ constexpr int kRowsB = 64;
 
 struct TcGradientArgs {
     const int32_t *part;   // [items]
+    const int32_t *order;  // [items] or null
     float *G;              // [K][items][d]
     long long d;
     int rows, K, items, stages;
@@ -367,7 +369,7 @@ cr_tc_gradient_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_con
     volatile int *flags = reinterpret_cast<volatile int *>(tmem_slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int item = blockIdx.y;
+    const int item = a.order ? __ldg(&a.order[blockIdx.y]) : (int)blockIdx.y;
     const int col0 = blockIdx.x * kTileM;
     const int p = __ldg(&a.part[item]);
     const int chunks = (a.rows + kRowsB - 1) / kRowsB;
@@ -478,9 +480,10 @@ bool multi_model_eligible(const float *X, const float *G, const void *workspace,
 }
 
 cudaError_t launch_partial_gradients_multi(const float *X, const float *y, const float *W, int K, const int32_t *part,
-                                           int items, int P, int rows, int64_t d, float *G, float *R_out, int loss,
-                                           void *workspace, int *status, EncodeTiledFn encode, cudaStream_t stream,
-                                           int64_t *launches) {
+                                           const int32_t *order, int items, int P, int rows, int64_t d, float *G,
+                                           float *R_out, int loss,
+                                           void *workspace, int *status, const Tuning &tune, EncodeTiledFn encode,
+                                           cudaStream_t stream, int64_t *launches) {
     using namespace tc;
     const int rows_pad = (rows + kTileM - 1) / kTileM * kTileM;
     float *Wh = reinterpret_cast<float *>(workspace);
@@ -522,7 +525,7 @@ cudaError_t launch_partial_gradients_multi(const float *X, const float *y, const
 
     {   // residuals
         TcResidualArgs ra;
-        ra.y = y; ra.part = part; ra.Rh = Rh; ra.Rl = Rl; ra.R_out = R_out; ra.rows = rows; ra.rows_pad = rows_pad;
+        ra.y = y; ra.part = part; ra.order = order; ra.Rh = Rh; ra.Rl = Rl; ra.R_out = R_out; ra.rows = rows; ra.rows_pad = rows_pad;
         ra.K = K; ra.loss = loss; ra.stages = 4; ra.kchunks = (int)((d + kBoxCols - 1) / kBoxCols); ra.status = status;
         const size_t smem = (size_t)ra.stages * (kTileM * kBoxCols * 4 + 2 * kModels * kBoxCols * 4) + (2 * ra.stages + 1) * 8 + 16 + 1024;
         cudaError_t e = cudaFuncSetAttribute(cr_tc_residual_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -534,7 +537,7 @@ cudaError_t launch_partial_gradients_multi(const float *X, const float *y, const
     }
     if (G) {   // gradients
         TcGradientArgs ga;
-        ga.part = part; ga.G = G; ga.d = d; ga.rows = rows; ga.K = K; ga.items = items; ga.stages = 3; ga.status = status;
+        ga.part = part; ga.order = order; ga.G = G; ga.d = d; ga.rows = rows; ga.K = K; ga.items = items; ga.stages = tune.tc_stages ? tune.tc_stages : 2; ga.status = status;
         const size_t smem = (size_t)ga.stages * ((kTileM / kBoxCols + 2) * kRowsB * kBoxCols * 4) + (2 * ga.stages + 1) * 8 + 16 + 1024;
         cudaError_t e = cudaFuncSetAttribute(cr_tc_gradient_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
