@@ -358,9 +358,9 @@ def run_ours(args, cfg):
         avg_launch = float(per.mean())
         avg_bytes = units / args.steps
         achieved = avg_bytes / avg_launch / 1e9
-        # single patterns over m = 4 trees are routed to the plain-load kernel (4 KB TMA boxes cannot keep up)
+        # single patterns over m = 4 or 8 trees are routed to the plain-load kernel (small TMA boxes cannot keep up)
         kern = ("cr_fused_batch_tma_kernel" if batch > 1 else
-                "cr_fused_ldg_kernel" if (m == 4 and not args.tune) else "cr_fused_tma_kernel")
+                "cr_fused_ldg_kernel" if (m in (4, 8) and d >= (1 << 19) and not args.tune) else "cr_fused_tma_kernel")
         traffic = NCU_TRAFFIC_BYTES.get((args.workload, args.dtype, d))
         roofline = {"bound": "hbm", "kernel": kern, "achieved": achieved, "peak": peak, "unit": "GB/s",
                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / 8000.0,

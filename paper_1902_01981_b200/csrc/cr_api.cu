@@ -612,14 +612,17 @@ cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *m
             if (pb[k].layer != p0[k].layer) { a.same_shape = 0; break; }
     }
 
-    // Four slot rows per node make TMA boxes of 4 KB, and a coded gradient (one row per node) boxes of
-    // 1 KB: too small for the copy engine to keep HBM busy (measured at d = 2^22 on the (12,2) tree:
-    // 6.0-6.6 TB/s with m = 4, 1.7 TB/s from coded gradients).  The plain-load kernel, which for these
-    // two shapes requests the rows of the next schedule entries before it folds the current ones,
-    // reaches 7.4 and 7.0 TB/s there.  Unless the caller fixed a TMA launch shape, single patterns of
-    // these shapes take that kernel.
-    const bool prefer_plain = batch == 1 && (a.m == 4 || a.m == 1) && hp.d % 4 == 0 && !plan->tune.ncw &&
-                              !plan->tune.stages && !plan->tune.ctas_per_sm && !plan->tune.rows;
+    // Few slot rows per node make small TMA boxes (m = 4: 4 KB; a coded gradient, one row per node:
+    // 1 KB), too small for the copy engine to keep HBM busy (measured at d = 2^22 on the (12,2) tree:
+    // 6.0-6.6 TB/s with m = 4, 1.7 TB/s from coded gradients).  The plain-load kernel, which requests
+    // the next group of rows before it combines the current one, reaches 7.3 and 7.0 TB/s there, and
+    // is still 2 % ahead at m = 8 ((4,3) tree: 7.32 against 7.16 TB/s).  Unless the caller fixed a TMA
+    // launch shape, single patterns of these shapes take that kernel.
+    // Short vectors stay with the TMA kernel unless they are coded gradients: its narrow tiles and
+    // deep rings fill more SMs (m = 4, d = 5004: 70 against 109 us; from coded gradients 51 against 37 us).
+    const bool prefer_plain = batch == 1 && (a.m == 1 || ((a.m == 4 || a.m == 8) && hp.d >= (1ll << 19))) &&
+                              hp.d % 4 == 0 && !plan->tune.ncw && !plan->tune.stages && !plan->tune.ctas_per_sm &&
+                              !plan->tune.rows;
 
     // A single short pattern needs no staging: its schedule travels in the kernel parameters.
     if (variant == CR_AGG_FUSED && !prefer_plain && batch == 1 && a.total_steps <= cr::inline_schedule_limit()) {
