@@ -125,3 +125,38 @@ def test_multi_model_rejects_bad_arguments():
         assert e.value.status == B.CR_ERR_OOM
     finally:
         B.cr_plan_destroy(plan)
+
+
+def test_item_order_and_ring_depth_do_not_change_results():
+    """The launch order of the items and the ring depth are tuning only: every setting gives the same bits."""
+    cfg = dict(n=4, L=2, s=1, P=24, d=640, code="cyclic", rows=150, K=5)
+    P, d, rows, K = cfg["P"], cfg["d"], cfg["rows"], cfg["K"]
+    plan = make_plan(cfg)
+    try:
+        X, y = make_data(B.CR_LOSS_LOGISTIC, P, rows, d, seed=31)
+        W = inputs.model_matrix(K, d, seed=32)
+        N, m = B.cr_plan_num_nodes(plan), B.cr_plan_load(plan)
+        X_dev, y_dev, W_dev = torch.from_numpy(X).cuda(), torch.from_numpy(y).cuda(), torch.from_numpy(W).cuda()
+        ws = torch.empty(B.cr_partial_gradients_multi_workspace_bytes(plan, rows), dtype=torch.uint8, device="cuda")
+        ws1 = torch.empty(max(16, B.cr_partial_gradients_workspace_bytes(plan, rows)), dtype=torch.uint8, device="cuda")
+        multi, single = [], []
+        for order, stages in ((0, 0), (1, 2), (2, 3), (2, 4)):
+            B.cr_plan_tune_items(plan, order, stages)
+            G = torch.full((K, N, m, d), float("nan"), device="cuda")
+            B.cr_partial_gradients_multi(plan, B.CR_LOSS_LOGISTIC, X_dev, y_dev, rows, W_dev, K, G, ws)
+            G1 = torch.full((N, m, d), float("nan"), device="cuda")
+            B.cr_partial_gradients_loss(plan, B.CR_LOSS_LOGISTIC, X_dev, y_dev, rows, W_dev[0], G1, ws1)
+            torch.cuda.synchronize()
+            B.cr_plan_device_status(plan)
+            multi.append(G.cpu().numpy())
+            single.append(G1.cpu().numpy())
+        for g in multi[1:]:
+            assert np.array_equal(g, multi[0])
+        for g in single[1:]:
+            assert np.array_equal(g, single[0])
+        with pytest.raises(B.CodedReduceError):
+            B.cr_plan_tune_items(plan, 3, 0)
+        with pytest.raises(B.CodedReduceError):
+            B.cr_plan_tune_items(plan, 0, 5)
+    finally:
+        B.cr_plan_destroy(plan)
