@@ -158,6 +158,10 @@ CONFIGS = {
                        batch=1, exactly_s=True, seed=0, mask_seed=1),
     "cfg_tree43": dict(n=4, L=3, s=1, P=112, d=1 << 22, code="cyclic", kind="aggregate", std=1.0, iters=20,
                        batch=1, exactly_s=True, seed=0, mask_seed=1),
+    # shaped like the paper's CNN run: p ~ 1.2e5 parameters, (12,2) tree, 5 of 12 children straggling in
+    # every group; (s+1) | n, so the 0/1 fractional repetition code exists (m = 36 slots per node)
+    "cfg_cnn": dict(n=12, L=2, s=5, P=216, d=120000, code="repetition", kind="aggregate", std=1.0, iters=20,
+                    batch=1, exactly_s=True, seed=0, mask_seed=1, int_bound=1 << 10),
     "cfg_rep": dict(n=4, L=2, s=1, P=24, d=1 << 20, code="repetition", kind="aggregate", std=1.0, iters=20,
                     batch=1, exactly_s=False, seed=0, mask_seed=1, int_bound=1 << 10),
 }

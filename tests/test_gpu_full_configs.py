@@ -101,6 +101,27 @@ def test_paper_cluster_trees_d_2_22(name):
         assert rel_l2(got[0], O.full_gradient(G_cols)) <= REL_L2_BAR
 
 
+@pytest.mark.parametrize("s", [1, 2, 3, 5])
+@pytest.mark.parametrize("d", [5001, 6500, 120000])
+def test_paper_cluster_straggler_fractions(s, d):
+    """(12,2) tree with s = alpha n stragglers tolerated per group for the paper's alpha = 1/12 .. 5/12, at
+    the model sizes of its three experiments (p = 5001, 6500, ~1.2e5); (s+1) divides 12, so the 0/1
+    fractional repetition code exists for each (m = (s+1)^2 slots per node, up to 36)."""
+    cfg = dict(n=12, L=2, s=s, P=O.partition_quantum(12, 2, s), d=d, code="repetition", seed=3, mask_seed=4,
+               int_bound=1 << 10)
+    for dtype in (B.CR_F32, B.CR_I32):
+        for flags in (B.CR_AGG_FUSED, B.CR_AGG_FUSED_LDG):
+            for code, local, got, G_cols, masks in aggregate_full(dict(cfg, batch=1), dtype, 2, flags):
+                if dtype == B.CR_I32:
+                    assert np.array_equal(got[0].astype(np.int64), G_cols.astype(np.int64).sum(0))
+                else:
+                    assert rel_l2(got[0], O.execute(code, local, G_cols, masks[0])) <= REL_L2_BAR
+    # a batch of patterns through the batch kernel
+    for code, local, got, G_cols, masks in aggregate_full(dict(cfg, batch=5), B.CR_F32, 1):
+        for b in range(5):
+            assert rel_l2(got[b], O.execute(code, local, G_cols, masks[b])) <= REL_L2_BAR
+
+
 @pytest.mark.parametrize("dtype", [B.CR_F32, B.CR_I32])
 def test_repetition_code_d_2_20(dtype):
     cfg = inputs.CONFIGS["cfg_rep"]
