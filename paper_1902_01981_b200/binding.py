@@ -127,10 +127,22 @@ def _stream_ptr(stream) -> int:
 
 
 def _masks(masks, cols: int) -> np.ndarray:
-    m = np.ascontiguousarray(np.asarray(masks, dtype=np.uint32))
+    m = masks if (isinstance(masks, np.ndarray) and masks.dtype == np.uint32 and masks.flags.c_contiguous) \
+        else np.ascontiguousarray(np.asarray(masks, dtype=np.uint32))
     if m.size % cols != 0:
         raise ValueError(f"mask array of {m.size} entries is not a multiple of {cols}")
     return m.reshape(-1, cols)
+
+
+_groups_of_plan = {}
+
+
+def _num_groups(plan: int) -> int:
+    """cr_plan_num_groups, remembered per live plan (the hot calls need it to shape the masks)."""
+    g = _groups_of_plan.get(plan)
+    if g is None:
+        g = _groups_of_plan[plan] = lib().cr_plan_num_groups(plan)
+    return g
 
 
 # ------------------------------------------------------------------ plan
@@ -155,6 +167,7 @@ def cr_plan_create(n: int, L: int, s: int, P: int, d: int, code: int = CR_CODE_C
 
 
 def cr_plan_destroy(plan: int) -> None:
+    _groups_of_plan.pop(plan, None)      # the handle may be reused by a later plan
     _check(lib().cr_plan_destroy(plan), "cr_plan_destroy")
 
 
@@ -310,7 +323,7 @@ def cr_aggregate_workspace_bytes(plan: int, batch: int, flags: int) -> int:
 
 def cr_aggregate(plan: int, G_slots, masks, g_out, flags: int = CR_AGG_FUSED, workspace=None, stream=None) -> None:
     """masks: [batch, groups] (or [groups]) uint32 on the host; g_out: [batch, d] device tensor."""
-    mk = _masks(masks, cr_plan_num_groups(plan))
+    mk = _masks(masks, _num_groups(plan))
     _check(lib().cr_aggregate(plan, _dev_ptr(G_slots), mk.ctypes.data, mk.shape[0], _dev_ptr(g_out), flags,
                               _dev_ptr(workspace),
                               0 if workspace is None else workspace.numel() * workspace.element_size(),

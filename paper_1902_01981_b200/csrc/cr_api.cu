@@ -158,7 +158,8 @@ cr_status_t check_device_plan(cr_plan *p) {
         std::snprintf(g_last_error, sizeof(g_last_error), "device work asked of a host-only plan");
         return CR_ERR_CUDA;
     }
-    CR_CUDA(cudaSetDevice(p->device));
+    int current = -1;
+    if (cudaGetDevice(&current) != cudaSuccess || current != p->device) CR_CUDA(cudaSetDevice(p->device));
     return CR_OK;
 }
 
@@ -630,6 +631,13 @@ cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *m
         cudaError_t e0 = cr::launch_fused_tma(a, plan->dev, plan->tune, plan->encode, s, &plan->launches, &done);
         if (e0 != cudaSuccess) { note_cuda(e0, "cr_aggregate"); return CR_ERR_CUDA; }
         if (done) return CR_OK;
+    }
+
+    if ((variant == CR_AGG_FUSED_LDG || (variant == CR_AGG_FUSED && prefer_plain)) && batch == 1 &&
+        a.total_steps <= cr::inline_schedule_limit()) {
+        cudaError_t e0 = cr::launch_fused_ldg(a, s, &plan->launches);
+        if (e0 != cudaSuccess) { note_cuda(e0, "cr_aggregate"); return CR_ERR_CUDA; }
+        return CR_OK;
     }
 
     // staging layout: steps | pattern offsets | union nodes

@@ -639,14 +639,25 @@ template <> struct Loader<int, 4> {
 // current four are combined, so that eight row loads per thread are in flight instead of four.
 // PIPE = 1 (m == 1, aggregation of coded gradients): the rows of four schedule entries are requested
 // at once, and the next four before these are folded.
+// A single short schedule travels in the kernel parameters (inl.n > 0; `steps` and `pat_off` unused).
+struct InlineSchedule {
+    int n;
+    Step steps[kInlineSteps];
+};
+
 template <typename T, int LMAX, int V, int PIPE>
 __global__ void __launch_bounds__(256)
 cr_fused_ldg_kernel(const T *__restrict__ G, const T *__restrict__ coeff, const Step *__restrict__ steps,
-                    const int32_t *__restrict__ pat_off, int m, long long d, T *__restrict__ out, int shift) {
+                    const int32_t *__restrict__ pat_off, int m, long long d, T *__restrict__ out, int shift,
+                    const __grid_constant__ InlineSchedule inl) {
     const int b = blockIdx.y;
     const long long col = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * V;
     if (col >= d) return;
-    const int k0 = __ldg(&pat_off[b]), k1 = __ldg(&pat_off[b + 1]);
+    const int k0 = inl.n ? 0 : __ldg(&pat_off[b]), k1 = inl.n ? inl.n : __ldg(&pat_off[b + 1]);
+    auto step_at = [&](int k) {
+        if (inl.n) { Step t = inl.steps[k]; t.layer &= 0xff; return t; }
+        return load_step(&steps[k]);
+    };
     T acc[LMAX][V];
 #pragma unroll
     for (int l = 0; l < LMAX; ++l)
@@ -656,16 +667,16 @@ cr_fused_ldg_kernel(const T *__restrict__ G, const T *__restrict__ coeff, const 
         T cur[4][V], nxt[4][V];
 #pragma unroll
         for (int j = 0; j < 4; ++j)
-            if (k0 + j < k1) Loader<T, V>::load(G + (size_t)__ldg(&steps[k0 + j].node) * d + col, cur[j]);
+            if (k0 + j < k1) Loader<T, V>::load(G + (size_t)step_at(k0 + j).node * d + col, cur[j]);
 #pragma unroll 2
         for (int k = k0; k < k1; k += 4) {
 #pragma unroll
             for (int j = 0; j < 4; ++j)
-                if (k + 4 + j < k1) Loader<T, V>::load(G + (size_t)__ldg(&steps[k + 4 + j].node) * d + col, nxt[j]);
+                if (k + 4 + j < k1) Loader<T, V>::load(G + (size_t)step_at(k + 4 + j).node * d + col, nxt[j]);
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 if (k + j < k1) {
-                    const Step st = load_step(&steps[k + j]);
+                    const Step st = step_at(k + j);
                     const T c = __ldg(coeff + st.node);
                     T e[V];
 #pragma unroll
@@ -683,7 +694,7 @@ cr_fused_ldg_kernel(const T *__restrict__ G, const T *__restrict__ coeff, const 
         T cur[4][V], nxt[4][V];
         const int gpn = m >> 2;
         int k = k0, g = 0;
-        Step st = k0 < k1 ? load_step(&steps[k0]) : Step{0, 0, 0u, 0};
+        Step st = k0 < k1 ? step_at(k0) : Step{0, 0, 0u, 0};
         if (k0 < k1) {
             const T *row = G + (size_t)st.node * m * d + col;
 #pragma unroll
@@ -698,7 +709,7 @@ cr_fused_ldg_kernel(const T *__restrict__ G, const T *__restrict__ coeff, const 
             Step sn = st;
             if (gn == gpn) {
                 gn = 0; ++kn;
-                if (kn < k1) sn = load_step(&steps[kn]);
+                if (kn < k1) sn = step_at(kn);
             }
             if (kn < k1) {
                 const T *row = G + ((size_t)sn.node * m + 4 * gn) * d + col;
@@ -722,7 +733,7 @@ cr_fused_ldg_kernel(const T *__restrict__ G, const T *__restrict__ coeff, const 
         }
     } else
     for (int k = k0; k < k1; ++k) {
-        const Step st = load_step(&steps[k]);
+        const Step st = step_at(k);
         const T *row = G + (size_t)st.node * m * d + col;
         const T *cf = coeff + (size_t)st.node * m;
         T e[V];
@@ -1355,26 +1366,33 @@ static cudaError_t run_ldg(const AggArgs &a, cudaStream_t stream) {
     const T *G = reinterpret_cast<const T *>(a.G);
     const T *cf = reinterpret_cast<const T *>(a.coeff);
     T *out = reinterpret_cast<T *>(a.out);
+    InlineSchedule inl;
+    inl.n = 0;
+    if (!a.steps) {   // single short pattern, not staged: the schedule rides in the parameters
+        if (!a.host_steps || a.batch != 1 || a.total_steps > kInlineSteps) return cudaErrorInvalidValue;
+        inl.n = a.total_steps;
+        for (int k = 0; k < a.total_steps; ++k) inl.steps[k] = a.host_steps[k];
+    }
     if (a.m % 4 == 0 && V == 4) {
         switch (pick_lmax(a.L)) {
-            case 2: cr_fused_ldg_kernel<T, 2, V, 4><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift); break;
-            case 4: cr_fused_ldg_kernel<T, 4, V, 4><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift); break;
-            default: cr_fused_ldg_kernel<T, 8, V, 4><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift); break;
+            case 2: cr_fused_ldg_kernel<T, 2, V, 4><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift, inl); break;
+            case 4: cr_fused_ldg_kernel<T, 4, V, 4><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift, inl); break;
+            default: cr_fused_ldg_kernel<T, 8, V, 4><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift, inl); break;
         }
         return cudaGetLastError();
     }
     if (a.m == 1 && V == 4) {
         switch (pick_lmax(a.L)) {
-            case 2: cr_fused_ldg_kernel<T, 2, V, 1><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift); break;
-            case 4: cr_fused_ldg_kernel<T, 4, V, 1><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift); break;
-            default: cr_fused_ldg_kernel<T, 8, V, 1><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift); break;
+            case 2: cr_fused_ldg_kernel<T, 2, V, 1><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift, inl); break;
+            case 4: cr_fused_ldg_kernel<T, 4, V, 1><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift, inl); break;
+            default: cr_fused_ldg_kernel<T, 8, V, 1><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift, inl); break;
         }
         return cudaGetLastError();
     }
     switch (pick_lmax(a.L)) {
-        case 2: cr_fused_ldg_kernel<T, 2, V, 0><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift); break;
-        case 4: cr_fused_ldg_kernel<T, 4, V, 0><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift); break;
-        default: cr_fused_ldg_kernel<T, 8, V, 0><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift); break;
+        case 2: cr_fused_ldg_kernel<T, 2, V, 0><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift, inl); break;
+        case 4: cr_fused_ldg_kernel<T, 4, V, 0><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift, inl); break;
+        default: cr_fused_ldg_kernel<T, 8, V, 0><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift, inl); break;
     }
     return cudaGetLastError();
 }
