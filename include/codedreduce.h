@@ -28,6 +28,9 @@
  *     the TMA path, anything else silently takes the plain-load kernels.
  *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Device
  *     calls only enqueue work and small async copies; they do not synchronise.
+ *     A plan is not thread-safe, and its device calls share plan-owned staging and
+ *     scratch buffers: work of one plan that may overlap on the device (two streams)
+ *     must be ordered by the caller (one stream, or events between the streams).
  *   - Every function returns a cr_status_t (CR_OK = 0) unless stated; nothing
  *     aborts or traps.  All argument and mask validation happens on the host
  *     before anything is launched.  There is no CPU fallback: device calls on a

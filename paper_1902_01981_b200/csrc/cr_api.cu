@@ -52,6 +52,7 @@ struct cr_plan {
     void *d_ones = nullptr;      // [N] the value 1 in the plan's element type (aggregation of coded gradients)
     int32_t *d_part = nullptr;   // [N*m]
     int32_t *d_order = nullptr;  // [N*m] slot items sorted by partition: launch order of the gradient kernels
+    void *d_split = nullptr;     // [n][d] scratch of the split form of short aggregations, allocated at first use
     int *d_status = nullptr;
     cr::DeviceInfo dev;
     cr::Tuning tune;
@@ -199,6 +200,7 @@ cr_status_t cr_plan_destroy(cr_plan_t *plan) {
         if (plan->d_ones) cudaFree(plan->d_ones);
         if (plan->d_part) cudaFree(plan->d_part);
         if (plan->d_order) cudaFree(plan->d_order);
+        if (plan->d_split) cudaFree(plan->d_split);
         if (plan->d_status) cudaFree(plan->d_status);
     }
     delete plan;
@@ -624,6 +626,27 @@ cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *m
     const bool prefer_plain = batch == 1 && (a.m == 1 || ((a.m == 4 || a.m == 8) && hp.d >= (1ll << 19))) &&
                               hp.d % 4 == 0 && !plan->tune.ncw && !plan->tune.stages && !plan->tune.ctas_per_sm &&
                               !plan->tune.rows;
+
+    // Short vectors under a large tree: one block per column range would walk all the consumed nodes
+    // one after the other (d = 5004 under the (12,2) tree: 132 nodes, 53 us).  The sub-trees below the
+    // master are independent until its decode, so each gets its own blocks and a second small kernel
+    // adds their weighted messages.
+    // Measured (us per call, split / TMA kernel): (12,2,1) d = 5004: 24 / 53, d = 120000: 48 / 113;
+    // with few sub-trees it does not pay: (4,3,1) d = 6500: 18.5 / 20.6, (3,4,1) d = 4096: 31 / 18.5.
+    const bool untuned = !plan->tune.ncw && !plan->tune.stages && !plan->tune.ctas_per_sm && !plan->tune.rows;
+    int subtrees = 0;
+    for (const cr::Step &st : ex.steps) subtrees += (st.layer & 0xff) == 1;
+    if (variant == CR_AGG_FUSED && untuned && batch == 1 && hp.L >= 2 && hp.d <= (1ll << 17) && subtrees >= 6 &&
+        a.total_steps >= 24 && a.total_steps <= cr::inline_schedule_limit() && subtrees <= cr::split_limit()) {
+        if (!plan->d_split) {
+            cudaError_t ea = cudaMalloc(&plan->d_split, (size_t)hp.n * (size_t)hp.d * 4);
+            if (ea != cudaSuccess) { note_cuda(ea, "cr_aggregate (split scratch)"); return CR_ERR_OOM; }
+        }
+        a.split_scratch = plan->d_split;
+        cudaError_t e0 = cr::launch_fused_ldg(a, s, &plan->launches);
+        if (e0 != cudaSuccess) { note_cuda(e0, "cr_aggregate"); return CR_ERR_CUDA; }
+        return CR_OK;
+    }
 
     // A single short pattern needs no staging: its schedule travels in the kernel parameters.
     if (variant == CR_AGG_FUSED && !prefer_plain && batch == 1 && a.total_steps <= cr::inline_schedule_limit()) {

@@ -640,8 +640,11 @@ template <> struct Loader<int, 4> {
 // PIPE = 1 (m == 1, aggregation of coded gradients): the rows of four schedule entries are requested
 // at once, and the next four before these are folded.
 // A single short schedule travels in the kernel parameters (inl.n > 0; `steps` and `pat_off` unused).
+constexpr int kMaxSplit = 16;
 struct InlineSchedule {
     int n;
+    int nseg;                      // > 0: block row b folds entries seg_off[b] .. seg_off[b+1]-1 only
+    int seg_off[kMaxSplit + 1];
     Step steps[kInlineSteps];
 };
 
@@ -653,7 +656,8 @@ cr_fused_ldg_kernel(const T *__restrict__ G, const T *__restrict__ coeff, const 
     const int b = blockIdx.y;
     const long long col = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * V;
     if (col >= d) return;
-    const int k0 = inl.n ? 0 : __ldg(&pat_off[b]), k1 = inl.n ? inl.n : __ldg(&pat_off[b + 1]);
+    const int k0 = inl.n ? (inl.nseg ? inl.seg_off[b] : 0) : __ldg(&pat_off[b]);
+    const int k1 = inl.n ? (inl.nseg ? inl.seg_off[b + 1] : inl.n) : __ldg(&pat_off[b + 1]);
     auto step_at = [&](int k) {
         if (inl.n) { Step t = inl.steps[k]; t.layer &= 0xff; return t; }
         return load_step(&steps[k]);
@@ -768,6 +772,18 @@ cr_fused_ldg_kernel(const T *__restrict__ G, const T *__restrict__ coeff, const 
 // ------------------------------------------------------------------------------------------------
 // K5: uncoded comparator -- plain sum of the same slot rows, all weights 1
 // ------------------------------------------------------------------------------------------------
+
+// out[col] = finish(sum_r rows[r][col]): the master's decode of the split form (the decode weights are
+// already applied by the sub-tree blocks).
+template <typename T>
+__global__ void __launch_bounds__(256)
+cr_sum_rows_kernel(const T *__restrict__ rows, int nrows, long long d, T *__restrict__ out, int shift) {
+    const long long col = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (col >= d) return;
+    T sum = T(0);
+    for (int r = 0; r < nrows; ++r) sum += rows[(size_t)r * d + col];
+    out[col] = finish<T>(sum, shift);
+}
 
 template <typename T, int V>
 __global__ void __launch_bounds__(256)
@@ -1360,51 +1376,79 @@ cudaError_t launch_fused_batch_tma(const AggArgs &a, const DeviceInfo &dev, cons
 }
 
 template <typename T, int V>
-static cudaError_t run_ldg(const AggArgs &a, cudaStream_t stream) {
-    const long long threads = (a.d + V - 1) / V;
-    dim3 grid((unsigned)((threads + 255) / 256), (unsigned)a.batch);
+static cudaError_t run_ldg_main(const AggArgs &a, dim3 grid, T *out, int shift, const InlineSchedule &inl, cudaStream_t stream) {
     const T *G = reinterpret_cast<const T *>(a.G);
     const T *cf = reinterpret_cast<const T *>(a.coeff);
-    T *out = reinterpret_cast<T *>(a.out);
-    InlineSchedule inl;
-    inl.n = 0;
-    if (!a.steps) {   // single short pattern, not staged: the schedule rides in the parameters
-        if (!a.host_steps || a.batch != 1 || a.total_steps > kInlineSteps) return cudaErrorInvalidValue;
-        inl.n = a.total_steps;
-        for (int k = 0; k < a.total_steps; ++k) inl.steps[k] = a.host_steps[k];
-    }
     if (a.m % 4 == 0 && V == 4) {
         switch (pick_lmax(a.L)) {
-            case 2: cr_fused_ldg_kernel<T, 2, V, 4><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift, inl); break;
-            case 4: cr_fused_ldg_kernel<T, 4, V, 4><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift, inl); break;
-            default: cr_fused_ldg_kernel<T, 8, V, 4><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift, inl); break;
+            case 2: cr_fused_ldg_kernel<T, 2, V, 4><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, shift, inl); break;
+            case 4: cr_fused_ldg_kernel<T, 4, V, 4><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, shift, inl); break;
+            default: cr_fused_ldg_kernel<T, 8, V, 4><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, shift, inl); break;
         }
         return cudaGetLastError();
     }
     if (a.m == 1 && V == 4) {
         switch (pick_lmax(a.L)) {
-            case 2: cr_fused_ldg_kernel<T, 2, V, 1><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift, inl); break;
-            case 4: cr_fused_ldg_kernel<T, 4, V, 1><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift, inl); break;
-            default: cr_fused_ldg_kernel<T, 8, V, 1><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift, inl); break;
+            case 2: cr_fused_ldg_kernel<T, 2, V, 1><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, shift, inl); break;
+            case 4: cr_fused_ldg_kernel<T, 4, V, 1><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, shift, inl); break;
+            default: cr_fused_ldg_kernel<T, 8, V, 1><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, shift, inl); break;
         }
         return cudaGetLastError();
     }
     switch (pick_lmax(a.L)) {
-        case 2: cr_fused_ldg_kernel<T, 2, V, 0><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift, inl); break;
-        case 4: cr_fused_ldg_kernel<T, 4, V, 0><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift, inl); break;
-        default: cr_fused_ldg_kernel<T, 8, V, 0><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, a.shift, inl); break;
+        case 2: cr_fused_ldg_kernel<T, 2, V, 0><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, shift, inl); break;
+        case 4: cr_fused_ldg_kernel<T, 4, V, 0><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, shift, inl); break;
+        default: cr_fused_ldg_kernel<T, 8, V, 0><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, shift, inl); break;
     }
     return cudaGetLastError();
 }
 
-cudaError_t launch_fused_ldg(const AggArgs &a, cudaStream_t stream, int64_t *launches) {
-    const bool v4 = vec4_ok(a.G, a.out, a.d);
-    cudaError_t err;
-    if (a.is_int) err = v4 ? run_ldg<int, 4>(a, stream) : run_ldg<int, 1>(a, stream);
-    else err = v4 ? run_ldg<float, 4>(a, stream) : run_ldg<float, 1>(a, stream);
-    if (err == cudaSuccess) ++*launches;
+
+template <typename T, int V>
+static cudaError_t run_ldg(const AggArgs &a, cudaStream_t stream, int64_t *launches) {
+    const long long threads = (a.d + V - 1) / V;
+    dim3 grid((unsigned)((threads + 255) / 256), (unsigned)a.batch);
+    T *out = reinterpret_cast<T *>(a.out);
+    InlineSchedule inl;
+    inl.n = 0; inl.nseg = 0;
+    int shift = a.shift;
+    if (!a.steps) {   // single short pattern, not staged: the schedule rides in the parameters
+        if (!a.host_steps || a.batch != 1 || a.total_steps > kInlineSteps) return cudaErrorInvalidValue;
+        inl.n = a.total_steps;
+        for (int k = 0; k < a.total_steps; ++k) inl.steps[k] = a.host_steps[k];
+        if (a.split_scratch) {
+            // post-order: the entries of a layer-1 sub-tree are contiguous and end with its root
+            inl.seg_off[0] = 0;
+            for (int k = 0; k < a.total_steps; ++k)
+                if ((a.host_steps[k].layer & 0xff) == 1) {
+                    if (inl.nseg == kMaxSplit) return cudaErrorInvalidValue;
+                    inl.seg_off[++inl.nseg] = k + 1;
+                }
+            if (inl.nseg == 0 || inl.seg_off[inl.nseg] != a.total_steps) return cudaErrorInvalidValue;
+            grid.y = (unsigned)inl.nseg;
+            out = reinterpret_cast<T *>(a.split_scratch);
+            shift = 0;   // applied once, by the kernel that adds the rows
+        }
+    }
+    cudaError_t err = run_ldg_main<T, V>(a, grid, out, shift, inl, stream);
+    if (err != cudaSuccess) return err;
+    ++*launches;
+    if (inl.nseg) {
+        cr_sum_rows_kernel<T><<<(unsigned)((a.d + 255) / 256), 256, 0, stream>>>(reinterpret_cast<const T *>(a.split_scratch), inl.nseg,
+                                                                             a.d, reinterpret_cast<T *>(a.out), a.shift);
+        err = cudaGetLastError();
+        if (err == cudaSuccess) ++*launches;
+    }
     return err;
 }
+
+cudaError_t launch_fused_ldg(const AggArgs &a, cudaStream_t stream, int64_t *launches) {
+    const bool v4 = vec4_ok(a.G, a.out, a.d) && (!a.split_scratch || aligned16(a.split_scratch));
+    if (a.is_int) return v4 ? run_ldg<int, 4>(a, stream, launches) : run_ldg<int, 1>(a, stream, launches);
+    return v4 ? run_ldg<float, 4>(a, stream, launches) : run_ldg<float, 1>(a, stream, launches);
+}
+
+int split_limit() { return kMaxSplit; }
 
 template <typename T, int V>
 static cudaError_t run_uncoded(const AggArgs &a, cudaStream_t stream) {

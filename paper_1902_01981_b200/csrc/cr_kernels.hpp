@@ -58,6 +58,8 @@ struct AggArgs {
     int *status;          // device status word (bounded waits)
     int is_int;
     int same_shape;       // batch > 1: all patterns' schedules share length and layer sequence
+    void *split_scratch = nullptr;  // launch_fused_ldg, single inline schedule: [n][d] scratch; when set, the
+                                    // sub-trees below the master run as separate blocks (see launch_fused_ldg)
 };
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -74,7 +76,13 @@ cudaError_t launch_fused_tma(const AggArgs &a, const DeviceInfo &dev, const Tuni
                              cudaStream_t stream, int64_t *launches, bool *done);
 cudaError_t launch_fused_batch_tma(const AggArgs &a, const DeviceInfo &dev, const Tuning &tune, EncodeTiledFn encode,
                                    cudaStream_t stream, int64_t *launches, bool *done);
+// With a.split_scratch the schedule of a single pattern is cut at the master's children: every layer-1
+// sub-tree is folded by its own blocks into a row of the scratch, and a second small kernel adds the
+// rows (the master's decode).  For short vectors, where one block per column range would walk all the
+// nodes of a large tree one after the other.
 cudaError_t launch_fused_ldg(const AggArgs &a, cudaStream_t stream, int64_t *launches);
+// Largest number of sub-trees below the master that the split form handles (= largest n).
+int split_limit();
 cudaError_t launch_uncoded_sum(const AggArgs &a, cudaStream_t stream, int64_t *launches);
 
 // E[v][:] = sum_j coeff[v*m+j] * G[v*m+j][:] for the nodes listed in `nodes` (device, count entries) or
