@@ -82,3 +82,38 @@ def test_library_matches_oracle(n, L, s, code):
             B.cr_latency_masks(plan, -np.ones(N), 0.1)
     finally:
         B.cr_plan_destroy(plan)
+
+
+@pytest.mark.parametrize("n,L,s", [(4, 2, 1), (12, 2, 3), (6, 3, 2)])
+def test_communication_term_lies_between_the_bounds_of_theorem_2(n, L, s):
+    """With instant computations the run time is pure communication: every parent hears n-s messages
+    one after the other, layer after layer: T = L (n-s) t_c.  Theorem 2's communication terms bracket
+    it: (n(1-alpha) + L - 1) t_c from below (the master's n-s receptions after one message per lower
+    layer), n L t_c from above."""
+    t_c = 0.25
+    N = O.num_nodes(n, L)
+    masks, T = O.latency_trial(n, L, s, np.zeros(N), t_c)
+    assert T == pytest.approx(L * (n - s) * t_c)
+    assert (n - s + L - 1) * t_c <= T <= n * L * t_c
+    # the stragglers are then the highest-indexed s children of every group (ties: lower index first)
+    assert all(m == sum(1 << j for j in range(n - s, n)) for m in masks)
+
+
+def test_expected_run_time_against_theorem_2_at_finite_n():
+    """E[T_CR] sampled on the (12,2) tree with alpha = 1/4.  Theorem 2's computation term, with the exact
+    order-statistic mean (H_n - H_s) of Appendix D in place of its limit log(1/alpha), plus one message
+    time bounds it from below (the master waits for the (n-s)-th of its children, whose own
+    computations alone take that long, and then receives a message); the expected slowest of all N
+    computations plus the theorem's n L t_c bounds it from above."""
+    n, L, s, a, mu, t_c = 12, 2, 3, 1e-3, 1.0, 0.05
+    P = O.partition_quantum(n, L, s)
+    load = O.computation_load(n, L, s) * P            # data units per worker, r_CR * d
+    N = O.num_nodes(n, L)
+    times = inputs.shifted_exponential_times(N, load, a, mu, seed=5, trials=3000)
+    mean_T = float(np.mean([O.latency_trial(n, L, s, t, t_c)[1] for t in times]))
+    stat_err = 4.0 * (load / mu) / np.sqrt(3000)      # four standard errors of a sample mean, generously
+    assert O.expected_order_statistic(n, s, load, a, mu) + t_c <= mean_T + stat_err
+    assert mean_T <= O.expected_order_statistic(N, 0, load, a, mu) + n * L * t_c + stat_err
+    # and the communication share is of the order the theorem states: between (n-s) and n L message times
+    no_comm = float(np.mean([O.latency_trial(n, L, s, t, 0.0)[1] for t in times]))
+    assert t_c <= mean_T - no_comm <= n * L * t_c
