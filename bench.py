@@ -349,7 +349,9 @@ def run_ours(args, cfg):
         e2e_units = float(sum(step_bytes[(args.warmup + i) % total] for i in range(e2e_steps)))
         e2e_elapsed, e2e_units = combine_ranks(e2e_elapsed, e2e_units, world, dist, dev)
         e2e = {"value": e2e_units / e2e_elapsed / 1e9, "unit": UNIT,
-               "h2d_bytes_per_step": int(N * m * d * 4 + masks[0].nbytes), "d2h_bytes_per_step": int(batch * d * 4),
+               # cr_aggregate_host sends the slots of the consumed nodes only (stragglers are not waited for)
+               "h2d_bytes_per_step": int(e2e_units / e2e_steps / world - batch * d * 4 + masks[0].nbytes),
+               "d2h_bytes_per_step": int(batch * d * 4),
                "steps": e2e_steps, "ms_per_step": e2e_elapsed / e2e_steps * 1e3}
         del host_slots
 

@@ -266,9 +266,12 @@ size_t cr_aggregate_workspace_bytes(const cr_plan_t *plan, int32_t batch, uint32
 cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *masks_host, int32_t batch,
                          void *g_out, uint32_t flags, void *workspace, size_t workspace_bytes, void *stream);
 
-/* Same computation with HOST buffers: copies G_slots_host (pinned or pageable host memory,
- * [N][m][d]) into dev_slots, runs cr_aggregate, copies the result into g_out_host and waits for the
- * stream.  dev_slots [N][m][d] and dev_out [batch][d] are caller-owned device staging buffers. */
+/* Same computation with HOST buffers: copies from G_slots_host (pinned or pageable host memory,
+ * [N][m][d]) into dev_slots the slots of the nodes that the batch consumes (the rest of dev_slots is
+ * left as it is: a straggler's data is never waited for; all nodes with CR_AGG_ALL_NODES), runs
+ * cr_aggregate, copies the result into g_out_host and waits for the stream.  dev_slots [N][m][d] and
+ * dev_out [batch][d] are caller-owned device staging buffers.  The bytes that cross the bus are those
+ * of cr_aggregate_bytes. */
 cr_status_t cr_aggregate_host(cr_plan_t *plan, const void *G_slots_host, const uint32_t *masks_host,
                               int32_t batch, void *g_out_host, uint32_t flags, void *dev_slots,
                               void *dev_out, void *workspace, size_t workspace_bytes, void *stream);

@@ -707,9 +707,33 @@ cr_status_t cr_aggregate_host(cr_plan_t *plan, const void *G_slots_host, const u
     if (st != CR_OK) return st;
     if (!G_slots_host || !g_out_host || !dev_slots || !dev_out || batch < 1) return CR_ERR_INVALID_ARG;
     cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
-    const size_t in_bytes = (size_t)plan->hp.N * plan->hp.m * (size_t)plan->hp.d * 4;
     const size_t out_bytes = (size_t)batch * (size_t)plan->hp.d * 4;
-    CR_CUDA(cudaMemcpyAsync(dev_slots, G_slots_host, in_bytes, cudaMemcpyHostToDevice, s));
+    // Only the slots of the nodes that some pattern of the batch consumes cross the bus: what a
+    // straggler holds is never waited for.  (One copy per run of consecutive used nodes.)
+    const bool from_coded = (flags & CR_AGG_FROM_CODED) != 0;
+    const size_t node_bytes = (from_coded ? (size_t)1 : (size_t)plan->hp.m) * (size_t)plan->hp.d * 4;
+    if (flags & CR_AGG_ALL_NODES) {
+        CR_CUDA(cudaMemcpyAsync(dev_slots, G_slots_host, node_bytes * plan->hp.N, cudaMemcpyHostToDevice, s));
+    } else {
+        if (!masks_host) return CR_ERR_INVALID_ARG;
+        std::vector<char> used((size_t)plan->hp.N, 0);
+        std::vector<cr::UsedNode> one;
+        for (int b = 0; b < batch; ++b) {
+            one.clear();
+            st = plan->hp.expand(masks_host + (size_t)b * plan->hp.groups, one);
+            if (st != CR_OK) return st;
+            for (const cr::UsedNode &u : one) used[u.node] = 1;
+        }
+        for (int v = 0; v < plan->hp.N;) {
+            if (!used[v]) { ++v; continue; }
+            int w = v;
+            while (w < plan->hp.N && used[w]) ++w;
+            CR_CUDA(cudaMemcpyAsync(static_cast<unsigned char *>(dev_slots) + node_bytes * v,
+                                    static_cast<const unsigned char *>(G_slots_host) + node_bytes * v,
+                                    node_bytes * (size_t)(w - v), cudaMemcpyHostToDevice, s));
+            v = w;
+        }
+    }
     st = cr_aggregate(plan, dev_slots, masks_host, batch, dev_out, flags, workspace, workspace_bytes, stream);
     if (st != CR_OK) return st;
     CR_CUDA(cudaMemcpyAsync(g_out_host, dev_out, out_bytes, cudaMemcpyDeviceToHost, s));

@@ -286,3 +286,45 @@ def test_device_error_paths():
         assert B.cr_plan_launch_count(plan) > 0
     finally:
         B.cr_plan_destroy(plan)
+
+
+@pytest.mark.parametrize("from_coded", [False, True])
+def test_host_buffer_entry_point_sends_only_consumed_nodes(from_coded):
+    """cr_aggregate_host: the device staging buffer starts full of NaN; the call must bring over every
+    slot that the patterns consume (the result is right) and nothing of the stragglers' nodes (their
+    rows stay NaN)."""
+    cfg = tree(4, 2, 1, "cyclic", 1536)
+    n, L, s, d = cfg["n"], cfg["L"], cfg["s"], cfg["d"]
+    plan = make_plan(cfg)
+    try:
+        code, local = check_slot_table(plan, cfg)
+        N, m = B.cr_plan_num_nodes(plan), B.cr_plan_load(plan)
+        G = inputs.partition_gradients(cfg["P"], d, seed=13)
+        part = B.slot_partitions(plan)
+        if from_coded:
+            host = torch.from_numpy(O.encode_all(local, G).astype(np.float32)).pin_memory()   # E [N][d]
+            rows_per_node = 1
+        else:
+            host = torch.from_numpy(G[part.reshape(-1)]).pin_memory()                         # [N*m][d]
+            rows_per_node = m
+        masks = inputs.straggler_masks(n, L, s, 3, seed=6, exactly_s=True)
+        dev = torch.full((N * rows_per_node, d), float("nan"), device="cuda")
+        dev_out = torch.zeros((3, d), device="cuda")
+        host_out = torch.zeros((3, d)).pin_memory()
+        flags = B.CR_AGG_FUSED | (B.CR_AGG_FROM_CODED if from_coded else 0)
+        B.cr_aggregate_host(plan, host, masks, host_out, dev, dev_out, flags)
+        used = set()
+        for b in range(3):
+            used |= set(O.used_nodes(code, masks[b]))
+            bar = REL_L2_BAR if not from_coded else 1e-5
+            assert rel_l2(host_out[b].numpy(), O.execute(code, local, G, masks[b])) <= bar
+        assert len(used) < N
+        got = dev.cpu().numpy().reshape(N, rows_per_node, d)
+        for v in range(N):
+            assert np.isnan(got[v]).all() != (v in used), v
+            if v in used:
+                assert np.array_equal(got[v], host.numpy().reshape(N, rows_per_node, d)[v])
+        nbytes, n_used = B.cr_aggregate_bytes(plan, masks)
+        assert n_used == len(used)
+    finally:
+        B.cr_plan_destroy(plan)
