@@ -113,7 +113,11 @@ def test_every_pattern_on_tiny_trees(cfg, flags):
 
 @pytest.mark.parametrize("cfg,batch", [(tree(4, 2, 1, "cyclic", 1 << 15), 9), (tree(5, 2, 2, "cyclic", 70000, P=80), 5),
                                        (tree(3, 4, 1, "printed_3_1", 5000), 64), (tree(4, 3, 1, "cyclic", 4100), 7),
-                                       (tree(2, 5, 0, "cyclic", 1000), 2), (tree(12, 2, 3, "cyclic", 1200, max_kappa=1e6), 3)])
+                                       (tree(2, 5, 0, "cyclic", 1000), 2), (tree(12, 2, 3, "cyclic", 1200, max_kappa=1e6), 3),
+                                       # the limits of the interface: deepest tree (L = 8, m = 256 slots per node, and
+                                       # m = 1 without redundancy), widest parents (n = 16)
+                                       (tree(2, 8, 1, "cyclic", 300), 3), (tree(2, 8, 0, "cyclic", 2052), 2),
+                                       (tree(16, 2, 1, "repetition", 520), 4), (tree(16, 1, 3, "repetition", 4096), 5)])
 @pytest.mark.parametrize("flags", FUSED_VARIANTS)
 def test_random_patterns_medium_trees(cfg, batch, flags):
     n, L, s, d = cfg["n"], cfg["L"], cfg["s"], cfg["d"]
