@@ -37,9 +37,9 @@ FALLBACK_HBM_GBS = 6650.0
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the timed kernel, from the ncu capture
 # summarised under profiles/ (absent = no capture of the current kernel on that workload).
-# cfg4: 917.4 MB measured at d = 2^21, scaled by 8 to d = 2^24 (traffic is proportional to d).
-# cfg5: 2083.3 MB measured at d = 2^18, scaled by 16 to d = 2^22.
-NCU_TRAFFIC_BYTES = {("cfg4", "f32", 1 << 24): 8 * 917.37e6, ("cfg5", "f32", 1 << 22): 16 * 2083.3e6}
+# cfg4: 917.3 MB measured at d = 2^21, scaled by 8 to d = 2^24 (traffic is proportional to d).
+# cfg5: 2083.8 MB measured at d = 2^18, scaled by 16 to d = 2^22.
+NCU_TRAFFIC_BYTES = {("cfg4", "f32", 1 << 24): 8 * 917.26e6, ("cfg5", "f32", 1 << 22): 16 * 2083.8e6}
 
 
 def peak_hbm():
@@ -127,6 +127,23 @@ class ClockSampler:
         return out
 
 
+class L2Flush:
+    """Pushes the workload's data out of L2 between timed steps: writes one 256 MB buffer (twice the L2),
+    then reads a second one.  The read pass matters: after the write alone L2 is left full of dirty lines,
+    and the timed launch that follows would pay for their write-back (it shows as DRAM write traffic
+    inside a read-only kernel)."""
+
+    def __init__(self, torch, device):
+        self.torch = torch
+        self.wbuf = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+        self.rbuf = torch.zeros(64 << 20, dtype=torch.int32, device=device)
+        self.sink = torch.zeros((), dtype=torch.int64, device=device)
+
+    def __call__(self, i: int):
+        self.wbuf.fill_(i & 0xff)
+        self.torch.sum(self.rbuf, out=self.sink)
+
+
 # ----------------------------------------------------------------------------- CPU oracle legs
 
 def oracle_sample(cfg, d_sample: int, steps: int, warmup: int, G=None):
@@ -197,12 +214,80 @@ def run_reference(args, cfg):
     print(json.dumps(line), flush=True)
 
 
+def oracle_regression_sample(workload, cfg, steps, warmup, seconds):
+    """Times the oracle's gradient-descent step on a regression workload: per step the fp64 partial
+    gradients of a bounded sample of the partitions (the definition, once per partition), CR.Execute over
+    all of them under a fresh straggler pattern, and the model update.  The sample is sized from the first
+    full gradient pass so that all steps take about `seconds`.
+    Returns (seconds per step, algorithmic bytes per step, description of the sample)."""
+    from oracle import cr_oracle as O
+    from oracle import cr_setup
+    code, local, _ = cr_setup.setup(cfg)
+    n, L, s, P, d, rows = cfg["n"], cfg["L"], cfg["s"], cfg["P"], cfg["d"], cfg["rows"]
+    logistic = cfg["kind"] == "logistic"
+    if logistic:
+        X, y, _ = inputs.logistic_partitions(P, rows, d, cfg["seed"], cfg["x_std"])
+    else:
+        X, y, _ = inputs.linreg_partitions(P, rows, d, cfg["seed"], cfg["x_std"], cfg["noise_std"])
+    grad = O.partial_gradient_logistic if logistic else O.partial_gradient_linreg
+    N, m = O.num_nodes(n, L), len(local[0])
+    w = np.zeros(d, dtype=np.float32)
+    total = steps + warmup
+    masks = inputs.straggler_masks(n, L, s, total, cfg.get("mask_seed", 1))
+    lr_eff = cfg["lr"] if workload == "cfg1" else cfg["lr"] / P
+    t0 = time.perf_counter()
+    G = np.stack([grad(X[p], y[p], w) for p in range(P)])
+    per_partition = (time.perf_counter() - t0) / P
+    sampled = int(min(P, max(1, seconds / total / per_partition)))
+    times, nbytes = [], []
+    for it in range(total):
+        t0 = time.perf_counter()
+        for p in range(sampled):
+            q = (it * sampled + p) % P
+            G[q] = grad(X[q], y[q], w)
+        g = O.execute(code, local, G, masks[it])
+        w = (w.astype(np.float64) - lr_eff * g).astype(np.float32)
+        dt = time.perf_counter() - t0
+        if it >= warmup:
+            times.append(dt)
+            # the workload's own count: every (node, slot) item reads its partition; scaled to the sample
+            nbytes.append(4.0 * rows * d * N * m * sampled / P + 4.0 * d * (m * len(O.used_nodes(code, masks[it])) + 1))
+    sample = (f"gradients of {sampled} of {P} partitions per step (each computed once, not once per slot), "
+              f"aggregation of all {P}, {steps} steps, NumPy fp64")
+    return float(np.mean(times)), float(np.mean(nbytes)), sample
+
+
+def regression_workload_name(workload, cfg):
+    return (f"{workload}: {'logistic' if cfg['kind'] == 'logistic' else 'linear'} regression n={cfg['n']} L={cfg['L']} "
+            f"s={cfg['s']} P={cfg['P']} rows={cfg['rows']} d={cfg['d']}")
+
+
+def run_reference_regression(args, cfg):
+    """The oracle as the reference arm of a regression workload (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    sec, nbytes, sample = oracle_regression_sample(args.workload, cfg, args.steps, args.warmup, 60.0)
+    value = nbytes / sec / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": regression_workload_name(args.workload, cfg)},
+        "iterations_per_s": 1.0 / sec,
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
+                         "host_threads_available": host_threads()},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
 # ----------------------------------------------------------------------------- our arm
 
 def workload_config(name, cfg, extra):
     out = {"workload": f"{name}: n={cfg['n']} L={cfg['L']} s={cfg['s']} code={cfg['code']} P={cfg['P']} "
                        f"d={cfg['d']} batch={cfg.get('batch', 1)}",
-           "l2": "inputs larger than L2 (no flush needed)" if cfg["d"] * 4 * cfg["P"] > 126e6 else "L2 flushed between steps",
+           "l2": "inputs larger than L2 (no flush needed)" if cfg["d"] * 4 * cfg["P"] > 126e6 else "L2 flushed between steps (256 MB written, then 256 MB read)",
            "parallelism": "independent replicas (no exchange step)"}
     if extra:
         out.update(extra)
@@ -260,7 +345,7 @@ def run_ours(args, cfg):
                                    cfg.get("exactly_s", False)).reshape(total, batch, groups)
     step_bytes = [B.cr_aggregate_bytes(plan, masks[i])[0] for i in range(total)]
     need_flush = d * 4 * cfg["P"] <= 126e6
-    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if need_flush else None
+    flush_buf = L2Flush(torch, dev) if need_flush else None
     stream = torch.cuda.current_stream()
 
     def timed_run(flags, ws=None, steps=args.steps, warmup=args.warmup):
@@ -276,7 +361,7 @@ def run_ours(args, cfg):
         n0 = B.cr_plan_launch_count(plan)
         for i in range(steps):
             if flush_buf is not None:
-                flush_buf.fill_(i & 0xff)
+                flush_buf(i)
             starts[i].record(stream)
             B.cr_aggregate(plan, G_slots, masks[(warmup + i) % total], out, flags, ws, stream)
             stops[i].record(stream)
@@ -431,7 +516,7 @@ def run_linreg(args, cfg):
     total = min(args.steps + args.warmup, 256)
     masks = inputs.straggler_masks(n, L, s, total, cfg.get("mask_seed", 1))
     lr_eff = cfg["lr"] if args.workload == "cfg1" else cfg["lr"] / P
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if X.nbytes <= 126e6 else None
+    flush = L2Flush(torch, "cuda") if X.nbytes <= 126e6 else None
     stream = torch.cuda.current_stream()
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
 
@@ -461,7 +546,7 @@ def run_linreg(args, cfg):
     t0 = time.time()
     for i in range(args.steps):
         if flush is not None:
-            flush.fill_(i & 0xff)
+            flush(i)
         step(args.warmup + i, ev[i])
     torch.cuda.synchronize()
     t1 = time.time()
@@ -477,6 +562,28 @@ def run_linreg(args, cfg):
     peak, peak_kind = peak_hbm()
     achieved = grad_bytes / float(t_grad.mean()) / 1e9
     w_final = w_dev.cpu().numpy()
+    # end to end: the data set stays resident (it does not change between steps); the model goes up from
+    # pinned host memory and the aggregated gradient comes back, every step, and the host applies the update
+    e2e = None
+    if not args.no_e2e:
+        e2e_steps = max(1, min(args.steps, 50))
+        w_host = torch.zeros(d, pin_memory=True)
+        g_host = torch.zeros(d, pin_memory=True)
+        t0 = time.perf_counter()
+        for i in range(e2e_steps):
+            w_dev.copy_(w_host, non_blocking=True)
+            step(i)
+            g_host.copy_(out[0], non_blocking=True)
+            torch.cuda.synchronize()
+            w_host.sub_(g_host, alpha=lr_eff)
+        e2e_sec = (time.perf_counter() - t0) / e2e_steps
+        e2e = {"value": step_bytes / e2e_sec / 1e9, "unit": UNIT, "h2d_bytes_per_step": int(4 * d + masks[0].nbytes),
+               "d2h_bytes_per_step": int(4 * d), "steps": e2e_steps, "ms_per_step": e2e_sec * 1e3}
+    cpu = None
+    if not args.no_cpu_baseline:
+        sec, nbytes, sample = oracle_regression_sample(args.workload, cfg, args.cpu_steps, 1, 15.0)
+        cpu = {"value": nbytes / sec / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
+               "ms_per_step_on_sample": sec * 1e3, "host_threads_available": host_threads()}
     line = {
         "metric": METRIC, "value": step_bytes * args.steps / elapsed / 1e9, "unit": UNIT, "n_gpus": 1,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": elapsed / args.steps * 1e3,
@@ -485,13 +592,13 @@ def run_linreg(args, cfg):
                                f"P={P} rows={rows} d={d}, step = "
                                + ("coded gradients of all N nodes (slot gradients never written)" if coded
                                   else "partial gradients of all N*m slots") + " + fused aggregation + model update",
-                   "l2": "inputs larger than L2 (no flush needed)" if flush is None else "L2 flushed between steps"},
+                   "l2": "inputs larger than L2 (no flush needed)" if flush is None else "L2 flushed between steps (256 MB written, then 256 MB read)"},
         "iterations_per_s": args.steps / elapsed,
         "roofline": {"bound": "hbm", "kernel": "partial gradients", "achieved": achieved, "peak": peak, "unit": "GB/s",
                      "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
                      "algorithmic_bytes_per_launch": grad_bytes, "avg_launch_ms": float(t_grad.mean()) * 1e3,
                      "aggregate_ms": float((t_step - t_grad).mean()) * 1e3},
-        "cpu_baseline": None, "e2e": None, "gpu_launches": int(launches), "clocks": clocks,
+        "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
         "normalized_error_rate": float(np.sum((w_final - w_star) ** 2) / np.sum(w_star ** 2)),
     }
     print(json.dumps(line), flush=True)
@@ -525,14 +632,14 @@ def run_multi(args, cfg):
     G = torch.zeros((K, N, m, d), device="cuda")
     ws = torch.empty(B.cr_partial_gradients_multi_workspace_bytes(plan, rows), dtype=torch.uint8, device="cuda")
     ws1 = torch.empty(max(16, B.cr_partial_gradients_workspace_bytes(plan, rows)), dtype=torch.uint8, device="cuda")
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if X.nbytes <= 126e6 else None
+    flush = L2Flush(torch, "cuda") if X.nbytes <= 126e6 else None
     stream = torch.cuda.current_stream()
 
     def timed(fn, steps):
         ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(steps)]
         for i in range(steps):
             if flush is not None:
-                flush.fill_(i & 0xff)
+                flush(i)
             ev[i][0].record(stream)
             fn()
             ev[i][1].record(stream)
@@ -572,7 +679,7 @@ def run_multi(args, cfg):
         "data": "synthetic",
         "config": {"workload": f"{args.workload}: partial gradients of K={K} models, n={n} L={L} s={s} P={P} rows={rows} "
                                f"d={d} ({items} slot items), X TF32-representable",
-                   "l2": "inputs larger than L2 (no flush needed)" if flush is None else "L2 flushed between steps"},
+                   "l2": "inputs larger than L2 (no flush needed)" if flush is None else "L2 flushed between steps (256 MB written, then 256 MB read)"},
         "roofline": {"bound": "hbm", "kernel": "cr_tc_residual_kernel + cr_tc_gradient_kernel", "achieved": achieved,
                      "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
                      "traffic": None, "algorithmic_bytes_per_launch": nbytes, "avg_launch_ms": sec * 1e3,
@@ -615,7 +722,7 @@ def main():
         args.gpus = world
     if cfg["kind"] in ("linreg", "logistic"):
         if args.impl == "reference":
-            print(json.dumps({"impl": "reference", "unavailable": "the reference arm times aggregation workloads only"}))
+            run_reference_regression(args, cfg)
         elif args.models:
             run_multi(args, cfg)
         else:
