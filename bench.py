@@ -141,7 +141,7 @@ class L2Flush:
 
     def __call__(self, i: int):
         self.wbuf.fill_(i & 0xff)
-        self.torch.sum(self.rbuf, out=self.sink)
+        self.torch.sum(self.rbuf, (0,), out=self.sink)
 
 
 # ----------------------------------------------------------------------------- CPU oracle legs
@@ -385,6 +385,7 @@ def run_ours(args, cfg):
     sampler.wait_first_sample()
     per, wall = timed_run(B.CR_AGG_FUSED)
     launches = timed_run.launches
+    timed_kernel = B.cr_plan_last_kernel(plan)
     clocks = sampler.stop(timed_run.window)
     assert B.cr_plan_device_status(plan) == B.CR_OK, "a device-side wait timed out"
     # device time of the K steps: first start event to last stop event on the launching stream (with
@@ -445,10 +446,8 @@ def run_ours(args, cfg):
         avg_launch = float(per.mean())
         avg_bytes = units / args.steps
         achieved = avg_bytes / avg_launch / 1e9
-        # single patterns over m = 4 or 8 trees are routed to the plain-load kernel (small TMA boxes cannot keep up)
-        kern = ("cr_fused_batch_tma_kernel" if batch > 1 else
-                "cr_fused_ldg_kernel" if (m in (4, 8) and d >= (1 << 19) and not args.tune) else "cr_fused_tma_kernel")
-        traffic = NCU_TRAFFIC_BYTES.get((args.workload, args.dtype, d))
+        kern = timed_kernel
+        traffic = NCU_TRAFFIC_BYTES.get((args.workload, args.dtype, d)) if not args.tune else None
         roofline = {"bound": "hbm", "kernel": kern, "achieved": achieved, "peak": peak, "unit": "GB/s",
                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / 8000.0,
                     "traffic": traffic, "algorithmic_bytes_per_launch": avg_bytes,

@@ -306,6 +306,10 @@ cr_status_t cr_plan_tune_items(cr_plan_t *plan, int32_t item_order, int32_t mult
 /* Kernel launches enqueued by this plan's device calls so far. */
 int64_t cr_plan_launch_count(const cr_plan_t *plan);
 
+/* Name of the kernel (family) that served this plan's latest cr_aggregate call; "" before the first.
+ * The string is static storage owned by the library. */
+const char *cr_plan_last_kernel(const cr_plan_t *plan);
+
 #ifdef __cplusplus
 }
 #endif

@@ -86,6 +86,7 @@ _SIGNATURES = {
     "cr_plan_tune_gradients": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32, C.c_int32]),
     "cr_plan_tune_items": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32]),
     "cr_plan_launch_count": (C.c_int64, [C.c_void_p]),
+    "cr_plan_last_kernel": (C.c_char_p, [C.c_void_p]),
 }
 
 
@@ -189,6 +190,10 @@ def cr_plan_int_scale(plan: int) -> int:
 
 def cr_plan_launch_count(plan: int) -> int:
     return lib().cr_plan_launch_count(plan)
+
+
+def cr_plan_last_kernel(plan: int) -> str:
+    return lib().cr_plan_last_kernel(plan).decode()
 
 
 def cr_plan_get_B(plan: int, level: int, n: int):

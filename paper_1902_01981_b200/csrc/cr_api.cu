@@ -45,6 +45,11 @@ size_t align16(size_t x) { return (x + 15) & ~(size_t)15; }
 
 }  // namespace
 
+// The split form of short aggregations (cr_aggregate): vectors of at most this length, under trees whose
+// master has at least this many children.
+constexpr long long kSplitMaxD = 1ll << 17;
+constexpr int kSplitMinSubtrees = 6;
+
 struct cr_plan {
     cr::HostPlan hp;
     int device = -1;
@@ -52,7 +57,8 @@ struct cr_plan {
     void *d_ones = nullptr;      // [N] the value 1 in the plan's element type (aggregation of coded gradients)
     int32_t *d_part = nullptr;   // [N*m]
     int32_t *d_order = nullptr;  // [N*m] slot items sorted by partition: launch order of the gradient kernels
-    void *d_split = nullptr;     // [n][d] scratch of the split form of short aggregations, allocated at first use
+    void *d_split = nullptr;     // [n][d] scratch of the split form of short aggregations (plans that can take it)
+    const char *last_kernel = "";  // kernel that served the latest cr_aggregate call
     int *d_status = nullptr;
     cr::DeviceInfo dev;
     cr::Tuning tune;
@@ -259,6 +265,10 @@ cr_status_t cr_plan_create(const cr_plan_desc_t *desc, cr_plan_t **out) {
             CR_CUDA_P(cudaMemcpy(p->d_order, order.data(), slots * 4, cudaMemcpyHostToDevice));
         }
         CR_CUDA_P(cudaMemset(p->d_status, 0, sizeof(int)));
+        // scratch of the split form of short aggregations under wide trees (see cr_aggregate): reserved
+        // here, so that no device call ever allocates
+        if (p->hp.L >= 2 && p->hp.d <= kSplitMaxD && p->hp.n >= kSplitMinSubtrees && p->hp.n <= cr::split_limit())
+            CR_CUDA_P(cudaMalloc(&p->d_split, (size_t)p->hp.n * (size_t)p->hp.d * 4));
         // cuTensorMapEncodeTiled through the runtime, so that the library needs no link to libcuda
         void *fn = nullptr;
         cudaDriverEntryPointQueryResult qres;
@@ -278,6 +288,7 @@ int32_t cr_plan_num_groups(const cr_plan_t *plan) { return plan ? plan->hp.group
 int32_t cr_plan_load(const cr_plan_t *plan) { return plan ? plan->hp.m : -1; }
 int64_t cr_plan_int_scale(const cr_plan_t *plan) { return plan ? plan->hp.int_scale : -1; }
 int64_t cr_plan_launch_count(const cr_plan_t *plan) { return plan ? plan->launches : -1; }
+const char *cr_plan_last_kernel(const cr_plan_t *plan) { return plan ? plan->last_kernel : ""; }
 
 cr_status_t cr_plan_tune(cr_plan_t *plan, int32_t consumer_warps, int32_t stages, int32_t ctas_per_sm, int32_t rows_per_box) {
     if (!plan || consumer_warps < 0 || stages < 0 || ctas_per_sm < 0 || rows_per_box < 0) return CR_ERR_INVALID_ARG;
@@ -592,6 +603,7 @@ cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *m
 
     if (variant == CR_AGG_UNFUSED) {
         if (!workspace || workspace_bytes < cr_aggregate_workspace_bytes(plan, batch, flags)) return CR_ERR_OOM;
+        plan->last_kernel = "cr_encode_kernel + cr_decode_kernel per level";
         return aggregate_unfused(plan, G_slots, masks_host, batch, g_out, (flags & CR_AGG_ALL_NODES) != 0, workspace, ex, s);
     }
 
@@ -636,15 +648,12 @@ cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *m
     const bool untuned = !plan->tune.ncw && !plan->tune.stages && !plan->tune.ctas_per_sm && !plan->tune.rows;
     int subtrees = 0;
     for (const cr::Step &st : ex.steps) subtrees += (st.layer & 0xff) == 1;
-    if (variant == CR_AGG_FUSED && untuned && batch == 1 && hp.L >= 2 && hp.d <= (1ll << 17) && subtrees >= 6 &&
+    if (variant == CR_AGG_FUSED && untuned && batch == 1 && plan->d_split && subtrees >= kSplitMinSubtrees &&
         a.total_steps >= 24 && a.total_steps <= cr::inline_schedule_limit() && subtrees <= cr::split_limit()) {
-        if (!plan->d_split) {
-            cudaError_t ea = cudaMalloc(&plan->d_split, (size_t)hp.n * (size_t)hp.d * 4);
-            if (ea != cudaSuccess) { note_cuda(ea, "cr_aggregate (split scratch)"); return CR_ERR_OOM; }
-        }
         a.split_scratch = plan->d_split;
         cudaError_t e0 = cr::launch_fused_ldg(a, s, &plan->launches);
         if (e0 != cudaSuccess) { note_cuda(e0, "cr_aggregate"); return CR_ERR_CUDA; }
+        plan->last_kernel = "cr_fused_ldg_kernel (one row of blocks per sub-tree) + cr_sum_rows_kernel";
         return CR_OK;
     }
 
@@ -653,13 +662,14 @@ cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *m
         bool done = false;
         cudaError_t e0 = cr::launch_fused_tma(a, plan->dev, plan->tune, plan->encode, s, &plan->launches, &done);
         if (e0 != cudaSuccess) { note_cuda(e0, "cr_aggregate"); return CR_ERR_CUDA; }
-        if (done) return CR_OK;
+        if (done) { plan->last_kernel = "cr_fused_tma_kernel"; return CR_OK; }
     }
 
     if ((variant == CR_AGG_FUSED_LDG || (variant == CR_AGG_FUSED && prefer_plain)) && batch == 1 &&
         a.total_steps <= cr::inline_schedule_limit()) {
         cudaError_t e0 = cr::launch_fused_ldg(a, s, &plan->launches);
         if (e0 != cudaSuccess) { note_cuda(e0, "cr_aggregate"); return CR_ERR_CUDA; }
+        plan->last_kernel = "cr_fused_ldg_kernel";
         return CR_OK;
     }
 
@@ -688,12 +698,14 @@ cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *m
     cudaError_t e = cudaSuccess;
     if (variant == CR_AGG_UNCODED_SUM) {
         e = cr::launch_uncoded_sum(a, s, &plan->launches);
+        plan->last_kernel = "cr_uncoded_sum_kernel";
     } else {
         bool done = false;
         if (variant == CR_AGG_FUSED && !prefer_plain) {
             if (batch == 1) e = cr::launch_fused_tma(a, plan->dev, plan->tune, plan->encode, s, &plan->launches, &done);
             else e = cr::launch_fused_batch_tma(a, plan->dev, plan->tune, plan->encode, s, &plan->launches, &done);
         }
+        plan->last_kernel = done ? (batch == 1 ? "cr_fused_tma_kernel" : "cr_fused_batch_tma_kernel") : "cr_fused_ldg_kernel";
         if (e == cudaSuccess && !done) e = cr::launch_fused_ldg(a, s, &plan->launches);
     }
     if (e != cudaSuccess) { note_cuda(e, "cr_aggregate"); return CR_ERR_CUDA; }
