@@ -700,6 +700,7 @@ def main():
     ap.add_argument("--workload", default="cfg4", choices=list(inputs.CONFIGS))
     ap.add_argument("--dtype", default="f32", choices=["f32", "int32"])
     ap.add_argument("--d", type=int, default=0, help="override the gradient length (profiling on a small case)")
+    ap.add_argument("--rows", type=int, default=0, help="regression workloads: override the rows per partition")
     ap.add_argument("--tune", default="", help="consumer_warps,stages,ctas_per_sm,rows_per_box (0 = auto)")
     ap.add_argument("--coded", action="store_true", help="regression workloads: gradient + encode in one kernel")
     ap.add_argument("--models", type=int, default=0, help="regression workloads: gradients of K models per pass (1..32)")
@@ -716,6 +717,8 @@ def main():
     cfg = dict(inputs.CONFIGS[args.workload])
     if args.d:
         cfg["d"] = args.d
+    if args.rows and "rows" in cfg:
+        cfg["rows"] = args.rows
     world = int(os.environ.get("WORLD_SIZE", "1"))
     if args.gpus != world and world > 1:
         args.gpus = world
