@@ -201,8 +201,10 @@ struct FusedArgs {
     int *status;
 };
 
+// (Four 160-thread CTAs per SM need at most 96 registers per thread; the L <= 4 instances sit at 97 without
+// the bound and lose nothing to it.)
 template <typename T, int LMAX, int NCW>
-__global__ void __launch_bounds__((NCW + 1) * 32, 1)
+__global__ void __launch_bounds__((NCW + 1) * 32, (LMAX <= 4 && NCW == 4) ? 4 : 1)
 cr_fused_tma_kernel(const __grid_constant__ CUtensorMap tmap, const FusedArgs a) {
     constexpr int TILE = NCW * 128;
     constexpr int BOXW = TILE < 256 ? TILE : 256;
