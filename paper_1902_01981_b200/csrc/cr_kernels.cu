@@ -10,6 +10,7 @@
 #include <cooperative_groups.h>
 
 #include <algorithm>
+#include <cmath>
 #include <map>
 #include <mutex>
 #include <tuple>
@@ -650,8 +651,11 @@ struct InlineSchedule {
     Step steps[kInlineSteps];
 };
 
+// (Four 256-thread blocks per SM, 64 registers per thread, keep the most loads in flight; the instances
+// bounded here fit that without spilling.  Unbounded, the four-layer float instance took 75 registers,
+// three blocks per SM, and lost a tenth of its throughput.)
 template <typename T, int LMAX, int V, int PIPE>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, (LMAX <= 2 || (LMAX <= 4 && PIPE != 1)) ? 4 : 1)
 cr_fused_ldg_kernel(const T *__restrict__ G, const T *__restrict__ coeff, const Step *__restrict__ steps,
                     const int32_t *__restrict__ pat_off, int m, long long d, T *__restrict__ out, int shift,
                     const __grid_constant__ InlineSchedule inl) {
@@ -1297,17 +1301,26 @@ cudaError_t launch_fused_tma(const AggArgs &a, const DeviceInfo &dev, const Tuni
     const long long tiles_now = (a.d + tile - 1) / tile;
     if (!tune.stages && tiles_now < (long long)dev.sm_count * ctas)
         stages = (int)std::min<long long>(8, std::max<long long>(stages, ((long long)dev.sm_count * ctas * stages + tiles_now - 1) / tiles_now));
-    // A tile count just above the resident CTAs would send a few CTAs through a second tile while the
-    // rest idle (d = 120000, 256-column tiles: 469 tiles on 444 CTAs took 26.7 us; on four CTAs per SM,
-    // one tile each, 22.4 us).  Up to the register limit of the CTA size, take enough CTAs per SM for one
-    // tile each and thin every ring so that the bytes in flight per SM stay about the same.
-    if (!tune.ctas_per_sm && tiles_now > (long long)dev.sm_count * ctas && tiles_now <= (long long)dev.sm_count * 6) {
-        const int want = (int)((tiles_now + dev.sm_count - 1) / dev.sm_count);
-        const int thin = tune.stages ? stages : std::max(2, stages * ctas / want);
-        if (fused_resident_any(a.is_int, ncw, pick_lmax(a.L), (size_t)thin * stage_bytes + (size_t)thin * 16 + 32) >= want) {
-            ctas = want;
-            stages = thin;
+    // With only a few tiles per CTA the last pass over the tiles is partly empty (d = 120000, 256-column
+    // tiles: 469 tiles on 444 CTAs, 26.7 us; on four CTAs per SM, one tile each, 22.4 us.  m = 9, d = 2^19:
+    // 1024 tiles on 444 CTAs 41.9 us, on 592 CTAs 39.5 us).  Of the CTA counts per SM that fit the
+    // registers and shared memory, take the one whose last pass is fullest, and thin every ring so that
+    // the bytes in flight per SM stay about the same.
+    if (!tune.ctas_per_sm && tiles_now > (long long)dev.sm_count * ctas && tiles_now < (long long)dev.sm_count * ctas * 6) {
+        auto fill = [&](int c) {   // share of the CTA-passes that carry a tile
+            const double x = (double)tiles_now / ((double)dev.sm_count * c);
+            return x <= 1.0 ? 1.0 : x / std::ceil(x);
+        };
+        int best = ctas, best_stages = stages;
+        double best_fill = fill(ctas);
+        for (int c = ctas + 1; c <= 6; ++c) {
+            const int thin = tune.stages ? stages : std::max(2, stages * ctas / c);
+            if (fused_resident_any(a.is_int, ncw, pick_lmax(a.L), (size_t)thin * stage_bytes + (size_t)thin * 16 + 32) < c) break;
+            if (fill(c) > best_fill + 0.03) { best = c; best_stages = thin; best_fill = fill(c); }
+            if ((long long)dev.sm_count * c >= tiles_now) break;
         }
+        ctas = best;
+        stages = best_stages;
     }
     const size_t usable = (size_t)dev.smem_per_sm - 2048;  // leave room for the per-CTA reserve
     while (ctas > 1 && ((size_t)stages * stage_bytes + 1024 + 256) * ctas > usable) --ctas;

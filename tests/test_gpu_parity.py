@@ -213,6 +213,43 @@ def test_uncoded_sum_reads_the_same_slots():
         B.cr_plan_destroy(plan)
 
 
+def test_last_kernel_names_the_route_taken():
+    """cr_plan_last_kernel reports which kernel served the latest call: the TMA kernel for a single
+    pattern, the batch kernel for several, plain loads and the comparator on request, and the split
+    form for a short vector under a wide tree -- each result checked against the oracle as well."""
+    cfg = tree(4, 2, 1, "cyclic", 4096)
+    plan = make_plan(cfg)
+    try:
+        code, local = check_slot_table(plan, cfg)
+        assert B.cr_plan_last_kernel(plan) == ""
+        G = inputs.partition_gradients(cfg["P"], cfg["d"], seed=3)
+        G_dev = slots_on_device(plan, G, torch)
+        masks = inputs.straggler_masks(4, 2, 1, 5, seed=4)
+        for m_, flags, name in ((masks[:1], B.CR_AGG_FUSED, "cr_fused_tma_kernel"),
+                                (masks, B.CR_AGG_FUSED, "cr_fused_batch_tma_kernel"),
+                                (masks[:1], B.CR_AGG_FUSED_LDG, "cr_fused_ldg_kernel"),
+                                (masks[:1], B.CR_AGG_UNCODED_SUM, "cr_uncoded_sum_kernel")):
+            got = run_aggregate(plan, G_dev, m_, cfg["d"], flags)
+            assert B.cr_plan_last_kernel(plan) == name
+            if flags != B.CR_AGG_UNCODED_SUM:
+                for b in range(len(m_)):
+                    assert rel_l2(got[b], O.execute(code, local, G, m_[b])) <= REL_L2_BAR
+    finally:
+        B.cr_plan_destroy(plan)
+    cfg = tree(12, 2, 1, "cyclic", 5004)
+    plan = make_plan(cfg)
+    try:
+        code, local = check_slot_table(plan, cfg)
+        G = inputs.partition_gradients(cfg["P"], cfg["d"], seed=5)
+        G_dev = slots_on_device(plan, G, torch)
+        masks = inputs.straggler_masks(12, 2, 1, 1, seed=6, exactly_s=True)
+        got = run_aggregate(plan, G_dev, masks, cfg["d"], B.CR_AGG_FUSED)
+        assert "cr_sum_rows_kernel" in B.cr_plan_last_kernel(plan)
+        assert rel_l2(got[0], O.execute(code, local, G, masks[0])) <= REL_L2_BAR
+    finally:
+        B.cr_plan_destroy(plan)
+
+
 # --------------------------------------------------------------------------- integer-exact mode
 
 @pytest.mark.parametrize("cfg,batch", [(tree(3, 2, 1, "printed_3_1", 1200), 20), (tree(3, 4, 1, "printed_3_1", 4104), 64),
