@@ -702,6 +702,7 @@ def main():
     ap.add_argument("--d", type=int, default=0, help="override the gradient length (profiling on a small case)")
     ap.add_argument("--tree", default="", help="override the tree of the workload: n,L,s,code[,c] with code in "
                     "printed_3_1|cyclic|repetition and P = c times the smallest partition count the tree allows")
+    ap.add_argument("--batch", type=int, default=0, help="aggregation workloads: straggler patterns per call")
     ap.add_argument("--rows", type=int, default=0, help="regression workloads: override the rows per partition")
     ap.add_argument("--tune", default="", help="consumer_warps,stages,ctas_per_sm,rows_per_box (0 = auto)")
     ap.add_argument("--coded", action="store_true", help="regression workloads: gradient + encode in one kernel")
@@ -724,6 +725,8 @@ def main():
         n, L, s_ = int(f[0]), int(f[1]), int(f[2])
         quantum = sum(n ** l * (s_ + 1) ** (L - l) for l in range(1, L + 1))
         cfg.update(n=n, L=L, s=s_, code=f[3], P=quantum * (int(f[4]) if len(f) > 4 else 1))
+    if args.batch and cfg["kind"] == "aggregate":
+        cfg["batch"] = args.batch
     if args.rows and "rows" in cfg:
         cfg["rows"] = args.rows
     world = int(os.environ.get("WORLD_SIZE", "1"))

@@ -632,10 +632,11 @@ cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *m
     // 6.0-6.6 TB/s with m = 4, 1.7 TB/s from coded gradients).  The plain-load kernel, which requests
     // the next group of rows before it combines the current one, reaches 7.3 and 7.0 TB/s there, and
     // is still 2 % ahead at m = 8 ((4,3) tree: 7.32 against 7.16 TB/s).  Unless the caller fixed a TMA
-    // launch shape, single patterns of these shapes take that kernel.
+    // launch shape, single patterns of these shapes take that kernel.  So do two or three rows per node
+    // (flat gradient coding, L = 1; n = 12, s = 1 at d = 2^22: 4.9 against 3.0 TB/s).
     // Short vectors stay with the TMA kernel unless they are coded gradients: its narrow tiles and
     // deep rings fill more SMs (m = 4, d = 5004: 70 against 109 us; from coded gradients 51 against 37 us).
-    const bool prefer_plain = batch == 1 && (a.m == 1 || ((a.m == 4 || a.m == 8) && hp.d >= (1ll << 19))) &&
+    const bool prefer_plain = batch == 1 && (a.m == 1 || ((a.m <= 4 || a.m == 8) && hp.d >= (1ll << 19))) &&
                               hp.d % 4 == 0 && !plan->tune.ncw && !plan->tune.stages && !plan->tune.ctas_per_sm &&
                               !plan->tune.rows;
 
@@ -678,7 +679,20 @@ cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *m
     const size_t off_bytes = align16(ex.pat_off.size() * 4);
     const size_t nodes_bytes = align16(ex.unodes.size() * 4);
     const size_t wtab_bytes = align16(ex.wtab.size() * 4);
-    const size_t total = steps_bytes + off_bytes + nodes_bytes + wtab_bytes;
+    // Batches over nodes with few slot rows (m <= 8, or coded gradients): one TMA box takes the rows of up
+    // to 16 / m union nodes with consecutive ids, which lie next to each other in the slot buffer.
+    std::vector<int2> boxes;
+    const int npb = (batch > 1 && variant == CR_AGG_FUSED && a.m <= 8) ? 16 / a.m : 1;
+    if (npb > 1 && ex.unodes.size() < (1u << 20)) {
+        for (size_t u = 0; u < ex.unodes.size();) {
+            size_t g = 1;
+            while (g < (size_t)npb && u + g < ex.unodes.size() && ex.unodes[u + g] == ex.unodes[u] + (int32_t)g) ++g;
+            boxes.push_back(make_int2(ex.unodes[u] * a.m, (int)u | (int)(g << 20)));
+            u += g;
+        }
+    }
+    const size_t boxes_bytes = align16(boxes.size() * sizeof(int2));
+    const size_t total = steps_bytes + off_bytes + nodes_bytes + wtab_bytes + boxes_bytes;
     StageSlot *slot = nullptr;
     st = stage_acquire(plan, total, &slot);
     if (st != CR_OK) return st;
@@ -686,6 +700,8 @@ cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *m
     std::memcpy(slot->host + steps_bytes, ex.pat_off.data(), ex.pat_off.size() * 4);
     std::memcpy(slot->host + steps_bytes + off_bytes, ex.unodes.data(), ex.unodes.size() * 4);
     std::memcpy(slot->host + steps_bytes + off_bytes + nodes_bytes, ex.wtab.data(), ex.wtab.size() * 4);
+    if (!boxes.empty())
+        std::memcpy(slot->host + steps_bytes + off_bytes + nodes_bytes + wtab_bytes, boxes.data(), boxes.size() * sizeof(int2));
     st = stage_commit(slot, total, s);
     if (st != CR_OK) return st;
 
@@ -693,6 +709,11 @@ cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *m
     a.pat_off = reinterpret_cast<const int32_t *>(slot->dev + steps_bytes);
     a.unodes = reinterpret_cast<const int32_t *>(slot->dev + steps_bytes + off_bytes);
     a.wtab = reinterpret_cast<const uint32_t *>(slot->dev + steps_bytes + off_bytes + nodes_bytes);
+    if (!boxes.empty()) {
+        a.boxes = reinterpret_cast<const int2 *>(slot->dev + steps_bytes + off_bytes + nodes_bytes + wtab_bytes);
+        a.n_boxes = (int)boxes.size();
+        a.npb = npb;
+    }
     a.host_steps = nullptr;
 
     cudaError_t e = cudaSuccess;

@@ -368,6 +368,8 @@ struct BatchArgs {
     const int32_t *unodes;
     const uint32_t *wtab;  // distinct weight bit patterns of the batch
     int n_wtab;
+    const int2 *boxes;     // npb > 1: boxes that cover several union nodes each (see AggArgs)
+    int n_boxes, npb;
     int n_union, batch;
     int m, R, cpn, stages;
     int same_shape;  // every pattern's schedule has the same length and layer sequence
@@ -428,7 +430,79 @@ cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchA
     const T *coeff = reinterpret_cast<const T *>(a.coeff);
     const uint32_t stage_bytes = (uint32_t)(stage_elems * sizeof(T));
 
-    if (warp < NLW) {
+    if (warp < NLW && a.npb > 1) {
+        // ---------------- loaders, few slot rows per node: a box holds the rows of up to npb union nodes ----------------
+        bool ok = true;
+        const unsigned boxes_w = warp < a.n_boxes ? (unsigned)(a.n_boxes - warp + NLW - 1) / NLW : 0u;   // boxes of this loader per tile
+        const unsigned my_tiles = blockIdx.x < a.ntiles ? (unsigned)((a.ntiles - 1 - blockIdx.x) / gridDim.x + 1) : 0u;
+        const unsigned total_boxes = my_tiles * boxes_w;
+        T *my_ring = ring + (size_t)warp * S * stage_elems;
+        uint64_t *my_full = full + warp * S;
+        unsigned issued = 0, it_t = 0, it_n = 0;
+        auto issue_next = [&]() {   // lane 0 only
+            const int slot = (int)(issued % (unsigned)S);
+            const long long tile = (long long)blockIdx.x + (long long)it_t * gridDim.x;
+            const int row0 = __ldg(&a.boxes[warp + (int)it_n * NLW].x);
+            mbar_expect_tx(&my_full[slot], stage_bytes);
+            tma_load_2d(my_ring + (size_t)slot * stage_elems, &tmap, (int)(tile * TILE), row0, &my_full[slot]);
+            ++issued;
+            if (++it_n == boxes_w) { it_n = 0; ++it_t; }
+        };
+        if (lane == 0)
+            while (issued < total_boxes && issued < (unsigned)S) issue_next();
+        unsigned q = 0;  // next box to consume
+        unsigned t = 0;  // tiles handled by this CTA so far
+        for (long long tile = blockIdx.x; tile < a.ntiles && ok; tile += gridDim.x, ++t) {
+            const int buf = (int)(t % (unsigned)a.nbuf);
+            const unsigned use = t / (unsigned)a.nbuf;
+            if (!mbar_wait_warp(&e_free[buf], (use & 1u) ^ 1u, &flags[0])) { ok = false; break; }
+            T *Eb = E + (size_t)buf * e_elems;
+            for (int bi = warp; bi < a.n_boxes && ok; bi += NLW, ++q) {
+                const int slot = (int)(q % (unsigned)S);
+                const uint32_t phase = (q / (unsigned)S) & 1u;
+                const int2 bx = __ldg(&a.boxes[bi]);
+                const int u0 = bx.y & 0xfffff, valid = (bx.y >> 20) * a.m;   // rows of the box that belong to union nodes
+                // a row's coefficient sits at the row's own index; fetched before the wait on the data
+                T cj[kMaxBoxRows];
+#pragma unroll
+                for (int j = 0; j < kMaxBoxRows; ++j) cj[j] = j < valid ? __ldg(coeff + bx.x + j) : T(0);
+                if (!mbar_wait_warp(&my_full[slot], phase, &flags[0])) { ok = false; break; }
+                const T *src = my_ring + (size_t)slot * stage_elems + lane * 4;
+                T e[4] = {T(0), T(0), T(0), T(0)};
+                int node_end = a.m, i = 0;
+#pragma unroll
+                for (int j = 0; j < kMaxBoxRows; ++j) {
+                    if (j < valid) {
+                        const V4 v = *reinterpret_cast<const V4 *>(src + (size_t)j * TILE);
+                        e[0] += cj[j] * v.x; e[1] += cj[j] * v.y; e[2] += cj[j] * v.z; e[3] += cj[j] * v.w;
+                        if (j + 1 == node_end) {   // last row of a node: its coded gradient is complete
+                            V4 o; o.x = e[0]; o.y = e[1]; o.z = e[2]; o.w = e[3];
+                            *reinterpret_cast<V4 *>(Eb + (size_t)(u0 + i) * TILE + lane * 4) = o;
+                            e[0] = e[1] = e[2] = e[3] = T(0);
+                            ++i; node_end += a.m;
+                        }
+                    }
+                }
+                // every lane has read the box: refill its buffer with box q + stages
+                __syncwarp();
+                if (lane == 0 && issued < total_boxes) {
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    issue_next();
+                }
+            }
+            if (!ok) break;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&e_full[buf]);
+        }
+        if (!ok) {
+            // give up: flag it, then wait (bounded) for this loader's copies still in flight
+            flags[0] = 1;
+            atomicExch(a.status, 1);
+            const unsigned in_flight_end = __shfl_sync(0xffffffffu, issued, 0);
+            for (unsigned b = q; b < in_flight_end; ++b)
+                mbar_wait(&my_full[b % (unsigned)S], (b / (unsigned)S) & 1u, &flags[1]);
+        }
+    } else if (warp < NLW) {
         // ---------------- loaders: stream their boxes, coded gradients of the union nodes -> E[buf] ----------------
         bool ok = true;
         const unsigned nodes_w = (unsigned)(a.n_union - warp + NLW - 1) / NLW;   // union nodes of this loader per tile
@@ -1405,6 +1479,16 @@ cudaError_t launch_fused_batch_tma(const AggArgs &a, const DeviceInfo &dev, cons
     // second E buffer, then six loaders rather than four.
     int nbuf = 0, stages = 0, R = 0, nlw = 0;
     const int want_loaders = tune.ctas_per_sm == 4 ? 4 : 6;
+    // Few slot rows per node (m <= 8, coded gradients): a box of one node would be 0.5-4 KB, too small for
+    // the copy engine.  Then a box takes the rows of npb consecutive union nodes; the selection below sees
+    // such a box as one tall node, and falls back to one node per box if tall boxes do not fit beside E.
+    bool multi = a.npb > 1 && a.boxes && a.n_boxes > 0 && a.npb * a.m <= kMaxBoxRows && !tune.rows;
+    for (int attempt = 0; attempt < 2 && !nbuf; ++attempt) {
+    if (attempt == 1) {
+        if (!multi) break;
+        multi = false;
+    }
+    const int node_rows = multi ? a.npb * a.m : a.m;
     for (int try_buf = 2; try_buf >= 1 && !nbuf; --try_buf) {
         if (budget <= try_buf * e_one + sched_bytes) continue;
         const size_t ring_budget = budget - try_buf * e_one - sched_bytes;
@@ -1414,14 +1498,16 @@ cudaError_t launch_fused_batch_tma(const AggArgs &a, const DeviceInfo &dev, cons
             for (int depth = want_stages; depth >= 2; --depth) {
                 const int cap = (int)std::min<size_t>(kMaxBoxRows, ring_budget / ((size_t)lw * depth * tile * 4));
                 if (cap < 1) continue;
-                const int r = tune.rows && a.m % tune.rows == 0 && tune.rows <= cap ? tune.rows : rows_per_box(a.m, cap);
+                const int r = multi ? (node_rows <= cap ? node_rows : 0)
+                                    : (tune.rows && a.m % tune.rows == 0 && tune.rows <= cap ? tune.rows : rows_per_box(a.m, cap));
                 if (r > best_r) { best_r = r; best_depth = depth; best_lw = lw; }
             }
         }
         // two buffers only if they do not cost more than half of the box height one buffer allows
-        if (best_r && (try_buf == 1 || 2 * best_r >= std::min(a.m, kMaxBoxRows))) {
+        if (best_r && (try_buf == 1 || 2 * best_r >= std::min(node_rows, kMaxBoxRows))) {
             nbuf = try_buf; R = best_r; stages = best_depth; nlw = best_lw;
         }
+    }
     }
     if (!nbuf) return cudaSuccess;  // union too large for shared memory: caller falls back
     const size_t stage_bytes = (size_t)R * tile * 4;
@@ -1430,7 +1516,7 @@ cudaError_t launch_fused_batch_tma(const AggArgs &a, const DeviceInfo &dev, cons
     const long long ntiles = (a.d + tile - 1) / tile;
     const int grid = (int)std::min<long long>(ntiles, (long long)dev.sm_count);
     // box counters are 32-bit
-    if ((ntiles / grid + 1) * (long long)a.n_union * (a.m / R) >= (1ll << 31)) return cudaSuccess;
+    if ((ntiles / grid + 1) * (long long)a.n_union * (multi ? 1 : a.m / R) >= (1ll << 31)) return cudaSuccess;
 
     CUtensorMap map;
     if (make_map(encode, &map, a, tile, R) != CUDA_SUCCESS) return cudaSuccess;
@@ -1440,6 +1526,8 @@ cudaError_t launch_fused_batch_tma(const AggArgs &a, const DeviceInfo &dev, cons
     ba.batch = a.batch; ba.same_shape = a.same_shape; ba.m = a.m; ba.R = R; ba.cpn = a.m / R; ba.stages = stages;
     ba.d = a.d; ba.ntiles = ntiles; ba.out = a.out; ba.shift = a.shift; ba.status = a.status;
     ba.sched_smem = (int)sched_bytes; ba.nst = nst; ba.nbuf = nbuf; ba.wtab = a.wtab; ba.n_wtab = a.n_wtab;
+    ba.boxes = multi ? a.boxes : nullptr; ba.n_boxes = multi ? a.n_boxes : 0; ba.npb = multi ? a.npb : 1;
+    if (multi) ba.cpn = 1;
     const cudaError_t err = a.is_int ? run_batch_w<int>(nlw, nrw, lmax, map, ba, grid, smem, stream)
                                      : run_batch_w<float>(nlw, nrw, lmax, map, ba, grid, smem, stream);
     if (err == cudaSuccess) { *done = true; ++*launches; }

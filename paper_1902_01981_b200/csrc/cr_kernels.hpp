@@ -46,6 +46,12 @@ struct AggArgs {
     const int32_t *unodes;   // device [n_union]: union of used nodes (batch kernel)
     const uint32_t *wtab;    // device [n_wtab]: distinct weight bit patterns of the batch (n_wtab = 0: none)
     int n_wtab;
+    // batch kernel, few slot rows per node: device [n_boxes] TMA boxes that each cover up to `npb` union
+    // nodes with consecutive ids (their slot rows are contiguous).  x = first slot row, y = position of the
+    // first node in the union list (bits 0..19) | number of union nodes covered (bits 20..).  npb <= 1: unused.
+    const int2 *boxes = nullptr;
+    int n_boxes = 0;
+    int npb = 0;
     int n_union;
     int batch;
     int total_steps;

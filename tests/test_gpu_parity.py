@@ -137,6 +137,42 @@ def test_random_patterns_medium_trees(cfg, batch, flags):
         B.cr_plan_destroy(plan)
 
 
+@pytest.mark.parametrize("cfg,dtype", [(tree(12, 2, 1, "cyclic", 4100), "f32"), (tree(4, 3, 1, "cyclic", 2600), "f32"),
+                                       (tree(3, 3, 1, "printed_3_1", 1500), "i32"), (tree(6, 1, 2, "repetition", 3000), "i32"),
+                                       (tree(16, 1, 1, "cyclic", 2100), "f32")])
+@pytest.mark.parametrize("batch", [2, 23])
+def test_batches_over_nodes_with_few_slot_rows(cfg, dtype, batch):
+    """m <= 8 slot rows per node: the batch kernel loads the rows of several consecutive union nodes
+    with one box.  Two patterns leave gaps in the union (runs of one to four nodes, a ragged last
+    box), twenty-three fill it; the same batches from coded gradients (one row per node, boxes of up
+    to sixteen nodes)."""
+    n, L, s, d = cfg["n"], cfg["L"], cfg["s"], cfg["d"]
+    is_int = dtype == "i32"
+    plan = make_plan(cfg, dtype=B.CR_I32 if is_int else B.CR_F32)
+    try:
+        code, local = check_slot_table(plan, cfg)
+        G = inputs.integer_gradients(cfg["P"], d, seed=31) if is_int else inputs.partition_gradients(cfg["P"], d, seed=31)
+        G_dev = slots_on_device(plan, G, torch)
+        masks = inputs.straggler_masks(n, L, s, batch, seed=32, exactly_s=True)
+        tdtype = torch.int32 if is_int else torch.float32
+        got = run_aggregate(plan, G_dev, masks, d, B.CR_AGG_FUSED, dtype=tdtype)
+        assert B.cr_plan_last_kernel(plan) == "cr_fused_batch_tma_kernel"
+        E = torch.zeros((B.cr_plan_num_nodes(plan), d), dtype=tdtype, device="cuda")
+        B.cr_encode(plan, G_dev, E)
+        got_coded = run_aggregate(plan, E, masks, d, B.CR_AGG_FUSED | B.CR_AGG_FROM_CODED, dtype=tdtype)
+        for b in range(batch):
+            if is_int:
+                want = O.execute_integer(code, local, G, masks[b])
+                assert np.array_equal(got[b].astype(np.int64), want)
+                assert np.array_equal(got_coded[b].astype(np.int64), want)
+            else:
+                want = O.execute(code, local, G, masks[b])
+                assert rel_l2(got[b], want) <= REL_L2_BAR
+                assert rel_l2(got_coded[b], want) <= REL_L2_BAR
+    finally:
+        B.cr_plan_destroy(plan)
+
+
 def test_batch_of_patterns_with_different_shapes():
     """An explicit code whose decode rows use two or three children depending on the straggler:
     the patterns of one batch then have schedules of different lengths."""
