@@ -401,7 +401,9 @@ cr_status_t cr_partial_gradients_loss(cr_plan_t *plan, int32_t loss, const float
                                                reinterpret_cast<cudaStream_t>(stream), &plan->launches);
     } else {
         if (!workspace || workspace_bytes < cr_partial_gradients_workspace_bytes(plan, rows)) return CR_ERR_OOM;
-        e = cr::launch_partial_gradients_two_pass(X, y, w, plan->d_part, items, rows, plan->hp.d,
+        // items grouped by partition unless the caller asked for (node, slot) order: the items that hold the
+        // same partition then read its rows from HBM once and share them through L2
+        e = cr::launch_partial_gradients_two_pass(X, y, w, plan->d_part, plan->tune.pg_order == 1 ? nullptr : plan->d_order, items, rows, plan->hp.d,
                                                   reinterpret_cast<float *>(workspace), G_slots, loss,
                                                   reinterpret_cast<cudaStream_t>(stream), &plan->launches);
     }
@@ -814,7 +816,7 @@ cr_status_t cr_partial_gradients_static(cr_plan_t *plan, const float *X, const f
         }
         scratch = g_static_ptr[plan->device];
     }
-    cudaError_t e = cr::launch_partial_gradients_two_pass(X, y, w, plan->d_part, plan->hp.N * plan->hp.m, rows, plan->hp.d,
+    cudaError_t e = cr::launch_partial_gradients_two_pass(X, y, w, plan->d_part, nullptr, plan->hp.N * plan->hp.m, rows, plan->hp.d,
                                                  scratch, G_slots, CR_LOSS_SQUARED, reinterpret_cast<cudaStream_t>(stream),
                                                  &plan->launches);
     if (e != cudaSuccess) { note_cuda(e, "cr_partial_gradients_static"); return CR_ERR_CUDA; }

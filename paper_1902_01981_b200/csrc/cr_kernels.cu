@@ -592,7 +592,11 @@ cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchA
                 // table (broadcast shared-memory loads); the loop is unrolled by two so that the E rows
                 // of the next step are in flight while the current one is folded.
                 const int nst = a.nst;
-                for (int g = rw; g * NP < a.batch; g += NRW) {
+                // fewer pattern groups than replay warps: the groups of consecutive tiles go to different
+                // warps, so that all of them work (on different E buffers) instead of the first few
+                const int ngroups = (a.batch + NP - 1) / NP;
+                const int g0 = ngroups < NRW ? (int)((rw + NRW - (t * (unsigned)ngroups) % NRW) % NRW) : rw;
+                for (int g = g0; g < ngroups; g += NRW) {
                     T acc[NP][LMAX][4];
 #pragma unroll
                     for (int p = 0; p < NP; ++p)
@@ -645,7 +649,8 @@ cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchA
             } else {
                 // General case, one pattern at a time: lane i fetches entry i of the pattern's schedule
                 // (one coalesced load per 32 entries); entries are broadcast with shuffles.
-                for (int b = rw; b < a.batch; b += NRW) {
+                const int b0 = a.batch < NRW ? (int)((rw + NRW - (t * (unsigned)a.batch) % NRW) % NRW) : rw;
+                for (int b = b0; b < a.batch; b += NRW) {
                     T acc[LMAX][4];
 #pragma unroll
                     for (int l = 0; l < LMAX; ++l)
@@ -962,13 +967,16 @@ cr_decode_kernel(const T *__restrict__ M_child, const T *__restrict__ E_parent, 
 template <int V>
 __global__ void __launch_bounds__(256)
 cr_residual_kernel(const float *__restrict__ X, const float *__restrict__ y, const float *__restrict__ w,
-                   const int32_t *__restrict__ part, long long total_rows, int rows, long long d,
-                   float *__restrict__ resid, int loss) {
+                   const int32_t *__restrict__ part, const int32_t *__restrict__ order, long long total_rows, int rows,
+                   long long d, float *__restrict__ resid, int loss) {
     const int lane = threadIdx.x & 31;
     const long long warps = ((long long)gridDim.x * blockDim.x) >> 5;
     for (long long idx = ((long long)blockIdx.x * blockDim.x + threadIdx.x) >> 5; idx < total_rows; idx += warps) {
-        const long long item = idx / rows;
-        const int row = (int)(idx - item * rows);
+        // `order` (may be null) lists the items grouped by partition: the warps that run side by side then
+        // read the same rows of X and share them through L2
+        const long long pos = idx / rows;
+        const int row = (int)(idx - pos * rows);
+        const long long item = order ? (long long)__ldg(&order[pos]) : pos;
         const int p = __ldg(&part[item]);
         const float *xr = X + ((size_t)p * rows + row) * d;
         float acc = 0.f;
@@ -985,7 +993,7 @@ cr_residual_kernel(const float *__restrict__ X, const float *__restrict__ y, con
         for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
         if (lane == 0) {
             if (loss == 1) acc = 1.f / (1.f + expf(-acc));   // logistic: sigmoid of the score
-            resid[idx] = acc - __ldg(&y[(size_t)p * rows + row]);
+            resid[item * rows + row] = acc - __ldg(&y[(size_t)p * rows + row]);
         }
     }
 }
@@ -993,9 +1001,9 @@ cr_residual_kernel(const float *__restrict__ X, const float *__restrict__ y, con
 // Pass 2: grid (column tiles, items); a thread owns V columns and walks all rows of the item.
 template <int V>
 __global__ void __launch_bounds__(128)
-cr_xt_r_kernel(const float *__restrict__ X, const int32_t *__restrict__ part, const float *__restrict__ resid,
-               int rows, long long d, float *__restrict__ G) {
-    const long long item = blockIdx.y;
+cr_xt_r_kernel(const float *__restrict__ X, const int32_t *__restrict__ part, const int32_t *__restrict__ order,
+               const float *__restrict__ resid, int rows, long long d, float *__restrict__ G) {
+    const long long item = order ? (long long)__ldg(&order[blockIdx.y]) : (long long)blockIdx.y;
     const long long col = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * V;
     if (col >= d) return;
     const int p = __ldg(&part[item]);
@@ -1676,23 +1684,23 @@ cudaError_t launch_decode(const void *M_child, const void *E_parent, const void 
 }
 
 cudaError_t launch_partial_gradients_two_pass(const float *X, const float *y, const float *w, const int32_t *part,
-                                              int items, int rows, int64_t d, float *resid, float *G, int loss,
-                                              cudaStream_t stream, int64_t *launches) {
+                                              const int32_t *order, int items, int rows, int64_t d, float *resid,
+                                              float *G, int loss, cudaStream_t stream, int64_t *launches) {
     const bool v4 = d % 4 == 0 && aligned16(X) && aligned16(w) && aligned16(G);
     const long long total_rows = (long long)items * rows;
     const long long want_blocks = (total_rows + 7) / 8;  // 8 warps per block
     const int blocks = (int)std::min<long long>(want_blocks, 148 * 32);
-    if (v4) cr_residual_kernel<4><<<blocks, 256, 0, stream>>>(X, y, w, part, total_rows, rows, d, resid, loss);
-    else cr_residual_kernel<1><<<blocks, 256, 0, stream>>>(X, y, w, part, total_rows, rows, d, resid, loss);
+    if (v4) cr_residual_kernel<4><<<blocks, 256, 0, stream>>>(X, y, w, part, order, total_rows, rows, d, resid, loss);
+    else cr_residual_kernel<1><<<blocks, 256, 0, stream>>>(X, y, w, part, order, total_rows, rows, d, resid, loss);
     cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) return err;
     ++*launches;
     if (v4) {
         dim3 grid((unsigned)((d / 4 + 127) / 128), (unsigned)items);
-        cr_xt_r_kernel<4><<<grid, 128, 0, stream>>>(X, part, resid, rows, d, G);
+        cr_xt_r_kernel<4><<<grid, 128, 0, stream>>>(X, part, order, resid, rows, d, G);
     } else {
         dim3 grid((unsigned)((d + 127) / 128), (unsigned)items);
-        cr_xt_r_kernel<1><<<grid, 128, 0, stream>>>(X, part, resid, rows, d, G);
+        cr_xt_r_kernel<1><<<grid, 128, 0, stream>>>(X, part, order, resid, rows, d, G);
     }
     err = cudaGetLastError();
     if (err == cudaSuccess) ++*launches;

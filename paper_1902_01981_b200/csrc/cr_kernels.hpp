@@ -105,9 +105,10 @@ cudaError_t launch_decode(const void *M_child, const void *E_parent, const void 
 // Partial gradients of linear regression, two passes over X: residuals r = X_p w - y_p into `resid`
 // ([items][rows]), then G[item][:] = X_p^T r.  part[item] is the partition of slot `item`.  Any d.
 // loss: 0 squared, 1 logistic (r = sigmoid(X_p w) - y_p).
+// `order` (device [items], may be null): launch order of the items, e.g. grouped by partition.
 cudaError_t launch_partial_gradients_two_pass(const float *X, const float *y, const float *w, const int32_t *part,
-                                              int items, int rows, int64_t d, float *resid, float *G, int loss,
-                                              cudaStream_t stream, int64_t *launches);
+                                              const int32_t *order, int items, int rows, int64_t d, float *resid,
+                                              float *G, int loss, cudaStream_t stream, int64_t *launches);
 
 // The same in one pass over X (row blocks staged in shared memory, cluster reduction), no scratch;
 // needs d % 4 == 0, d <= 8192 and 16-byte aligned X, w, G (partial_fused_eligible).
