@@ -634,11 +634,14 @@ cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *m
     // 6.0-6.6 TB/s with m = 4, 1.7 TB/s from coded gradients).  The plain-load kernel, which requests
     // the next group of rows before it combines the current one, reaches 7.3 and 7.0 TB/s there, and
     // is still 2 % ahead at m = 8 ((4,3) tree: 7.32 against 7.16 TB/s).  Unless the caller fixed a TMA
-    // launch shape, single patterns of these shapes take that kernel.  So do two or three rows per node
+    // launch shape, single patterns of these shapes take that kernel.  Taller nodes whose rows come in fours
+    // (m = 12, 16, ..) do too up to d = 2^23, where the prefetching form is still ahead (m = 16, (4,2,3) tree:
+    // 6.8 against 6.2 TB/s at d = 2^22, 7.0 against 6.6 at 2^23, 6.8 against 6.9 at 2^24).  So do two or three rows per node
     // (flat gradient coding, L = 1; n = 12, s = 1 at d = 2^22: 4.9 against 3.0 TB/s).
     // Short vectors stay with the TMA kernel unless they are coded gradients: its narrow tiles and
     // deep rings fill more SMs (m = 4, d = 5004: 70 against 109 us; from coded gradients 51 against 37 us).
-    const bool prefer_plain = batch == 1 && (a.m == 1 || ((a.m <= 4 || a.m == 8) && hp.d >= (1ll << 19))) &&
+    const bool prefer_plain = batch == 1 &&
+                              (a.m == 1 || ((a.m <= 4 || a.m % 4 == 0) && hp.d >= (1ll << 19) && (a.m <= 8 || hp.d <= (1ll << 23)))) &&
                               hp.d % 4 == 0 && !plan->tune.ncw && !plan->tune.stages && !plan->tune.ctas_per_sm &&
                               !plan->tune.rows;
 

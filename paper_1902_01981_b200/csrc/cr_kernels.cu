@@ -14,6 +14,7 @@
 #include <map>
 #include <mutex>
 #include <tuple>
+#include <type_traits>
 #include <cstdio>
 
 namespace cr {
@@ -731,10 +732,14 @@ struct InlineSchedule {
 };
 
 // (Four 256-thread blocks per SM, 64 registers per thread, keep the most loads in flight; the instances
-// bounded here fit that without spilling.  Unbounded, the four-layer float instance took 75 registers,
+// bounded here fit that without spilling.  The generic path of two-layer trees, which serves the short
+// launches of flat gradient coding -- two or three rows per node, a few dozen rows per thread -- gains
+// from more resident threads instead: six blocks at 40 registers (five for int32), n = 12, s = 1 at
+// d = 2^22: 4.9 -> 5.8 TB/s.  Unbounded, the four-layer float instance took 75 registers,
 // three blocks per SM, and lost a tenth of its throughput.)
 template <typename T, int LMAX, int V, int PIPE>
-__global__ void __launch_bounds__(256, (LMAX <= 2 || (LMAX <= 4 && PIPE != 1)) ? 4 : 1)
+__global__ void __launch_bounds__(256, (LMAX <= 2 && PIPE == 0) ? (std::is_floating_point<T>::value ? 6 : 5)
+                                                                     : ((LMAX <= 2 || (LMAX <= 4 && PIPE != 1)) ? 4 : 1))
 cr_fused_ldg_kernel(const T *__restrict__ G, const T *__restrict__ coeff, const Step *__restrict__ steps,
                     const int32_t *__restrict__ pat_off, int m, long long d, T *__restrict__ out, int shift,
                     const __grid_constant__ InlineSchedule inl) {
