@@ -38,8 +38,8 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the timed kernel, from the ncu capture
 # summarised under profiles/ (absent = no capture of the current kernel on that workload).
 # cfg4: 917.5 MB measured at d = 2^21, scaled by 8 to d = 2^24 (traffic is proportional to d).
-# cfg5: 2076.7 MB measured at d = 2^18, scaled by 16 to d = 2^22.
-NCU_TRAFFIC_BYTES = {("cfg4", "f32", 1 << 24): 8 * 917.46e6, ("cfg5", "f32", 1 << 22): 16 * 2076.66e6}
+# cfg5: 2076.0 MB measured at d = 2^18, scaled by 16 to d = 2^22.
+NCU_TRAFFIC_BYTES = {("cfg4", "f32", 1 << 24): 8 * 917.46e6, ("cfg5", "f32", 1 << 22): 16 * 2076.03e6}
 
 
 def peak_hbm():
