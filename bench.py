@@ -691,6 +691,16 @@ def run_multi(args, cfg):
     B.cr_plan_destroy(plan)
 
 
+def apply_tree_override(cfg, text):
+    """`--tree n,L,s,code[,c]`: replaces the tree of a workload; P becomes c times the smallest partition
+    count that the tree splits into whole chunks at every level."""
+    f = text.split(",")
+    n, L, s_ = int(f[0]), int(f[1]), int(f[2])
+    quantum = sum(n ** l * (s_ + 1) ** (L - l) for l in range(1, L + 1))
+    cfg.update(n=n, L=L, s=s_, code=f[3], P=quantum * (int(f[4]) if len(f) > 4 else 1))
+    return cfg
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -721,10 +731,7 @@ def main():
     if args.d:
         cfg["d"] = args.d
     if args.tree:
-        f = args.tree.split(",")
-        n, L, s_ = int(f[0]), int(f[1]), int(f[2])
-        quantum = sum(n ** l * (s_ + 1) ** (L - l) for l in range(1, L + 1))
-        cfg.update(n=n, L=L, s=s_, code=f[3], P=quantum * (int(f[4]) if len(f) > 4 else 1))
+        apply_tree_override(cfg, args.tree)
     if args.batch and cfg["kind"] == "aggregate":
         cfg["batch"] = args.batch
     if args.rows and "rows" in cfg:

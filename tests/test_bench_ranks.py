@@ -68,3 +68,35 @@ def test_reference_arm_prints_the_contract_line():
     assert line["impl"] == "reference" and line["unit"] == "GB/s" and line["value"] > 0
     assert line["cpu_baseline"]["kind"] == "oracle" and line["e2e"]["h2d_bytes_per_step"] == 0
     assert line["config"]["workload"].startswith("cfg2")
+
+
+def test_reference_arm_of_a_regression_workload():
+    """Regression workloads time the oracle's gradient-descent step (gradients of a sample of the
+    partitions, aggregation of all, model update); other ranks print nothing."""
+    env = dict(os.environ)
+    env.pop("RANK", None)
+    cmd = [sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--steps", "3", "--warmup", "1",
+           "--workload", "cfg1"]
+    out = subprocess.run(cmd, env=env, capture_output=True, text=True, timeout=300)
+    assert out.returncode == 0, out.stderr
+    line = json.loads(out.stdout.strip().splitlines()[-1])
+    assert line["impl"] == "reference" and line["unit"] == "GB/s" and line["value"] > 0 and line["gpu_launches"] == 0
+    assert line["cpu_baseline"]["kind"] == "oracle" and "partitions per step" in line["cpu_baseline"]["sample"]
+    assert line["config"]["workload"].startswith("cfg1") and line["dtype"] == "f64"
+    quiet = subprocess.run(cmd, env=dict(env, RANK="1", WORLD_SIZE="2"), capture_output=True, text=True, timeout=300)
+    assert quiet.returncode == 0 and quiet.stdout.strip() == ""
+
+
+def test_tree_override_keeps_the_partition_count_feasible():
+    """`--tree n,L,s,code[,c]` sets P to c times the smallest count the tree can split into whole chunks:
+    the oracle's allocation accepts it and gives every node c (s+1)^L slots."""
+    sys.path.insert(0, ROOT)
+    import bench
+    from oracle import cr_oracle as O
+    from oracle import cr_setup
+    for text, c in (("12,1,1,cyclic", 1), ("4,3,1,cyclic,2", 2), ("6,2,2,repetition", 1)):
+        cfg = bench.apply_tree_override(dict(d=64, seed=0), text)
+        n, L, s = cfg["n"], cfg["L"], cfg["s"]
+        assert cfg["P"] == c * O.partition_quantum(n, L, s)
+        _, local, _ = cr_setup.setup(cfg)
+        assert len(local) == O.num_nodes(n, L) and all(len(pairs) == c * (s + 1) ** L for pairs in local)
