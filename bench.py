@@ -498,6 +498,8 @@ def run_linreg(args, cfg):
                "repetition": B.CR_CODE_FRACTIONAL_REPETITION}[cfg["code"]]
     n, L, s, P, d, rows = cfg["n"], cfg["L"], cfg["s"], cfg["P"], cfg["d"], cfg["rows"]
     plan = B.cr_plan_create(n, L, s, P, d, code=code_id, device=0)
+    if args.tune_gradients:
+        B.cr_plan_tune_gradients(plan, *[int(x) for x in args.tune_gradients.split(",")])
     N, m, groups = B.cr_plan_num_nodes(plan), B.cr_plan_load(plan), B.cr_plan_num_groups(plan)
     logistic = cfg["kind"] == "logistic"
     loss = B.CR_LOSS_LOGISTIC if logistic else B.CR_LOSS_SQUARED
@@ -715,6 +717,8 @@ def main():
     ap.add_argument("--batch", type=int, default=0, help="aggregation workloads: straggler patterns per call")
     ap.add_argument("--rows", type=int, default=0, help="regression workloads: override the rows per partition")
     ap.add_argument("--tune", default="", help="consumer_warps,stages,ctas_per_sm,rows_per_box (0 = auto)")
+    ap.add_argument("--tune-gradients", default="", help="regression workloads: block_kb,stages,cluster of the one-pass "
+                    "gradient kernel (0 = auto)")
     ap.add_argument("--coded", action="store_true", help="regression workloads: gradient + encode in one kernel")
     ap.add_argument("--models", type=int, default=0, help="regression workloads: gradients of K models per pass (1..32)")
     ap.add_argument("--no-e2e", action="store_true")
