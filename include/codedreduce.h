@@ -92,10 +92,11 @@ typedef struct {
 
 /* Variants of cr_aggregate (low byte of `flags`) and option bits. */
 enum {
-    CR_AGG_FUSED = 0,        /* one kernel, TMA-staged tiles, all levels in registers/shared memory (single
-                                patterns whose TMA boxes would be 8 KB or less -- trees with m = 4 or 8 slot
-                                rows per node, and CR_AGG_FROM_CODED -- take the plain-load kernel unless
-                                cr_plan_tune fixed a TMA shape) */
+    CR_AGG_FUSED = 0,        /* one kernel, TMA-staged tiles, all levels in registers/shared memory.  Single
+                                patterns for which the plain-load form measures faster take it unless
+                                cr_plan_tune fixed a TMA shape: m <= 4 or m = 8 slot rows per node at
+                                d >= 2^19, m = 12, 16, .. for 2^19 <= d <= 2^23, and CR_AGG_FROM_CODED;
+                                cr_plan_last_kernel tells which kernel served a call */
     CR_AGG_FUSED_LDG = 1,    /* same dataflow with plain 128-bit loads (any d, any alignment) */
     CR_AGG_UNFUSED = 2,      /* cr_encode + cr_decode per level through the workspace */
     CR_AGG_UNCODED_SUM = 3,  /* comparator: plain sum of the same used slots, all weights 1 */
