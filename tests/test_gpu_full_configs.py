@@ -101,6 +101,21 @@ def test_paper_cluster_trees_d_2_22(name):
         assert rel_l2(got[0], O.full_gradient(G_cols)) <= REL_L2_BAR
 
 
+@pytest.mark.parametrize("n,s,code", [(12, 1, "cyclic"), (12, 3, "repetition"), (3, 1, "printed_3_1")])
+def test_flat_gradient_coding_d_2_22(n, s, code):
+    """L = 1: CodedReduce is flat gradient coding (master and n workers, m = s + 1 slot rows per worker).
+    Full-size single patterns, as `bench.py --tree n,1,s,code --d 4194304` launches them, and a batch of
+    patterns over the same slots; the result is the plain sum of the partition gradients."""
+    cfg = dict(n=n, L=1, s=s, P=O.partition_quantum(n, 1, s), d=1 << 22, code=code, seed=5, mask_seed=6, batch=1,
+               exactly_s=True, std=1.0)
+    for code_, local, got, G_cols, masks in aggregate_full(cfg, B.CR_F32, 3):
+        assert rel_l2(got[0], O.execute(code_, local, G_cols, masks[0])) <= REL_L2_BAR
+        assert rel_l2(got[0], O.full_gradient(G_cols)) <= REL_L2_BAR
+    for code_, local, got, G_cols, masks in aggregate_full(dict(cfg, batch=6, exactly_s=False), B.CR_F32, 1):
+        for b in range(6):
+            assert rel_l2(got[b], O.execute(code_, local, G_cols, masks[b])) <= REL_L2_BAR
+
+
 @pytest.mark.parametrize("s", [1, 2, 3, 5])
 @pytest.mark.parametrize("d", [5001, 6500, 120000])
 def test_paper_cluster_straggler_fractions(s, d):
