@@ -732,13 +732,13 @@ struct InlineSchedule {
 };
 
 // (Four 256-thread blocks per SM, 64 registers per thread, keep the most loads in flight; the instances
-// bounded here fit that without spilling.  The generic path of two-layer trees, which serves the short
-// launches of flat gradient coding -- two or three rows per node, a few dozen rows per thread -- gains
-// from more resident threads instead: six blocks at 40 registers (five for int32), n = 12, s = 1 at
-// d = 2^22: 4.9 -> 5.8 TB/s.  Unbounded, the four-layer float instance took 75 registers,
+// bounded here fit that without spilling.  PIPE = 5 is the generic path (PIPE = 0) for two or three rows
+// per node, the short launches of flat gradient coding with a few dozen rows per thread, which gain from
+// more resident threads instead: six blocks at 40 registers (five for int32), n = 12, s = 1 at d = 2^22:
+// 4.9 -> 5.8 TB/s.  With nine rows per node the same bound costs 14 % at d = 2^20, so it is not general.  Unbounded, the four-layer float instance took 75 registers,
 // three blocks per SM, and lost a tenth of its throughput.)
 template <typename T, int LMAX, int V, int PIPE>
-__global__ void __launch_bounds__(256, (LMAX <= 2 && PIPE == 0) ? (std::is_floating_point<T>::value ? 6 : 5)
+__global__ void __launch_bounds__(256, (LMAX <= 2 && PIPE == 5) ? (std::is_floating_point<T>::value ? 6 : 5)
                                                                      : ((LMAX <= 2 || (LMAX <= 4 && PIPE != 1)) ? 4 : 1))
 cr_fused_ldg_kernel(const T *__restrict__ G, const T *__restrict__ coeff, const Step *__restrict__ steps,
                     const int32_t *__restrict__ pat_off, int m, long long d, T *__restrict__ out, int shift,
@@ -1584,6 +1584,10 @@ static cudaError_t run_ldg_main(const AggArgs &a, dim3 grid, T *out, int shift, 
             case 4: cr_fused_ldg_kernel<T, 4, V, 1><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, shift, inl); break;
             default: cr_fused_ldg_kernel<T, 8, V, 1><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, shift, inl); break;
         }
+        return cudaGetLastError();
+    }
+    if (a.m < 4 && V == 4 && pick_lmax(a.L) == 2) {
+        cr_fused_ldg_kernel<T, 2, V, 5><<<grid, 256, 0, stream>>>(G, cf, a.steps, a.pat_off, a.m, a.d, out, shift, inl);
         return cudaGetLastError();
     }
     switch (pick_lmax(a.L)) {
