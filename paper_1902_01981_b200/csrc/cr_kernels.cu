@@ -1842,6 +1842,11 @@ cudaError_t launch_partial_gradients_fused(const float *X, const float *y, const
     if (d <= 1024) err = run_partial_fused<1>(pa, csplit, fit, items, smem, stream);
     else if (d <= 2048) err = run_partial_fused<2>(pa, csplit, fit, items, smem, stream);
     else if (d <= 4096) err = run_partial_fused<4>(pa, csplit, fit, items, smem, stream);
+    // between 4096 and 8192 in steps of 1024 columns: a thread's column groups beyond d are predicated off
+    // but still issue, and the model sizes of the paper's regressions (p = 5001, 6500) lie here
+    else if (d <= 5120) err = run_partial_fused<5>(pa, csplit, fit, items, smem, stream);
+    else if (d <= 6144) err = run_partial_fused<6>(pa, csplit, fit, items, smem, stream);
+    else if (d <= 7168) err = run_partial_fused<7>(pa, csplit, fit, items, smem, stream);
     else err = run_partial_fused<8>(pa, csplit, fit, items, smem, stream);
     if (err == cudaSuccess) ++*launches;
     return err;
