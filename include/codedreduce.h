@@ -167,7 +167,7 @@ cr_status_t cr_latency_masks(const cr_plan_t *plan, const double *compute_time, 
  * this plan ever gave up waiting for a copy.  Synchronises the device. */
 cr_status_t cr_plan_device_status(cr_plan_t *plan);
 
-/* ---- CR.Execute, step "all nodes compute their local partial gradients" (Algorithm 2) ---------
+/* ---- CR.Execute step 1, the workers' local partial gradients (Section III-A, Algorithm 2) ------
  * Linear-regression instance of Eq. (g): for every node v and slot j holding partition p,
  *   G_slots[v][j][:] = X_p^T (X_p w - y_p).
  * X [P][rows][d], y [P][rows], w [d], G_slots [N][m][d]: device pointers, fp32, row-major.
@@ -227,7 +227,9 @@ cr_status_t cr_partial_gradients_multi(cr_plan_t *plan, int32_t loss, const floa
  * has been handed in full to another component's pool, a plug-in that is given raw pointers and a
  * stream but no allocator.  For them the residuals (one float per node, slot and row) live in a fixed
  * array inside the library: 4 MiB of device memory on every GPU that loads the library, kept until the
- * process exits.  Arguments, layouts, results and kernels are those of cr_partial_gradients.
+ * process exits.  Arguments, layouts and results are those of cr_partial_gradients (squared loss);
+ * the work is always done by the two-pass kernel pair, whatever d is, since that is the form that
+ * needs the scratch.
  *   - N * m * rows must not exceed cr_partial_gradients_static_capacity() (1,048,576 residuals);
  *     larger problems return CR_ERR_OOM with an explanatory cr_last_cuda_error() text and launch nothing.
  *   - The call never allocates or frees (no cudaMalloc/cudaFree, no staging buffers, no library

@@ -207,8 +207,13 @@ def decode_row(B: np.ndarray, s: int, straggler_mask: int) -> np.ndarray:
     (Section II-C: g = a_f B G).  Solved by least squares on the consistent
     system B_U^T a_U = 1.
 
-    Pinned by the printed A for the printed B, by a B = 1 residuals and by the
-    root-equals-brute-force tests.
+    A survivor whose weight comes out of the solver as rounding noise (at most
+    1e-13 of the largest weight) gets an exact zero: the parent needs "any n-s"
+    children, and a child with zero weight is one it does not consult.
+
+    Pinned by the printed A for the printed B, by a B = 1 residuals, by the
+    root-equals-brute-force tests, and (the zeroing rule) by a 4 x 4 code whose
+    decode rows are solved by hand.
     """
     n = B.shape[0]
     U = survivors(n, s, straggler_mask)
@@ -235,7 +240,10 @@ def decode_row_repetition(n: int, s: int, straggler_mask: int) -> np.ndarray:
 
 def conditioning(B: np.ndarray, s: int) -> float:
     """kappa = max over exactly-s straggler sets of sum_j |a_j| * ||b_j||_1:
-    the worst-case amplification of rounding error by one decode."""
+    the worst-case amplification of rounding error by one decode.
+    Pinned by the hand value 5 for the code printed in Eq. gc3nodes (row norms
+    1.5, 2, 1.5 against the printed decode rows) and by its invariance under
+    rescaling a row of B."""
     n = B.shape[0]
     worst = 0.0
     for S in combinations(range(n), s):
@@ -401,7 +409,9 @@ def execute_levels(code: Code, local: list, G_parts: np.ndarray, masks):
 
 def used_nodes(code: Code, masks) -> list[int]:
     """Flat indices of the nodes whose local data enters the result for this
-    straggler pattern (children with non-zero decode weight, recursively)."""
+    straggler pattern (children with non-zero decode weight, recursively).
+    Pinned by the node sets of the worked (3,2) example written out by hand
+    and by the count sum_l (n-s)**l under exactly s stragglers per group."""
     n, L = code.n, code.L
     used = []
 
@@ -431,7 +441,8 @@ def full_gradient(G_parts: np.ndarray) -> np.ndarray:
 def partial_gradient_linreg(X: np.ndarray, y: np.ndarray, w: np.ndarray) -> np.ndarray:
     """Gradient of l(w) = 1/2 ||X w - y||^2 summed over the rows of one
     partition: X^T (X w - y), in fp64 from whatever precision the inputs have.
-    Pinned by a central finite difference of the loss."""
+    Pinned by a central finite difference of the loss and by a 2 x 2 case
+    worked by hand (gradient and loss as numbers)."""
     X = np.asarray(X, dtype=np.float64)
     return X.T @ (X @ np.asarray(w, dtype=np.float64) - np.asarray(y, dtype=np.float64))
 
@@ -457,7 +468,7 @@ def loss_logistic(X: np.ndarray, y: np.ndarray, w: np.ndarray) -> float:
 
 
 def normalized_error_rate(w: np.ndarray, w_star: np.ndarray) -> float:
-    """||w - w*||^2 / ||w*||^2 (Eq. NER)."""
+    """||w - w*||^2 / ||w*||^2 (Eq. NER).  Pinned by a two-element case worked by hand."""
     w = w.astype(np.float64)
     w_star = w_star.astype(np.float64)
     return float(np.sum((w - w_star) ** 2) / np.sum(w_star ** 2))

@@ -819,9 +819,10 @@ cr_status_t cr_partial_gradients_static(cr_plan_t *plan, const float *X, const f
         }
         scratch = g_static_ptr[plan->device];
     }
-    cudaError_t e = cr::launch_partial_gradients_two_pass(X, y, w, plan->d_part, nullptr, plan->hp.N * plan->hp.m, rows, plan->hp.d,
-                                                 scratch, G_slots, CR_LOSS_SQUARED, reinterpret_cast<cudaStream_t>(stream),
-                                                 &plan->launches);
+    // items grouped by partition, as in cr_partial_gradients, unless the plan was tuned to (node, slot) order
+    cudaError_t e = cr::launch_partial_gradients_two_pass(X, y, w, plan->d_part, plan->tune.pg_order == 1 ? nullptr : plan->d_order,
+                                                 plan->hp.N * plan->hp.m, rows, plan->hp.d, scratch, G_slots, CR_LOSS_SQUARED,
+                                                 reinterpret_cast<cudaStream_t>(stream), &plan->launches);
     if (e != cudaSuccess) { note_cuda(e, "cr_partial_gradients_static"); return CR_ERR_CUDA; }
     return CR_OK;
 }

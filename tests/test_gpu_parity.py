@@ -127,7 +127,11 @@ def test_random_patterns_medium_trees(cfg, batch, flags):
         G = inputs.partition_gradients(cfg["P"], d, seed=8)
         G_dev = slots_on_device(plan, G, torch)
         masks = inputs.straggler_masks(n, L, s, batch, seed=4, exactly_s=(n == 5))
-        bar = REL_L2_BAR if n < 12 else 1e-3     # (12,2,3): kappa in the thousands, outside the 1e-5 regime
+        # the 1e-5 bar is claimed for codes whose conditioning figure is at most 100; the random cyclic
+        # (12,2,3) code has it in the thousands and is held to 1e-3, the 0/1 repetition codes at n = 16 to 1e-5
+        kappa = O.conditioning(code.B_levels[0], s)
+        assert (kappa <= 100.0) == (cfg["code"] != "cyclic" or n < 12)
+        bar = REL_L2_BAR if kappa <= 100.0 else 1e-3
         got = run_aggregate(plan, G_dev, masks, d, flags)
         for b in range(batch):
             assert rel_l2(got[b], O.execute(code, local, G, masks[b])) <= bar

@@ -379,3 +379,83 @@ def test_pins_catch_planted_mistakes(monkeypatch):
     # wrong sign in a decode row
     monkeypatch.setattr(O, "printed_code_3_1", lambda: (np.array([[0, 1, 2], [1, 0, 1], [2, 1, 0.0]]), B))
     assert not root_ok()
+
+
+# ------------------------------------------------ hand-worked numbers (no oracle formula repeated)
+
+def test_conditioning_of_the_printed_code_by_hand():
+    """Eq. (gc3nodes): the rows of the printed B have 1-norms 1.5, 2, 1.5; the printed decode rows
+    (0,1,2), (1,0,1), (2,-1,0) then give 1*2 + 2*1.5 = 5, 1.5 + 1.5 = 3 and 2*1.5 + 1*2 = 5."""
+    _, B = O.printed_code_3_1()
+    assert abs(O.conditioning(B, 1) - 5.0) < 1e-12
+    # doubling a row of B doubles its norm and halves its decode weight: the figure does not move
+    B2 = B.copy()
+    B2[1] *= 2.0
+    assert abs(O.conditioning(B2, 1) - 5.0) < 1e-12
+    # 0/1 repetition on (4,1): decode rows are 0/1 with two ones, every row of B has norm 2
+    assert abs(O.conditioning(O.fractional_repetition_code(4, 1), 1) - 4.0) < 1e-12
+
+
+def test_used_nodes_of_the_worked_example_by_hand():
+    """Section III-B example on the (3,2) tree: with child 2 of the master straggling the master
+    listens to (1,1) and (1,3); (1,1) with its child 3 straggling listens to (2,1), (2,2); (1,3) without
+    a straggler takes its two lowest children (2,7), (2,8).  Flat indices: layer 1 = 0..2, layer 2 = 3..11."""
+    code = make_code("printed", 3, 2, 1)
+    assert O.used_nodes(code, [0b010, 0b100, 0, 0]) == [0, 2, 3, 4, 9, 10]
+    # child 1 of the master straggles -> (1,2), (1,3); (1,2) loses its child 2 -> (2,4), (2,6);
+    # (1,3) loses its child 1 -> (2,8), (2,9).  The mask below the straggler (group 1) is never read.
+    assert O.used_nodes(code, [0b001, 0b111, 0b010, 0b001]) == [1, 2, 6, 8, 10, 11]
+
+
+@pytest.mark.parametrize("name,count", [("cfg2", 12), ("cfg3", 12), ("cfg4", 12), ("cfg5", 30)])
+def test_used_node_count_with_exactly_s_stragglers(name, count):
+    """With exactly s stragglers per group a parent consults exactly n-s children, so a pattern
+    consumes sum_l (n-s)^l nodes: 3+9 for the (4,2,1) and (5,2,2) trees, 2+4+8+16 for (3,4,1)."""
+    from oracle import cr_setup
+    cfg = inputs.CONFIGS[name]
+    n, L, s = cfg["n"], cfg["L"], cfg["s"]
+    code = cr_setup.code_for(cfg)
+    masks = inputs.straggler_masks(n, L, s, 5, seed=21, exactly_s=True)
+    for b in range(5):
+        used = O.used_nodes(code, masks[b])
+        assert len(used) == count == sum((n - s) ** l for l in range(1, L + 1))
+        assert len(set(used)) == len(used)
+        # exactly n-s of every consulted parent's children, and the master's
+        assert sum(1 for v in used if v < n) == n - s
+
+
+def test_linear_regression_gradient_and_loss_by_hand():
+    """Eq. (g) with the squared loss on X = [[1,2],[3,4]], y = (0,1), w = (1,-1): X w = (-1,-1), residual
+    (-1,-2), loss (1+4)/2, gradient X^T r = (1*-1 + 3*-2, 2*-1 + 4*-2)."""
+    X = np.array([[1.0, 2.0], [3.0, 4.0]], dtype=np.float32)
+    y = np.array([0.0, 1.0], dtype=np.float32)
+    w = np.array([1.0, -1.0], dtype=np.float32)
+    assert np.array_equal(O.partial_gradient_linreg(X, y, w), np.array([-7.0, -10.0]))
+    assert O.loss_linreg(X, y, w) == 2.5
+    assert O.partial_gradient_linreg(X, y, w).dtype == np.float64
+
+
+def test_normalized_error_rate_by_hand():
+    """Eq. (NER): w = (1,2), w* = (3,4): (4 + 4) / (9 + 16)."""
+    assert O.normalized_error_rate(np.array([1.0, 2.0], dtype=np.float32), np.array([3.0, 4.0], dtype=np.float32)) == 8.0 / 25.0
+    assert O.normalized_error_rate(np.zeros(2), np.array([3.0, 4.0])) == 1.0
+
+
+def test_unneeded_survivor_gets_an_exact_zero():
+    """CR.Execute lets a parent recover from ANY n-s children.  For B with rows (1,1,0,0), (0,0,1,1),
+    (1,0,2,0), (0,1,0,2) and s = 1 the three lowest survivors are more than needed in two cases: solving
+    a B_U = 1 by hand gives a = (1,1,0,0) without a straggler and with child 3 or child 4 straggling --
+    the third survivor's weight is zero, so that child (and its sub-tree) is not consulted -- while
+    child 1 straggling needs three children, a = (0,-1,1,1), and child 2 straggling a = (1/2,0,1/2,1/2)."""
+    Bx = np.array([[1, 1, 0, 0], [0, 0, 1, 1], [1, 0, 2, 0], [0, 1, 0, 2]], dtype=np.float64)
+    for mask, want in ((0b0000, [1, 1, 0, 0]), (0b1000, [1, 1, 0, 0]), (0b0100, [1, 1, 0, 0]),
+                       (0b0001, [0, -1, 1, 1]), (0b0010, [0.5, 0, 0.5, 0.5])):
+        a = O.decode_row(Bx, 1, mask)
+        assert np.allclose(a, want, atol=1e-14)
+        assert all(a[j] == 0.0 for j in range(4) if want[j] == 0)      # exact zeros, not rounding noise
+        assert np.allclose(a @ Bx, 1.0, atol=1e-14)
+    code = O.Code(4, 2, 1, [Bx, Bx], kind="solve")
+    # master without straggler: children 1, 2 only; each of them, without straggler, its children 1, 2
+    assert O.used_nodes(code, [0, 0, 0, 0, 0]) == [0, 1, 4, 5, 8, 9]
+    # child 1 of the master straggles: children 2, 3, 4 are all needed
+    assert sorted(v for v in O.used_nodes(code, [1, 0, 0, 0, 0]) if v < 4) == [1, 2, 3]

@@ -1,4 +1,4 @@
-"""The allocation-free partial-gradient entry point against the ordinary one.
+"""The allocation-free partial-gradient entry point against the ordinary one and the CPU oracle.
 
 Collected last on purpose (file name): a run that stops at the first failure has then already run
 every other test.  The entry point serves callers that cannot obtain device memory for the
@@ -9,6 +9,7 @@ and a stream -- by keeping that workspace in a fixed array inside the library.
 import numpy as np
 import pytest
 
+from oracle import cr_oracle as O
 from paper_1902_01981_b200 import binding as B
 from paper_1902_01981_b200 import build as cr_build
 from paper_1902_01981_b200 import inputs
@@ -32,7 +33,8 @@ def test_static_scratch_variant_matches_workspace_variant_twice():
         # two calls in a row, on different models: the second finds the first one's residuals in the
         # shared array and must not be affected by them
         for call, seed in enumerate((32, 33)):
-            w_dev = torch.from_numpy(inputs.model_vector(d, seed)).cuda()
+            w = inputs.model_vector(d, seed)
+            w_dev = torch.from_numpy(w).cuda()
             want = torch.zeros((N, m, d), device="cuda")
             got = torch.full((N, m, d), float("nan"), device="cuda")
             B.cr_partial_gradients(plan, X_dev, y_dev, rows, w_dev, want, ws)
@@ -42,6 +44,11 @@ def test_static_scratch_variant_matches_workspace_variant_twice():
             assert np.isfinite(got_h).all()
             worst = max(rel_l2(got_h[v, j], want_h[v, j]) for v in range(N) for j in range(m))
             assert worst <= REL_L2_BAR, f"call {call}: {worst:.2e}"
+            # and against the definition, X_p^T (X_p w - y_p) in fp64, slot by slot
+            part = B.slot_partitions(plan)
+            truth = [O.partial_gradient_linreg(X[p], y[p], w) for p in range(P)]
+            worst = max(rel_l2(got_h[v, j], truth[part[v, j]]) for v in range(N) for j in range(m))
+            assert worst <= REL_L2_BAR, f"call {call} against the oracle: {worst:.2e}"
         # a problem beyond the fixed scratch is refused before anything is launched
         too_many = B.cr_partial_gradients_static_capacity() // (N * m) + 1
         launches = B.cr_plan_launch_count(plan)
