@@ -323,6 +323,8 @@ def run_ours(args, cfg):
                             dtype=B.CR_I32 if is_int else B.CR_F32, seed=0, device=local_rank)
     if args.tune:
         B.cr_plan_tune(plan, *[int(x) for x in args.tune.split(",")])
+    if args.share or args.e_buffers:
+        B.cr_plan_tune_batch(plan, args.share, args.e_buffers)
     N, m, groups = B.cr_plan_num_nodes(plan), B.cr_plan_load(plan), B.cr_plan_num_groups(plan)
     d, batch = cfg["d"], cfg.get("batch", 1)
     tdtype = torch.int32 if is_int else torch.float32
@@ -719,6 +721,9 @@ def main():
     ap.add_argument("--tune", default="", help="consumer_warps,stages,ctas_per_sm,rows_per_box (0 = auto)")
     ap.add_argument("--tune-gradients", default="", help="regression workloads: block_kb,stages,cluster of the one-pass "
                     "gradient kernel (0 = auto)")
+    ap.add_argument("--share", type=int, default=0, help="batches: messages shared by the patterns: 0 built-in choice, "
+                    "1 never, 2 whenever possible")
+    ap.add_argument("--e-buffers", type=int, default=0, help="batches: buffers of coded gradients in shared memory (1, 2)")
     ap.add_argument("--coded", action="store_true", help="regression workloads: gradient + encode in one kernel")
     ap.add_argument("--models", type=int, default=0, help="regression workloads: gradients of K models per pass (1..32)")
     ap.add_argument("--no-e2e", action="store_true")

@@ -47,6 +47,7 @@ extern "C" {
 #endif
 
 typedef struct cr_plan cr_plan_t;
+typedef struct cr_schedule cr_schedule_t;
 
 typedef enum {
     CR_OK = 0,
@@ -121,8 +122,11 @@ typedef enum {
  * increasing kappa, keeps the first m = r_CR * P pairs (Theorem 1) and passes the rest down.  It also
  * solves, in fp64, the decode row a (a B = 1, supported on the lowest-indexed n-s non-stragglers)
  * for every straggler mask with at most s bits, per level.  With device >= 0 it makes that device
- * current for the call, allocates small device mirrors of the tables and a ring of pinned staging
- * buffers; cr_plan_destroy frees them.  *out is written only on CR_OK. */
+ * current for the call and allocates small device mirrors of the tables and a ring of eight staging
+ * buffers (pinned host + device, 64 KB each or 64 bytes per node if that is more), through which
+ * cr_aggregate and cr_decode send the expanded straggler patterns.  A call whose tables exceed a slot
+ * (a large batch) re-allocates that slot once, which synchronises the device; cr_schedule_create keeps
+ * even that out of a loop.  cr_plan_destroy frees everything.  *out is written only on CR_OK. */
 cr_status_t cr_plan_create(const cr_plan_desc_t *desc, cr_plan_t **out);
 cr_status_t cr_plan_destroy(cr_plan_t *plan);
 
@@ -163,9 +167,20 @@ cr_status_t cr_plan_expand(const cr_plan_t *plan, const uint32_t *masks, int32_t
 cr_status_t cr_latency_masks(const cr_plan_t *plan, const double *compute_time, double t_c, uint32_t *masks_out,
                              double *t_total);
 
-/* Sticky status word written by bounded device-side waits: CR_OK, or CR_ERR_TIMEOUT if a kernel of
- * this plan ever gave up waiting for a copy.  Synchronises the device. */
+/* Status word written by bounded device-side waits: CR_OK, or CR_ERR_TIMEOUT if a kernel of this plan
+ * gave up waiting for a copy.  The word is sticky on purpose -- results produced after a timeout are
+ * not to be trusted until someone has looked -- and stays set until cr_plan_clear_status.  Both calls
+ * synchronise the device. */
 cr_status_t cr_plan_device_status(cr_plan_t *plan);
+cr_status_t cr_plan_clear_status(cr_plan_t *plan);
+/* Bound of every device-side wait of this plan's kernels, in nanoseconds (default 2e9; accepted range
+ * 1e3 .. 6e10).  It travels to the kernels as an argument of each launch. */
+cr_status_t cr_plan_set_wait_limit(cr_plan_t *plan, uint64_t limit_ns);
+/* Shows the give-up path without harming anything: enqueues one small kernel whose single thread waits
+ * limit_ns (1e3 .. 1e8) on a barrier that nobody completes, through the same bounded wait as the
+ * aggregation and gradient kernels, and then sets the status word as they would.  No copy is in flight
+ * and nothing traps; afterwards cr_plan_device_status returns CR_ERR_TIMEOUT until the word is cleared. */
+cr_status_t cr_selftest_wait(cr_plan_t *plan, uint64_t limit_ns, void *stream);
 
 /* ---- CR.Execute step 1, the workers' local partial gradients (Section III-A, Algorithm 2) ------
  * Linear-regression instance of Eq. (g): for every node v and slot j holding partition p,
@@ -269,6 +284,23 @@ size_t cr_aggregate_workspace_bytes(const cr_plan_t *plan, int32_t batch, uint32
 cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *masks_host, int32_t batch,
                          void *g_out, uint32_t flags, void *workspace, size_t workspace_bytes, void *stream);
 
+/* ---- CR.Execute with the straggler sets fixed in advance ------------------------------------------
+ * The straggler sets are an input of CR.Execute (Algorithm 2); everything cr_aggregate derives from them
+ * -- the post-order list of consumed nodes with their decode weights, the union of a batch, the tables
+ * of the batch kernel -- depends on the masks alone, not on the gradients.  cr_schedule_create does that
+ * work once for `batch` patterns (masks_host [batch][num_groups], host) and `flags` (as cr_aggregate) and
+ * keeps the tables in device memory it allocates; cr_aggregate_scheduled then only launches: no mask is
+ * validated or expanded, nothing is allocated and nothing is copied.  A schedule belongs to its plan,
+ * may be used any number of times, by one stream at a time like the plan itself, and must be destroyed
+ * before the plan.  Results are those of cr_aggregate with the same masks and flags, bit for bit.
+ * cr_schedule_bytes: the algorithmic bytes of one call (as cr_aggregate_bytes). */
+cr_status_t cr_schedule_create(cr_plan_t *plan, const uint32_t *masks_host, int32_t batch, uint32_t flags,
+                               cr_schedule_t **out);
+cr_status_t cr_schedule_destroy(cr_schedule_t *sched);
+cr_status_t cr_schedule_bytes(const cr_schedule_t *sched, int64_t *bytes, int32_t *used_nodes);
+cr_status_t cr_aggregate_scheduled(cr_plan_t *plan, const void *G_slots, const cr_schedule_t *sched, void *g_out,
+                                   void *workspace, size_t workspace_bytes, void *stream);
+
 /* Same computation with HOST buffers: copies from G_slots_host (pinned or pageable host memory,
  * [N][m][d]) into dev_slots the slots of the nodes that the batch consumes (the rest of dev_slots is
  * left as it is: a straggler's data is never waited for; all nodes with CR_AGG_ALL_NODES), runs
@@ -293,6 +325,15 @@ cr_status_t cr_aggregate_bytes(const cr_plan_t *plan, const uint32_t *masks_host
  * above.  Shapes that do not fit shared memory fall back to smaller ones or to plain loads. */
 cr_status_t cr_plan_tune(cr_plan_t *plan, int32_t consumer_warps, int32_t stages, int32_t ctas_per_sm,
                          int32_t rows_per_box);
+
+/* Batches of patterns (CR_AGG_FUSED, batch > 1, L >= 2): a parent's message depends only on the straggler
+ * sets of its own sub-tree (CR.Execute), so the patterns of a batch can share the messages of the nodes
+ * whose children are leaves.  share_messages: 0 = share when it halves the replay work (built-in
+ * choice), 1 = never, 2 = whenever the tables fit.  Read when a batch is expanded
+ * (cr_aggregate, cr_schedule_create).  e_buffers: buffers of coded gradients the batch kernel keeps in
+ * shared memory, 0 = built-in choice (two when they fit beside tall boxes), 1 or 2; one buffer leaves
+ * room for more and deeper loader rings (cr_plan_tune). */
+cr_status_t cr_plan_tune_batch(cr_plan_t *plan, int32_t share_messages, int32_t e_buffers);
 
 /* Launch shape of the one-pass partial-gradient kernel; 0 keeps the built-in choice for that field.
  * block_kb = KB of X per staged row block (1..128), stages = row-block buffers per CTA (2..8),

@@ -61,6 +61,15 @@ _SIGNATURES = {
                                  C.POINTER(C.c_int32)]),
     "cr_latency_masks": (C.c_int, [C.c_void_p, C.c_void_p, C.c_double, C.c_void_p, C.POINTER(C.c_double)]),
     "cr_plan_device_status": (C.c_int, [C.c_void_p]),
+    "cr_plan_clear_status": (C.c_int, [C.c_void_p]),
+    "cr_plan_set_wait_limit": (C.c_int, [C.c_void_p, C.c_uint64]),
+    "cr_selftest_wait": (C.c_int, [C.c_void_p, C.c_uint64, C.c_void_p]),
+    "cr_plan_tune_batch": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32]),
+    "cr_schedule_create": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_uint32, C.POINTER(C.c_void_p)]),
+    "cr_schedule_destroy": (C.c_int, [C.c_void_p]),
+    "cr_schedule_bytes": (C.c_int, [C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_int32)]),
+    "cr_aggregate_scheduled": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t,
+                                         C.c_void_p]),
     "cr_partial_gradients_workspace_bytes": (C.c_size_t, [C.c_void_p, C.c_int32]),
     "cr_partial_gradients": (C.c_int, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p, C.c_void_p,
                                        C.c_void_p, C.c_size_t, C.c_void_p]),
@@ -248,6 +257,23 @@ def cr_plan_device_status(plan: int) -> int:
     return lib().cr_plan_device_status(plan)
 
 
+def cr_plan_clear_status(plan: int) -> None:
+    _check(lib().cr_plan_clear_status(plan), "cr_plan_clear_status")
+
+
+def cr_plan_set_wait_limit(plan: int, limit_ns: int) -> None:
+    _check(lib().cr_plan_set_wait_limit(plan, limit_ns), "cr_plan_set_wait_limit")
+
+
+def cr_selftest_wait(plan: int, limit_ns: int, stream=None) -> None:
+    """Enqueues the kernel that lets one bounded wait run out (see codedreduce.h)."""
+    _check(lib().cr_selftest_wait(plan, limit_ns, _stream_ptr(stream)), "cr_selftest_wait")
+
+
+def cr_plan_tune_batch(plan: int, share_messages: int = 0, e_buffers: int = 0) -> None:
+    _check(lib().cr_plan_tune_batch(plan, share_messages, e_buffers), "cr_plan_tune_batch")
+
+
 def cr_plan_tune(plan: int, consumer_warps: int = 0, stages: int = 0, ctas_per_sm: int = 0,
                  rows_per_box: int = 0) -> None:
     _check(lib().cr_plan_tune(plan, consumer_warps, stages, ctas_per_sm, rows_per_box), "cr_plan_tune")
@@ -333,6 +359,42 @@ def cr_aggregate(plan: int, G_slots, masks, g_out, flags: int = CR_AGG_FUSED, wo
                               _dev_ptr(workspace),
                               0 if workspace is None else workspace.numel() * workspace.element_size(),
                               _stream_ptr(stream)), "cr_aggregate")
+
+
+def cr_schedule_create(plan: int, masks, flags: int = CR_AGG_FUSED) -> int:
+    """Expands masks [batch, groups] (or [groups]) once; returns an opaque schedule handle."""
+    mk = _masks(masks, _num_groups(plan))
+    out = C.c_void_p()
+    _check(lib().cr_schedule_create(plan, mk.ctypes.data, mk.shape[0], flags, C.byref(out)), "cr_schedule_create")
+    return out.value
+
+
+def cr_schedule_destroy(sched: int) -> None:
+    _check(lib().cr_schedule_destroy(sched), "cr_schedule_destroy")
+
+
+def cr_schedule_bytes(sched: int):
+    """(algorithmic bytes, size of the union of used nodes) of one call with this schedule."""
+    nbytes, used = C.c_int64(), C.c_int32()
+    _check(lib().cr_schedule_bytes(sched, C.byref(nbytes), C.byref(used)), "cr_schedule_bytes")
+    return nbytes.value, used.value
+
+
+def _ptr_and_bytes(t):
+    return (0, 0) if t is None else (_dev_ptr(t), t.numel() * t.element_size())
+
+
+def cr_aggregate_scheduled(plan: int, G_slots, sched: int, g_out, workspace=None, stream=None) -> None:
+    """cr_aggregate with a schedule made by cr_schedule_create.  G_slots / g_out / workspace are torch
+    CUDA tensors, or plain integer device addresses (workspace then as (address, bytes)) for loops that
+    do not want to pay for the tensor look-ups; stream likewise a torch stream, None or a raw handle."""
+    g = G_slots if isinstance(G_slots, int) else _dev_ptr(G_slots)
+    o = g_out if isinstance(g_out, int) else _dev_ptr(g_out)
+    w, wb = workspace if isinstance(workspace, tuple) else _ptr_and_bytes(workspace)
+    st = stream if isinstance(stream, int) else _stream_ptr(stream)
+    rc = lib().cr_aggregate_scheduled(plan, g, sched, o, w, wb, st)
+    if rc != CR_OK:
+        raise CodedReduceError(rc, "cr_aggregate_scheduled")
 
 
 def cr_aggregate_host(plan: int, G_slots_host, masks, g_out_host, dev_slots, dev_out, flags: int = CR_AGG_FUSED,

@@ -6,6 +6,7 @@
 #include <algorithm>
 #include <cstdio>
 #include <cstring>
+#include <map>
 #include <mutex>
 #include <new>
 #include <vector>
@@ -112,14 +113,24 @@ uint32_t weight_bits(const cr::HostPlan &hp, double w) {
 }
 
 struct Expanded {
-    std::vector<cr::Step> steps;       // all patterns, concatenated
+    std::vector<cr::Step> steps;       // all patterns, concatenated: every consumed node in post-order
     std::vector<int32_t> pat_off;      // [batch+1]
     std::vector<int32_t> unodes;       // union of used nodes, ascending
     std::vector<uint32_t> wtab;        // distinct decode-weight bit patterns of the batch (empty: none / too many)
     std::vector<std::vector<cr::UsedNode>> per_pattern;
+    // Messages shared by the patterns of a batch (batch kernel).  The message of a node of layer L-1, whose
+    // children are leaves, depends only on the decode row of its own group, so the batch needs one copy per
+    // distinct row.  `ops` lists those nodes, `vtab` their weight records and variant lists (layouts: BatchArgs), and the
+    // reduced schedules name a message row where the full ones have the node and its leaves.
+    std::vector<int4> ops;
+    std::vector<uint32_t> vtab;
+    std::vector<cr::Step> red_steps;
+    std::vector<int32_t> red_off;
+    int n_rows = 0;                    // rows of an E buffer: the union, then extra message rows
 };
 
-cr_status_t expand_all(const cr::HostPlan &hp, const uint32_t *masks, int batch, Expanded &ex) {
+// share: 0 = build the shared-message tables when they save replay work, 1 = never, 2 = whenever possible
+cr_status_t expand_all(const cr::HostPlan &hp, const uint32_t *masks, int batch, int share, Expanded &ex) {
     std::vector<int32_t> pos(hp.N, -1);
     ex.pat_off.assign(1, 0);
     ex.per_pattern.resize(batch);
@@ -135,12 +146,13 @@ cr_status_t expand_all(const cr::HostPlan &hp, const uint32_t *masks, int batch,
     // index of the step's weight in the table of distinct weights: the batch kernel can then keep a
     // 4-byte entry per step and pattern in shared memory.
     bool table_ok = batch > 1 && ex.unodes.size() <= 4096;
+    std::vector<int32_t> widx;   // per step: index of its weight in the table
     for (int b = 0; b < batch; ++b) {
         for (const cr::UsedNode &u : ex.per_pattern[b]) {
             const uint32_t wb = weight_bits(hp, u.weight);
             int32_t index = pos[u.node];
+            size_t wi = 0;
             if (table_ok) {
-                size_t wi = 0;
                 while (wi < ex.wtab.size() && ex.wtab[wi] != wb) ++wi;
                 if (wi == ex.wtab.size()) {
                     if (ex.wtab.size() >= 1024) table_ok = false;
@@ -148,6 +160,7 @@ cr_status_t expand_all(const cr::HostPlan &hp, const uint32_t *masks, int batch,
                 }
                 if (table_ok) index |= (int32_t)(wi << 12);
             }
+            widx.push_back((int32_t)wi);
             ex.steps.push_back(cr::Step{u.node, u.layer | (u.first ? 0x100 : 0), wb, index});
         }
         ex.pat_off.push_back((int32_t)ex.steps.size());
@@ -156,8 +169,103 @@ cr_status_t expand_all(const cr::HostPlan &hp, const uint32_t *masks, int batch,
         ex.wtab.clear();
         for (cr::Step &st : ex.steps) st.index = pos[st.node];   // plain positions
     }
+    ex.n_rows = (int)ex.unodes.size();
+    if (!table_ok || batch < 2 || hp.L < 2 || share == 1) return CR_OK;
+
+    // ---- shared messages of the bottom layer (parents of the leaves) ----
+    const int lb = hp.L - 1;
+    struct Build {
+        int own_row, child_row0, cnt;
+        std::vector<std::vector<uint32_t>> weights;   // per variant: decode weights of the children in the union
+        std::vector<int> dst;                          // per variant: row of its message
+    };
+    std::vector<Build> builds;
+    std::vector<int32_t> op_of(hp.N, -1);
+    int extra = 0;
+    ex.red_off.assign(1, 0);
+    std::vector<uint32_t> key;
+    for (int b = 0; b < batch; ++b) {
+        const std::vector<cr::UsedNode> &pp = ex.per_pattern[b];
+        const size_t base = (size_t)ex.pat_off[b];
+        size_t leaf_from = 0;   // the leaves since the last inner node are the children of the next bottom node
+        for (size_t k = 0; k < pp.size(); ++k) {
+            const cr::UsedNode &u = pp[k];
+            if (u.layer == hp.L) continue;
+            if (u.layer != lb) {
+                ex.red_steps.push_back(ex.steps[base + k]);
+                leaf_from = k + 1;
+                continue;
+            }
+            int32_t &op = op_of[u.node];
+            if (op < 0) {
+                op = (int32_t)builds.size();
+                Build nb;
+                nb.own_row = pos[u.node];
+                const int first_child = hp.layer_offset[hp.L] + (u.node - hp.layer_offset[lb]) * hp.n;
+                nb.child_row0 = -1; nb.cnt = 0;
+                for (int j = 0; j < hp.n; ++j)
+                    if (pos[first_child + j] >= 0) { if (nb.child_row0 < 0) nb.child_row0 = pos[first_child + j]; ++nb.cnt; }
+                builds.push_back(nb);
+            }
+            Build &bd = builds[op];
+            key.assign((size_t)bd.cnt, 0u);
+            for (size_t c = leaf_from; c < k; ++c) key[(size_t)(pos[pp[c].node] - bd.child_row0)] = ex.steps[base + c].wbits;
+            size_t v = 0;
+            while (v < bd.weights.size() && bd.weights[v] != key) ++v;
+            if (v == bd.weights.size()) {
+                // the node's own row and its children's rows are dead once its variants are formed: they hold
+                // the first variants, the others go behind the union
+                const int reuse = 1 + bd.cnt;
+                bd.dst.push_back((int)v == 0 ? bd.own_row : ((int)v < reuse ? bd.child_row0 + (int)v - 1 : ex.n_rows + extra++));
+                bd.weights.push_back(key);
+            }
+            cr::Step st = ex.steps[base + k];
+            st.layer |= 0x200;   // a complete message: no children of its own in the reduced schedule
+            st.index = bd.dst[v] | (widx[base + k] << 12);
+            ex.red_steps.push_back(st);
+            leaf_from = k + 1;
+        }
+        ex.red_off.push_back((int32_t)ex.red_steps.size());
+    }
+    // Replay work in rows of shared memory read or written per tile: every schedule entry one row; with shared
+    // messages the reduced entries plus, per bottom node, its own row, its children and its variants.  Sharing
+    // is taken when it halves that work.  Measured (64 patterns, ms per launch without / with): (12,2,1) at
+    // d = 2^20 4.85 / 1.08, (4,3,1) 1.39 / 0.63 (ratios 0.32 and 0.37); (3,4,1) at d = 2^22, ratio 0.57, where the
+    // loads already set the pace: 5.12 / 5.15.
+    size_t work_new = ex.red_steps.size();
+    for (const Build &bd : builds) work_new += 1 + (size_t)bd.cnt + bd.weights.size();
+    const bool pays = share == 2 || work_new * 2 <= ex.steps.size();
+    if (!pays || ex.n_rows + extra > 4096) {
+        ex.red_steps.clear(); ex.red_off.clear();
+        return CR_OK;
+    }
+    ex.n_rows += extra;
+    // weight records first (padded to four words, equal ones stored once: with the whole tree in the union
+    // the nodes of a level all use the same few decode rows), then the variant lists of the nodes
+    std::map<std::vector<uint32_t>, uint32_t> record_at;
+    std::vector<std::vector<uint32_t>> rec_of(builds.size());
+    for (size_t o = 0; o < builds.size(); ++o) {
+        for (std::vector<uint32_t> w : builds[o].weights) {
+            w.resize((w.size() + 3) & ~(size_t)3, 0u);
+            auto it = record_at.find(w);
+            if (it == record_at.end()) {
+                it = record_at.emplace(w, (uint32_t)ex.vtab.size()).first;
+                ex.vtab.insert(ex.vtab.end(), w.begin(), w.end());
+            }
+            rec_of[o].push_back(it->second);
+        }
+    }
+    for (size_t o = 0; o < builds.size(); ++o) {
+        const Build &bd = builds[o];
+        ex.ops.push_back(make_int4(bd.own_row, bd.child_row0, bd.cnt | ((int)bd.weights.size() << 8), (int)ex.vtab.size()));
+        for (size_t v = 0; v < bd.weights.size(); ++v) {
+            ex.vtab.push_back((uint32_t)bd.dst[v]);
+            ex.vtab.push_back(rec_of[o][v]);
+        }
+    }
     return CR_OK;
 }
+
 
 cr_status_t check_device_plan(cr_plan *p) {
     if (!p) return CR_ERR_INVALID_ARG;
@@ -269,6 +377,17 @@ cr_status_t cr_plan_create(const cr_plan_desc_t *desc, cr_plan_t **out) {
         // here, so that no device call ever allocates
         if (p->hp.L >= 2 && p->hp.d <= kSplitMaxD && p->hp.n >= kSplitMinSubtrees && p->hp.n <= cr::split_limit())
             CR_CUDA_P(cudaMalloc(&p->d_split, (size_t)p->hp.n * (size_t)p->hp.d * 4));
+        // staging ring for the expanded schedules: sized here for single patterns and small batches, so
+        // that the device calls of an ordinary loop never allocate (a larger batch grows its slot once)
+        {
+            const size_t cap = std::max<size_t>(64 * 1024, align16((size_t)p->hp.N * 64));
+            for (StageSlot &s : p->ring) {
+                CR_CUDA_P(cudaMallocHost(reinterpret_cast<void **>(&s.host), cap));
+                CR_CUDA_P(cudaMalloc(reinterpret_cast<void **>(&s.dev), cap));
+                CR_CUDA_P(cudaEventCreateWithFlags(&s.ev, cudaEventDisableTiming));
+                s.bytes = cap;
+            }
+        }
         // cuTensorMapEncodeTiled through the runtime, so that the library needs no link to libcuda
         void *fn = nullptr;
         cudaDriverEntryPointQueryResult qres;
@@ -369,11 +488,42 @@ cr_status_t cr_plan_device_status(cr_plan_t *plan) {
     return word == 0 ? CR_OK : CR_ERR_TIMEOUT;
 }
 
+cr_status_t cr_plan_clear_status(cr_plan_t *plan) {
+    cr_status_t st = check_device_plan(plan);
+    if (st != CR_OK) return st;
+    CR_CUDA(cudaDeviceSynchronize());
+    CR_CUDA(cudaMemset(plan->d_status, 0, sizeof(int)));
+    return CR_OK;
+}
+
+cr_status_t cr_plan_set_wait_limit(cr_plan_t *plan, uint64_t limit_ns) {
+    if (!plan || limit_ns < 1000 || limit_ns > 60000000000ull) return CR_ERR_INVALID_ARG;
+    plan->tune.wait_limit_ns = limit_ns;
+    return CR_OK;
+}
+
+cr_status_t cr_selftest_wait(cr_plan_t *plan, uint64_t limit_ns, void *stream) {
+    cr_status_t st = check_device_plan(plan);
+    if (st != CR_OK) return st;
+    // a bounded range: the self-test is there to show the give-up path, not to hold the GPU
+    if (limit_ns < 1000 || limit_ns > 100000000ull) return CR_ERR_INVALID_ARG;
+    cudaError_t e = cr::launch_wait_selftest(plan->d_status, limit_ns, reinterpret_cast<cudaStream_t>(stream), &plan->launches);
+    if (e != cudaSuccess) { note_cuda(e, "cr_selftest_wait"); return CR_ERR_CUDA; }
+    return CR_OK;
+}
+
+cr_status_t cr_plan_tune_batch(cr_plan_t *plan, int32_t share_messages, int32_t e_buffers) {
+    if (!plan || share_messages < 0 || share_messages > 2 || e_buffers < 0 || e_buffers > 2) return CR_ERR_INVALID_ARG;
+    plan->tune.share = share_messages;
+    plan->tune.e_buffers = e_buffers;
+    return CR_OK;
+}
+
 cr_status_t cr_aggregate_bytes(const cr_plan_t *plan, const uint32_t *masks_host, int32_t batch, int64_t *bytes,
                                int32_t *used_nodes) {
     if (!plan || !masks_host || batch < 1 || !bytes) return CR_ERR_INVALID_ARG;
     Expanded ex;
-    cr_status_t st = expand_all(plan->hp, masks_host, batch, ex);
+    cr_status_t st = expand_all(plan->hp, masks_host, batch, 1, ex);
     if (st != CR_OK) return st;
     *bytes = 4ll * plan->hp.d * ((int64_t)plan->hp.m * (int64_t)ex.unodes.size() + batch);
     if (used_nodes) *used_nodes = (int32_t)ex.unodes.size();
@@ -404,7 +554,7 @@ cr_status_t cr_partial_gradients_loss(cr_plan_t *plan, int32_t loss, const float
         // items grouped by partition unless the caller asked for (node, slot) order: the items that hold the
         // same partition then read its rows from HBM once and share them through L2
         e = cr::launch_partial_gradients_two_pass(X, y, w, plan->d_part, plan->tune.pg_order == 1 ? nullptr : plan->d_order, items, rows, plan->hp.d,
-                                                  reinterpret_cast<float *>(workspace), G_slots, loss,
+                                                  reinterpret_cast<float *>(workspace), G_slots, loss, plan->dev.sm_count,
                                                   reinterpret_cast<cudaStream_t>(stream), &plan->launches);
     }
     if (e != cudaSuccess) { note_cuda(e, "cr_partial_gradients"); return CR_ERR_CUDA; }
@@ -500,8 +650,10 @@ cr_status_t cr_decode(cr_plan_t *plan, int32_t parent_layer, const void *M_child
     const int shift = (hp.dtype == CR_I32 && parent_layer == 0) ? hp.int_shift : 0;
     cudaError_t e = cr::launch_decode(M_child, E_parent, slot->dev, nullptr, parents, hp.n, hp.d, M_parent, shift,
                                       hp.dtype == CR_I32, s, &plan->launches);
+    // the slot is guarded by an event on the error path too: its copy may still be queued
+    st = stage_release(slot, s);
     if (e != cudaSuccess) { note_cuda(e, "cr_decode"); return CR_ERR_CUDA; }
-    return stage_release(slot, s);
+    return st;
 }
 
 size_t cr_aggregate_workspace_bytes(const cr_plan_t *plan, int32_t batch, uint32_t flags) {
@@ -514,51 +666,135 @@ size_t cr_aggregate_workspace_bytes(const cr_plan_t *plan, int32_t batch, uint32
     return (size_t)(hp.N + nonleaf) * (size_t)hp.d * 4;
 }
 
-static cr_status_t aggregate_unfused(cr_plan *plan, const void *G_slots, const uint32_t *masks_host, int batch,
-                                     void *g_out, bool all_nodes, void *workspace, const Expanded &ex,
-                                     cudaStream_t s) {
+}  // extern "C"
+
+namespace {
+
+// A batch of straggler patterns, expanded: everything cr_aggregate derives from the masks before it can
+// launch, with the tables the kernels read laid out as one block of bytes (`blob`) ready to be copied to
+// the device.  Built per call by cr_aggregate, once by cr_schedule_create.
+struct Prepared {
+    int batch = 0;
+    uint32_t flags = 0, variant = 0;
+    Expanded ex;
+    int same_shape = 1;       // fused forms: all full schedules share length and layer sequence
+    int red_same_shape = 1;   // the same for the reduced schedules (shared messages)
+    int subtrees = 0;         // single pattern: consumed children of the master
+    int m_eff = 0;            // slot rows per node as the kernels see them (1 when the input is coded gradients)
+    std::vector<unsigned char> blob;
+    // fused forms: offsets of the tables inside the blob
+    size_t off_steps = 0, off_pat = 0, off_unodes = 0, off_wtab = 0, off_boxes = 0, off_ops = 0, off_vtab = 0,
+           off_red_steps = 0, off_red_pat = 0;
+    int n_boxes = 0, npb = 1;
+    // unfused form: per pattern and level the weight rows and the active flags
+    std::vector<size_t> w_off, a_off;
+    size_t per_pattern = 0, nodes_bytes = 0;
+};
+
+bool same_layers(const std::vector<cr::Step> &steps, const std::vector<int32_t> &off, int batch) {
+    const int32_t len = off[1] - off[0];
+    for (int b = 1; b < batch; ++b) {
+        if (off[b + 1] - off[b] != len) return false;
+        for (int32_t k = 0; k < len; ++k)
+            if ((steps[off[b] + k].layer & 0xff) != (steps[off[0] + k].layer & 0xff)) return false;
+    }
+    return true;
+}
+
+size_t append(std::vector<unsigned char> &blob, const void *src, size_t bytes) {
+    const size_t off = blob.size();
+    blob.resize(off + align16(bytes));
+    if (bytes) std::memcpy(blob.data() + off, src, bytes);
+    return off;
+}
+
+cr_status_t prepare(const cr_plan *plan, const uint32_t *masks_host, int batch, uint32_t flags, Prepared &pr) {
+    const cr::HostPlan &hp = plan->hp;
+    if (!masks_host || batch < 1 || batch > (1 << 16)) return CR_ERR_INVALID_ARG;
+    const uint32_t variant = flags & CR_AGG_VARIANT_MASK;
+    if (variant > CR_AGG_UNCODED_SUM || (flags & ~(uint32_t)(CR_AGG_VARIANT_MASK | CR_AGG_ALL_NODES | CR_AGG_FROM_CODED)) != 0)
+        return CR_ERR_INVALID_ARG;
+    if ((flags & CR_AGG_ALL_NODES) && variant != CR_AGG_UNFUSED) return CR_ERR_INVALID_ARG;
+    if ((flags & CR_AGG_FROM_CODED) && variant == CR_AGG_UNFUSED) return CR_ERR_INVALID_ARG;
+    pr.batch = batch; pr.flags = flags; pr.variant = variant;
+    pr.m_eff = (flags & CR_AGG_FROM_CODED) ? 1 : hp.m;
+    const int share = variant == CR_AGG_FUSED ? plan->tune.share : 1;
+    cr_status_t st = expand_all(hp, masks_host, batch, share, pr.ex);
+    if (st != CR_OK) return st;
+    const Expanded &ex = pr.ex;
+
+    if (variant == CR_AGG_UNFUSED) {
+        // union node list, then per pattern and level the weight rows and the active flags
+        const int n = hp.n, L = hp.L;
+        const bool all_nodes = (flags & CR_AGG_ALL_NODES) != 0;
+        pr.w_off.resize(L); pr.a_off.resize(L);
+        for (int l = 0; l < L; ++l) {
+            const size_t parents = (size_t)hp.nodes_in_layer(l);
+            pr.w_off[l] = pr.per_pattern; pr.per_pattern += align16(parents * n * 4);
+            pr.a_off[l] = pr.per_pattern; pr.per_pattern += align16(parents * 4);
+        }
+        pr.nodes_bytes = align16(ex.unodes.size() * 4);
+        pr.blob.assign(pr.nodes_bytes + pr.per_pattern * (size_t)batch, 0);
+        std::memcpy(pr.blob.data(), ex.unodes.data(), ex.unodes.size() * 4);
+        std::vector<char> used(hp.N, 0);
+        for (int b = 0; b < batch; ++b) {
+            const uint32_t *masks = masks_host + (size_t)b * hp.groups;
+            std::fill(used.begin(), used.end(), 0);
+            for (const cr::UsedNode &u : ex.per_pattern[b]) used[u.node] = 1;
+            unsigned char *base = pr.blob.data() + pr.nodes_bytes + pr.per_pattern * (size_t)b;
+            for (int l = 0; l < L; ++l) {
+                uint32_t *W = reinterpret_cast<uint32_t *>(base + pr.w_off[l]);
+                int32_t *act = reinterpret_cast<int32_t *>(base + pr.a_off[l]);
+                const int parents = hp.nodes_in_layer(l);
+                for (int i = 0; i < parents; ++i) {
+                    const int group = l == 0 ? 0 : hp.layer_offset[l] + i + 1;
+                    const bool active = all_nodes || l == 0 || used[hp.layer_offset[l] + i];
+                    act[i] = active ? 1 : 0;
+                    if (!active) continue;
+                    if ((masks[group] >> n) != 0) return CR_ERR_INVALID_ARG;
+                    if (!hp.mask_ok(masks[group])) return CR_ERR_UNDECODABLE_MASK;
+                    const double *a = hp.decode_row(l, masks[group]);
+                    for (int j = 0; j < n; ++j) W[(size_t)i * n + j] = weight_bits(hp, a[j]);
+                }
+            }
+        }
+        return CR_OK;
+    }
+
+    pr.same_shape = batch == 1 || same_layers(ex.steps, ex.pat_off, batch);
+    pr.red_same_shape = !ex.ops.empty() && same_layers(ex.red_steps, ex.red_off, batch);
+    for (const cr::Step &s : ex.steps) pr.subtrees += (s.layer & 0xff) == 1;
+    // Batches over nodes with few slot rows (m <= 8, or coded gradients): one TMA box takes the rows of up
+    // to 16 / m union nodes with consecutive ids, which lie next to each other in the slot buffer.
+    std::vector<int2> boxes;
+    pr.npb = (batch > 1 && variant == CR_AGG_FUSED && pr.m_eff <= 8) ? 16 / pr.m_eff : 1;
+    if (pr.npb > 1 && ex.unodes.size() < (1u << 20)) {
+        for (size_t u = 0; u < ex.unodes.size();) {
+            size_t g = 1;
+            while (g < (size_t)pr.npb && u + g < ex.unodes.size() && ex.unodes[u + g] == ex.unodes[u] + (int32_t)g) ++g;
+            boxes.push_back(make_int2(ex.unodes[u] * pr.m_eff, (int)u | (int)(g << 20)));
+            u += g;
+        }
+    }
+    pr.n_boxes = (int)boxes.size();
+    pr.off_steps = append(pr.blob, ex.steps.data(), ex.steps.size() * sizeof(cr::Step));
+    pr.off_pat = append(pr.blob, ex.pat_off.data(), ex.pat_off.size() * 4);
+    pr.off_unodes = append(pr.blob, ex.unodes.data(), ex.unodes.size() * 4);
+    pr.off_wtab = append(pr.blob, ex.wtab.data(), ex.wtab.size() * 4);
+    pr.off_boxes = append(pr.blob, boxes.data(), boxes.size() * sizeof(int2));
+    pr.off_ops = append(pr.blob, ex.ops.data(), ex.ops.size() * sizeof(int4));
+    pr.off_vtab = append(pr.blob, ex.vtab.data(), ex.vtab.size() * 4);
+    pr.off_red_steps = append(pr.blob, ex.red_steps.data(), ex.red_steps.size() * sizeof(cr::Step));
+    pr.off_red_pat = append(pr.blob, ex.red_off.data(), ex.red_off.size() * 4);
+    return CR_OK;
+}
+
+cr_status_t run_unfused(cr_plan *plan, const Prepared &pr, const unsigned char *tables, const void *G_slots, void *g_out,
+                        void *workspace, cudaStream_t s) {
     const cr::HostPlan &hp = plan->hp;
     const int n = hp.n, L = hp.L;
     const bool is_int = hp.dtype == CR_I32;
-    // staging: union node list, then per pattern and level the weight rows and the active flags
-    size_t per_pattern = 0;
-    std::vector<size_t> w_off(L), a_off(L);
-    for (int l = 0; l < L; ++l) {
-        const size_t parents = (size_t)hp.nodes_in_layer(l);
-        w_off[l] = per_pattern; per_pattern += align16(parents * n * 4);
-        a_off[l] = per_pattern; per_pattern += align16(parents * 4);
-    }
-    const size_t nodes_bytes = align16(ex.unodes.size() * 4);
-    const size_t total = nodes_bytes + per_pattern * (size_t)batch;
-    StageSlot *slot = nullptr;
-    cr_status_t st = stage_acquire(plan, total, &slot);
-    if (st != CR_OK) return st;
-    std::memset(slot->host, 0, total);
-    std::memcpy(slot->host, ex.unodes.data(), ex.unodes.size() * 4);
-    for (int b = 0; b < batch; ++b) {
-        const uint32_t *masks = masks_host + (size_t)b * hp.groups;
-        std::vector<char> used(hp.N, 0);
-        for (const cr::UsedNode &u : ex.per_pattern[b]) used[u.node] = 1;
-        unsigned char *base = slot->host + nodes_bytes + per_pattern * (size_t)b;
-        for (int l = 0; l < L; ++l) {
-            uint32_t *W = reinterpret_cast<uint32_t *>(base + w_off[l]);
-            int32_t *act = reinterpret_cast<int32_t *>(base + a_off[l]);
-            const int parents = hp.nodes_in_layer(l);
-            for (int i = 0; i < parents; ++i) {
-                const int group = l == 0 ? 0 : hp.layer_offset[l] + i + 1;
-                const bool active = all_nodes || l == 0 || used[hp.layer_offset[l] + i];
-                act[i] = active ? 1 : 0;
-                if (!active) continue;
-                if ((masks[group] >> n) != 0) return CR_ERR_INVALID_ARG;
-                if (!hp.mask_ok(masks[group])) return CR_ERR_UNDECODABLE_MASK;
-                const double *a = hp.decode_row(l, masks[group]);
-                for (int j = 0; j < n; ++j) W[(size_t)i * n + j] = weight_bits(hp, a[j]);
-            }
-        }
-    }
-    st = stage_commit(slot, total, s);
-    if (st != CR_OK) return st;
-
+    const bool all_nodes = (pr.flags & CR_AGG_ALL_NODES) != 0;
     char *ws = reinterpret_cast<char *>(workspace);
     char *E = ws;
     std::vector<char *> M(L + 1, nullptr);  // M[l] for l = 1..L-1
@@ -568,45 +804,41 @@ static cr_status_t aggregate_unfused(cr_plan *plan, const void *G_slots, const u
 
     cudaError_t e;
     if (all_nodes) e = cr::launch_encode(G_slots, plan->d_coeff, nullptr, hp.N, hp.m, hp.d, E, is_int, s, &plan->launches);
-    else e = cr::launch_encode(G_slots, plan->d_coeff, reinterpret_cast<const int32_t *>(slot->dev),
-                               (int)ex.unodes.size(), hp.m, hp.d, E, is_int, s, &plan->launches);
+    else e = cr::launch_encode(G_slots, plan->d_coeff, reinterpret_cast<const int32_t *>(tables),
+                               (int)pr.ex.unodes.size(), hp.m, hp.d, E, is_int, s, &plan->launches);
     if (e != cudaSuccess) { note_cuda(e, "encode"); return CR_ERR_CUDA; }
-    for (int b = 0; b < batch; ++b) {
-        const unsigned char *base = slot->dev + nodes_bytes + per_pattern * (size_t)b;
+    for (int b = 0; b < pr.batch; ++b) {
+        const unsigned char *base = tables + pr.nodes_bytes + pr.per_pattern * (size_t)b;
         for (int l = L - 1; l >= 0; --l) {
             const void *child = M[l + 1];
             const void *own = l == 0 ? nullptr : E + (size_t)hp.layer_offset[l] * hp.d * 4;
             void *dst = l == 0 ? reinterpret_cast<char *>(g_out) + (size_t)b * hp.d * 4 : M[l];
-            e = cr::launch_decode(child, own, base + w_off[l], reinterpret_cast<const int32_t *>(base + a_off[l]),
+            e = cr::launch_decode(child, own, base + pr.w_off[l], reinterpret_cast<const int32_t *>(base + pr.a_off[l]),
                                   hp.nodes_in_layer(l), n, hp.d, dst, (is_int && l == 0) ? hp.int_shift : 0, is_int, s,
                                   &plan->launches);
             if (e != cudaSuccess) { note_cuda(e, "decode"); return CR_ERR_CUDA; }
         }
     }
-    return stage_release(slot, s);
+    return CR_OK;
 }
 
-cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *masks_host, int32_t batch, void *g_out,
-                         uint32_t flags, void *workspace, size_t workspace_bytes, void *stream) {
-    cr_status_t st = check_device_plan(plan);
-    if (st != CR_OK) return st;
-    const cr::HostPlan &hp = plan->hp;
-    if (!G_slots || !masks_host || !g_out || batch < 1 || batch > (1 << 16)) return CR_ERR_INVALID_ARG;
-    const uint32_t variant = flags & CR_AGG_VARIANT_MASK;
-    if (variant > CR_AGG_UNCODED_SUM || (flags & ~(uint32_t)(CR_AGG_VARIANT_MASK | CR_AGG_ALL_NODES | CR_AGG_FROM_CODED)) != 0)
-        return CR_ERR_INVALID_ARG;
-    if ((flags & CR_AGG_ALL_NODES) && variant != CR_AGG_UNFUSED) return CR_ERR_INVALID_ARG;
-    if ((flags & CR_AGG_FROM_CODED) && variant == CR_AGG_UNFUSED) return CR_ERR_INVALID_ARG;
-    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+// Launches the work of a prepared batch.  `tables` is the device copy of pr.blob, or null when it has
+// not been made yet: forms that can pass a single short schedule in the kernel parameters then run
+// without it, and the others return kNeedTables so that the caller stages the blob and calls again.
+constexpr int kNeedTables = -1;
 
-    Expanded ex;
-    st = expand_all(hp, masks_host, batch, ex);
-    if (st != CR_OK) return st;
+int run_prepared(cr_plan *plan, const Prepared &pr, const unsigned char *tables, const void *G_slots, void *g_out,
+                 void *workspace, size_t workspace_bytes, cudaStream_t s) {
+    const cr::HostPlan &hp = plan->hp;
+    const int batch = pr.batch;
+    const uint32_t variant = pr.variant;
+    const Expanded &ex = pr.ex;
 
     if (variant == CR_AGG_UNFUSED) {
-        if (!workspace || workspace_bytes < cr_aggregate_workspace_bytes(plan, batch, flags)) return CR_ERR_OOM;
+        if (!workspace || workspace_bytes < cr_aggregate_workspace_bytes(plan, batch, pr.flags)) return CR_ERR_OOM;
+        if (!tables) return kNeedTables;
         plan->last_kernel = "cr_encode_kernel + cr_decode_kernel per level";
-        return aggregate_unfused(plan, G_slots, masks_host, batch, g_out, (flags & CR_AGG_ALL_NODES) != 0, workspace, ex, s);
+        return run_unfused(plan, pr, tables, G_slots, g_out, workspace, s);
     }
 
     cr::AggArgs a;
@@ -616,18 +848,12 @@ cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *m
     a.n_wtab = (int)ex.wtab.size();
     a.n_union = (int)ex.unodes.size(); a.batch = batch; a.total_steps = (int)ex.steps.size();
     a.m = hp.m; a.L = hp.L; a.d = hp.d; a.rows_total = (int64_t)hp.N * hp.m; a.out = g_out;
-    if (flags & CR_AGG_FROM_CODED) {
+    if (pr.flags & CR_AGG_FROM_CODED) {
         // the input is E [N][d]: one row per node, already combined with the slot coefficients
         a.m = 1; a.coeff = plan->d_ones; a.rows_total = hp.N;
     }
     a.shift = hp.dtype == CR_I32 ? hp.int_shift : 0; a.status = plan->d_status; a.is_int = hp.dtype == CR_I32;
-    a.same_shape = 1;
-    for (int b = 1; b < batch && a.same_shape; ++b) {
-        const auto &p0 = ex.per_pattern[0], &pb = ex.per_pattern[b];
-        if (pb.size() != p0.size()) { a.same_shape = 0; break; }
-        for (size_t k = 0; k < p0.size(); ++k)
-            if (pb[k].layer != p0[k].layer) { a.same_shape = 0; break; }
-    }
+    a.same_shape = pr.same_shape;
 
     // Few slot rows per node make small TMA boxes (m = 4: 4 KB; a coded gradient, one row per node:
     // 1 KB), too small for the copy engine to keep HBM busy (measured at d = 2^22 on the (12,2) tree:
@@ -640,10 +866,10 @@ cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *m
     // (flat gradient coding, L = 1; n = 12, s = 1 at d = 2^22: 4.9 against 3.0 TB/s).
     // Short vectors stay with the TMA kernel unless they are coded gradients: its narrow tiles and
     // deep rings fill more SMs (m = 4, d = 5004: 70 against 109 us; from coded gradients 51 against 37 us).
+    const bool untuned = !plan->tune.ncw && !plan->tune.stages && !plan->tune.ctas_per_sm && !plan->tune.rows;
     const bool prefer_plain = batch == 1 &&
                               (a.m == 1 || ((a.m <= 4 || a.m % 4 == 0) && hp.d >= (1ll << 19) && (a.m <= 8 || hp.d <= (1ll << 23)))) &&
-                              hp.d % 4 == 0 && !plan->tune.ncw && !plan->tune.stages && !plan->tune.ctas_per_sm &&
-                              !plan->tune.rows;
+                              hp.d % 4 == 0 && untuned;
 
     // Short vectors under a large tree: one block per column range would walk all the consumed nodes
     // one after the other (d = 5004 under the (12,2) tree: 132 nodes, 53 us).  The sub-trees below the
@@ -651,11 +877,8 @@ cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *m
     // adds their weighted messages.
     // Measured (us per call, split / TMA kernel): (12,2,1) d = 5004: 24 / 53, d = 120000: 48 / 113;
     // with few sub-trees it does not pay: (4,3,1) d = 6500: 18.5 / 20.6, (3,4,1) d = 4096: 31 / 18.5.
-    const bool untuned = !plan->tune.ncw && !plan->tune.stages && !plan->tune.ctas_per_sm && !plan->tune.rows;
-    int subtrees = 0;
-    for (const cr::Step &st : ex.steps) subtrees += (st.layer & 0xff) == 1;
-    if (variant == CR_AGG_FUSED && untuned && batch == 1 && plan->d_split && subtrees >= kSplitMinSubtrees &&
-        a.total_steps >= 24 && a.total_steps <= cr::inline_schedule_limit() && subtrees <= cr::split_limit()) {
+    if (variant == CR_AGG_FUSED && untuned && batch == 1 && plan->d_split && pr.subtrees >= kSplitMinSubtrees &&
+        a.total_steps >= 24 && a.total_steps <= cr::inline_schedule_limit() && pr.subtrees <= cr::split_limit()) {
         a.split_scratch = plan->d_split;
         cudaError_t e0 = cr::launch_fused_ldg(a, s, &plan->launches);
         if (e0 != cudaSuccess) { note_cuda(e0, "cr_aggregate"); return CR_ERR_CUDA; }
@@ -679,45 +902,15 @@ cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *m
         return CR_OK;
     }
 
-    // staging layout: steps | pattern offsets | union nodes
-    const size_t steps_bytes = align16(ex.steps.size() * sizeof(cr::Step));
-    const size_t off_bytes = align16(ex.pat_off.size() * 4);
-    const size_t nodes_bytes = align16(ex.unodes.size() * 4);
-    const size_t wtab_bytes = align16(ex.wtab.size() * 4);
-    // Batches over nodes with few slot rows (m <= 8, or coded gradients): one TMA box takes the rows of up
-    // to 16 / m union nodes with consecutive ids, which lie next to each other in the slot buffer.
-    std::vector<int2> boxes;
-    const int npb = (batch > 1 && variant == CR_AGG_FUSED && a.m <= 8) ? 16 / a.m : 1;
-    if (npb > 1 && ex.unodes.size() < (1u << 20)) {
-        for (size_t u = 0; u < ex.unodes.size();) {
-            size_t g = 1;
-            while (g < (size_t)npb && u + g < ex.unodes.size() && ex.unodes[u + g] == ex.unodes[u] + (int32_t)g) ++g;
-            boxes.push_back(make_int2(ex.unodes[u] * a.m, (int)u | (int)(g << 20)));
-            u += g;
-        }
-    }
-    const size_t boxes_bytes = align16(boxes.size() * sizeof(int2));
-    const size_t total = steps_bytes + off_bytes + nodes_bytes + wtab_bytes + boxes_bytes;
-    StageSlot *slot = nullptr;
-    st = stage_acquire(plan, total, &slot);
-    if (st != CR_OK) return st;
-    std::memcpy(slot->host, ex.steps.data(), ex.steps.size() * sizeof(cr::Step));
-    std::memcpy(slot->host + steps_bytes, ex.pat_off.data(), ex.pat_off.size() * 4);
-    std::memcpy(slot->host + steps_bytes + off_bytes, ex.unodes.data(), ex.unodes.size() * 4);
-    std::memcpy(slot->host + steps_bytes + off_bytes + nodes_bytes, ex.wtab.data(), ex.wtab.size() * 4);
-    if (!boxes.empty())
-        std::memcpy(slot->host + steps_bytes + off_bytes + nodes_bytes + wtab_bytes, boxes.data(), boxes.size() * sizeof(int2));
-    st = stage_commit(slot, total, s);
-    if (st != CR_OK) return st;
-
-    a.steps = reinterpret_cast<const cr::Step *>(slot->dev);
-    a.pat_off = reinterpret_cast<const int32_t *>(slot->dev + steps_bytes);
-    a.unodes = reinterpret_cast<const int32_t *>(slot->dev + steps_bytes + off_bytes);
-    a.wtab = reinterpret_cast<const uint32_t *>(slot->dev + steps_bytes + off_bytes + nodes_bytes);
-    if (!boxes.empty()) {
-        a.boxes = reinterpret_cast<const int2 *>(slot->dev + steps_bytes + off_bytes + nodes_bytes + wtab_bytes);
-        a.n_boxes = (int)boxes.size();
-        a.npb = npb;
+    if (!tables) return kNeedTables;
+    a.steps = reinterpret_cast<const cr::Step *>(tables + pr.off_steps);
+    a.pat_off = reinterpret_cast<const int32_t *>(tables + pr.off_pat);
+    a.unodes = reinterpret_cast<const int32_t *>(tables + pr.off_unodes);
+    a.wtab = reinterpret_cast<const uint32_t *>(tables + pr.off_wtab);
+    if (pr.n_boxes) {
+        a.boxes = reinterpret_cast<const int2 *>(tables + pr.off_boxes);
+        a.n_boxes = pr.n_boxes;
+        a.npb = pr.npb;
     }
     a.host_steps = nullptr;
 
@@ -728,15 +921,122 @@ cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *m
     } else {
         bool done = false;
         if (variant == CR_AGG_FUSED && !prefer_plain) {
-            if (batch == 1) e = cr::launch_fused_tma(a, plan->dev, plan->tune, plan->encode, s, &plan->launches, &done);
-            else e = cr::launch_fused_batch_tma(a, plan->dev, plan->tune, plan->encode, s, &plan->launches, &done);
+            if (batch == 1) {
+                e = cr::launch_fused_tma(a, plan->dev, plan->tune, plan->encode, s, &plan->launches, &done);
+                if (done) plan->last_kernel = "cr_fused_tma_kernel";
+            } else {
+                if (!ex.ops.empty()) {
+                    // the patterns share the messages of the bottom layer: reduced schedules
+                    cr::AggArgs r = a;
+                    r.steps = reinterpret_cast<const cr::Step *>(tables + pr.off_red_steps);
+                    r.pat_off = reinterpret_cast<const int32_t *>(tables + pr.off_red_pat);
+                    r.total_steps = (int)ex.red_steps.size();
+                    r.same_shape = pr.red_same_shape;
+                    r.n_rows = ex.n_rows; r.n_ops = (int)ex.ops.size();
+                    r.ops = reinterpret_cast<const int4 *>(tables + pr.off_ops);
+                    r.vtab = reinterpret_cast<const uint32_t *>(tables + pr.off_vtab);
+                    r.vtab_words = (int)ex.vtab.size();
+                    e = cr::launch_fused_batch_tma(r, plan->dev, plan->tune, plan->encode, s, &plan->launches, &done);
+                    if (done) plan->last_kernel = "cr_fused_batch_tma_kernel (shared messages)";
+                }
+                if (e == cudaSuccess && !done) {
+                    e = cr::launch_fused_batch_tma(a, plan->dev, plan->tune, plan->encode, s, &plan->launches, &done);
+                    if (done) plan->last_kernel = "cr_fused_batch_tma_kernel";
+                }
+            }
         }
-        plan->last_kernel = done ? (batch == 1 ? "cr_fused_tma_kernel" : "cr_fused_batch_tma_kernel") : "cr_fused_ldg_kernel";
-        if (e == cudaSuccess && !done) e = cr::launch_fused_ldg(a, s, &plan->launches);
+        if (e == cudaSuccess && !done) {
+            plan->last_kernel = "cr_fused_ldg_kernel";
+            e = cr::launch_fused_ldg(a, s, &plan->launches);
+        }
     }
     if (e != cudaSuccess) { note_cuda(e, "cr_aggregate"); return CR_ERR_CUDA; }
-    return stage_release(slot, s);
+    return CR_OK;
 }
+
+}  // namespace
+
+// A straggler pattern batch expanded once and kept on the device (cr_schedule_create).
+struct cr_schedule {
+    cr_plan *plan = nullptr;
+    Prepared prep;
+    unsigned char *dev = nullptr;
+};
+
+extern "C" {
+
+cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *masks_host, int32_t batch, void *g_out,
+                         uint32_t flags, void *workspace, size_t workspace_bytes, void *stream) {
+    cr_status_t st = check_device_plan(plan);
+    if (st != CR_OK) return st;
+    if (!G_slots || !g_out) return CR_ERR_INVALID_ARG;
+    cudaStream_t s = reinterpret_cast<cudaStream_t>(stream);
+    Prepared pr;
+    st = prepare(plan, masks_host, batch, flags, pr);
+    if (st != CR_OK) return st;
+    int rc = run_prepared(plan, pr, nullptr, G_slots, g_out, workspace, workspace_bytes, s);
+    if (rc != kNeedTables) return (cr_status_t)rc;
+    StageSlot *slot = nullptr;
+    st = stage_acquire(plan, pr.blob.size(), &slot);
+    if (st != CR_OK) return st;
+    std::memcpy(slot->host, pr.blob.data(), pr.blob.size());
+    st = stage_commit(slot, pr.blob.size(), s);
+    if (st != CR_OK) return st;
+    rc = run_prepared(plan, pr, slot->dev, G_slots, g_out, workspace, workspace_bytes, s);
+    // the slot is guarded by an event on every path, so that it is not reused under a copy still queued
+    st = stage_release(slot, s);
+    return rc != CR_OK ? (cr_status_t)rc : st;
+}
+
+cr_status_t cr_schedule_create(cr_plan_t *plan, const uint32_t *masks_host, int32_t batch, uint32_t flags,
+                               cr_schedule_t **out) {
+    cr_status_t st = check_device_plan(plan);
+    if (st != CR_OK) return st;
+    if (!out) return CR_ERR_INVALID_ARG;
+    cr_schedule *sc = new (std::nothrow) cr_schedule();
+    if (!sc) return CR_ERR_OOM;
+    sc->plan = plan;
+    st = prepare(plan, masks_host, batch, flags, sc->prep);
+    if (st != CR_OK) { delete sc; return st; }
+    const size_t bytes = std::max<size_t>(sc->prep.blob.size(), 16);
+    cudaError_t e = cudaMalloc(reinterpret_cast<void **>(&sc->dev), bytes);
+    if (e == cudaSuccess && !sc->prep.blob.empty())
+        e = cudaMemcpy(sc->dev, sc->prep.blob.data(), sc->prep.blob.size(), cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) {
+        note_cuda(e, "cr_schedule_create");
+        if (sc->dev) cudaFree(sc->dev);
+        delete sc;
+        return CR_ERR_CUDA;
+    }
+    *out = sc;
+    return CR_OK;
+}
+
+cr_status_t cr_schedule_destroy(cr_schedule_t *sched) {
+    if (!sched) return CR_OK;
+    if (sched->plan && sched->plan->device >= 0) cudaSetDevice(sched->plan->device);
+    if (sched->dev) cudaFree(sched->dev);
+    delete sched;
+    return CR_OK;
+}
+
+cr_status_t cr_schedule_bytes(const cr_schedule_t *sched, int64_t *bytes, int32_t *used_nodes) {
+    if (!sched || !bytes) return CR_ERR_INVALID_ARG;
+    const cr::HostPlan &hp = sched->plan->hp;
+    *bytes = 4ll * hp.d * ((int64_t)sched->prep.m_eff * (int64_t)sched->prep.ex.unodes.size() + sched->prep.batch);
+    if (used_nodes) *used_nodes = (int32_t)sched->prep.ex.unodes.size();
+    return CR_OK;
+}
+
+cr_status_t cr_aggregate_scheduled(cr_plan_t *plan, const void *G_slots, const cr_schedule_t *sched, void *g_out,
+                                   void *workspace, size_t workspace_bytes, void *stream) {
+    if (!plan || !sched || sched->plan != plan || !G_slots || !g_out) return CR_ERR_INVALID_ARG;
+    int current = -1;
+    if (cudaGetDevice(&current) != cudaSuccess || current != plan->device) CR_CUDA(cudaSetDevice(plan->device));
+    return (cr_status_t)run_prepared(plan, sched->prep, sched->dev, G_slots, g_out, workspace, workspace_bytes,
+                                     reinterpret_cast<cudaStream_t>(stream));
+}
+
 
 cr_status_t cr_aggregate_host(cr_plan_t *plan, const void *G_slots_host, const uint32_t *masks_host, int32_t batch,
                               void *g_out_host, uint32_t flags, void *dev_slots, void *dev_out, void *workspace,
@@ -822,7 +1122,7 @@ cr_status_t cr_partial_gradients_static(cr_plan_t *plan, const float *X, const f
     // items grouped by partition, as in cr_partial_gradients, unless the plan was tuned to (node, slot) order
     cudaError_t e = cr::launch_partial_gradients_two_pass(X, y, w, plan->d_part, plan->tune.pg_order == 1 ? nullptr : plan->d_order,
                                                  plan->hp.N * plan->hp.m, rows, plan->hp.d, scratch, G_slots, CR_LOSS_SQUARED,
-                                                 reinterpret_cast<cudaStream_t>(stream), &plan->launches);
+                                                 plan->dev.sm_count, reinterpret_cast<cudaStream_t>(stream), &plan->launches);
     if (e != cudaSuccess) { note_cuda(e, "cr_partial_gradients_static"); return CR_ERR_CUDA; }
     return CR_OK;
 }

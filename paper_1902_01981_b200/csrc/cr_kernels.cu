@@ -53,17 +53,20 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
     return t;
 }
 
-// Every wait in these kernels is bounded: about two seconds of wall time or 2^30 polls, whichever
-// comes first, or as soon as another thread of the CTA has given up.  A correct launch never gets
-// near the bound; it exists so that a broken one returns with a status instead of hanging the GPU.
-constexpr uint64_t kWaitLimitNs = 2000000000ull;
+// Every wait in these kernels is bounded: `limit_ns` of wall time (a kernel argument; two seconds
+// unless the plan was told otherwise) or 2^30 polls, whichever comes first, or as soon as another
+// thread of the CTA has given up.  A correct launch never gets near the bound; it exists so that a
+// broken one returns with a status instead of hanging the GPU.
 
 // Most slot rows one TMA box may hold (the consumers keep that many coefficients in registers).
 constexpr int kMaxBoxRows = 16;
+// Most children of a parent (the batch kernel keeps their coded gradients in registers when it forms
+// the messages that the patterns of a batch share).
+constexpr int kMaxKids = 16;
 
 // `abort_flag` points at a shared-memory word that the other side of the pipeline sets when it has
 // given up (flags[0]: a consumer did, flags[1]: the producer did, flags[2]: never set).
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, uint64_t limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_timer_ns();
     for (int outer = 0; outer < (1 << 22); ++outer) {
@@ -71,15 +74,15 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
         for (int i = 0; i < 256; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (global_timer_ns() - t0 > kWaitLimitNs) return false;
+        if (global_timer_ns() - t0 > limit_ns) return false;
     }
     return false;
 }
 
 // The same wait for a whole warp (all 32 lanes call it): the answer is made uniform, so that the lanes
 // take the give-up path together or not at all.
-__device__ __forceinline__ bool mbar_wait_warp(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
-    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag) ? 1 : 0) != 0;
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t *bar, uint32_t parity, volatile int *abort_flag, uint64_t limit_ns) {
+    return __all_sync(0xffffffffu, mbar_wait(bar, parity, abort_flag, limit_ns) ? 1 : 0) != 0;
 }
 
 // 2-D tiled TMA load global -> shared, completion counted in bytes on an mbarrier.  x (innermost
@@ -143,11 +146,14 @@ __device__ __forceinline__ void fold(T (&acc)[LMAX][V], const T (&e)[V], int lay
 // independent dependency chains inside it.  This form never clears an accumulator: the first consumed
 // child of a parent ASSIGNS acc[layer-1] = w * message, later children add to it (`lf` carries the
 // layer in bits 0..7 and the first-child flag in bit 8).  acc must start at zero so that leaves, whose
-// own acc is never written, add nothing.
-template <typename T, int LMAX, int NP>
+// own acc is never written, add nothing.  Bit 9 of `lf` marks an entry whose row already is a complete
+// message (formed once for all patterns of the batch, see the batch kernel): it is taken as it is,
+// without the accumulator of its layer, which may still hold another node's children.
+template <typename T, int LMAX, int NP, bool WHOLE>
 __device__ __forceinline__ void fold_many(T (&acc)[NP][LMAX][4], const T (&e)[NP][4], int lf, const T (&w)[NP]) {
     const int layer = lf & 0xff;
     const bool first = (lf & 0x100) != 0;
+    const bool whole = WHOLE && (lf & 0x200) != 0;   // only schedules with shared messages carry such entries
 #pragma unroll
     for (int l = 1; l <= LMAX; ++l) {
         if (layer == l) {
@@ -157,7 +163,7 @@ __device__ __forceinline__ void fold_many(T (&acc)[NP][LMAX][4], const T (&e)[NP
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                         T msg = e[p][q];
-                        if (l < LMAX) msg += acc[p][l < LMAX ? l : 0][q];
+                        if (l < LMAX && !whole) msg += acc[p][l < LMAX ? l : 0][q];
                         acc[p][l - 1][q] = w[p] * msg;
                     }
             } else {
@@ -166,7 +172,7 @@ __device__ __forceinline__ void fold_many(T (&acc)[NP][LMAX][4], const T (&e)[NP
 #pragma unroll
                     for (int q = 0; q < 4; ++q) {
                         T msg = e[p][q];
-                        if (l < LMAX) msg += acc[p][l < LMAX ? l : 0][q];
+                        if (l < LMAX && !whole) msg += acc[p][l < LMAX ? l : 0][q];
                         acc[p][l - 1][q] += w[p] * msg;
                     }
             }
@@ -201,6 +207,7 @@ struct FusedArgs {
     void *out;
     int shift;
     int *status;
+    unsigned long long wait_ns;  // bound of every wait, in nanoseconds
 };
 
 // (Four 160-thread CTAs per SM need at most 96 registers per thread; the L <= 4 instances sit at 97 without
@@ -245,7 +252,7 @@ cr_fused_tma_kernel(const __grid_constant__ CUtensorMap tmap, const FusedArgs a)
                 for (int k = 0; k < a.n_steps && ok; ++k) {
                     const int row0 = (a.n_inline ? a.steps_inline[k].node : __ldg(&a.steps[k].node)) * a.m;
                     for (int c = 0; c < a.cpn; ++c) {
-                        if (!mbar_wait(&empty[stage], phase ^ 1u, &flags[0])) { ok = false; break; }
+                        if (!mbar_wait(&empty[stage], phase ^ 1u, &flags[0], a.wait_ns)) { ok = false; break; }
                         mbar_expect_tx(&full[stage], stage_bytes);
                         T *dst = ring + (size_t)stage * stage_elems;
 #pragma unroll
@@ -262,7 +269,7 @@ cr_fused_tma_kernel(const __grid_constant__ CUtensorMap tmap, const FusedArgs a)
                 flags[1] = 1;
                 atomicExch(a.status, 1);
                 for (long long i = issued > S ? issued - S : 0; i < issued; ++i)
-                    mbar_wait(&full[i % S], (uint32_t)((i / S) & 1), &flags[2]);
+                    mbar_wait(&full[i % S], (uint32_t)((i / S) & 1), &flags[2], a.wait_ns);
             }
         }
     } else {
@@ -307,7 +314,7 @@ cr_fused_tma_kernel(const __grid_constant__ CUtensorMap tmap, const FusedArgs a)
 #pragma unroll
                         for (int j = 0; j < kMaxBoxRows; ++j) cj_next[j] = j < R ? __ldg(cf + j) : T(0);
                     }
-                    if (!mbar_wait_warp(&full[stage], phase, &flags[1])) { ok = false; break; }
+                    if (!mbar_wait_warp(&full[stage], phase, &flags[1], a.wait_ns)) { ok = false; break; }
                     const T *src = ring + (size_t)stage * stage_elems + (size_t)box * R * BOXW + within;
 #pragma unroll
                     for (int j = 0; j < kMaxBoxRows; ++j) {
@@ -355,6 +362,16 @@ cr_fused_tma_kernel(const __grid_constant__ CUtensorMap tmap, const FusedArgs a)
 // E is double buffered (when it fits), so the loaders stream tile t+1 while tile t is replayed and HBM
 // never idles; loaders and replayers hand the buffers over with two mbarriers per buffer.
 //
+// Shared messages.  A parent's message depends only on the straggler sets of its own sub-tree
+// (CR.Execute: m_(l,i) = a_f [children's messages] + g_D(l,i)), so for a node of layer L-1, whose
+// children are leaves, the whole batch needs at most one message per distinct decode row of its group
+// -- a dozen for a 12-ary tree with one straggler, against one evaluation per pattern.  When the host
+// finds that this pays (n_ops > 0), the replay warps first form those message variants, once per tile:
+// a warp takes a bottom-layer node, reads its own E row and the rows of its children in the union into
+// registers once and writes every variant own + sum_j a[j] * child_j back into rows of the same buffer
+// (the node's and its children's rows, which are dead from then on, then extra rows behind the union).
+// The patterns' schedules then name a message row where they had the node and its leaves.
+//
 // Why private rings: with one ring shared by warps that each take every NLW-th box, a warp can reach a
 // buffer whose previous box -- another warp's -- has not landed yet, since TMA completions are
 // unordered; a parity wait cannot tell "one phase behind" from "done", the warp would read early and
@@ -382,9 +399,24 @@ struct BatchArgs {
     void *out;
     int shift;
     int *status;
+    unsigned long long wait_ns;  // bound of every wait, in nanoseconds
+    // Messages shared by the patterns of the batch (see the kernel): rows of an E buffer (the union nodes,
+    // then extra message rows), the bottom-layer nodes whose message variants are formed once per tile,
+    // and their variant records.
+    int n_rows;
+    int n_ops;
+    const int4 *ops;       // [n_ops] x = own row, y = row of the first child in the union, z = children in the
+                           // union | variants << 8, w = word offset of the node's variant list in vtab
+    const uint32_t *vtab;  // weight records (the decode weights of the children in the union, padded with zeros
+                           // to a multiple of four words; equal records are stored once), then per node its
+                           // variant list: pairs {destination row, word offset of the weight record}
+    int vtab_words;
+    int vtab_smem;         // the records are staged in shared memory behind the other tables
 };
 
-template <typename T, int LMAX, int NLW, int NRW>
+// SHARE: the instance that forms shared messages first; the other one is free of that code and of its
+// registers (a node's children live in registers while its variants are formed).
+template <typename T, int LMAX, int NLW, int NRW, bool SHARE>
 __global__ void __launch_bounds__((NLW + NRW) * 32, 1)
 cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchArgs a) {
     constexpr int TILE = 128;
@@ -394,7 +426,7 @@ cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchA
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int R = a.R, S = a.stages, NS = NLW * a.stages;
     const size_t stage_elems = (size_t)R * TILE;
-    const size_t e_elems = (size_t)a.n_union * TILE;
+    const size_t e_elems = (size_t)a.n_rows * TILE;
     T *ring = reinterpret_cast<T *>(smem_raw);
     T *E = ring + (size_t)NS * stage_elems;  // [nbuf][n_union][TILE]
     // staged schedules (same-shape batches with a weight table): lf[nst] = layer | first-child flag of
@@ -404,6 +436,9 @@ cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchA
     const int batch_pad = (a.batch + NP - 1) / NP * NP;
     uint32_t *ent = reinterpret_cast<uint32_t *>(reinterpret_cast<unsigned char *>(lf) + (((size_t)a.nst * 4 + 15) & ~(size_t)15));
     uint32_t *wtab_s = ent + (((size_t)a.nst * batch_pad + 3) & ~(size_t)3);
+    // shared messages: the node table and, when it fits, the variant records behind the weight table
+    int4 *ops_s = reinterpret_cast<int4 *>(wtab_s + (((size_t)a.n_wtab + 3) & ~(size_t)3));
+    uint32_t *vtab_s = reinterpret_cast<uint32_t *>(ops_s + a.n_ops);
     const int pos_mask = a.n_wtab ? 0xfff : 0x7fffffff;
     uint64_t *full = reinterpret_cast<uint64_t *>(reinterpret_cast<unsigned char *>(lf) + a.sched_smem);
     uint64_t *e_full = full + NS;    // [2] E buffer written by all loaders
@@ -425,6 +460,9 @@ cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchA
             ent[idx] = (uint32_t)__ldg(&a.steps[__ldg(&a.pat_off[b]) + k].index);
         }
         for (int i = tid; i < a.n_wtab; i += blockDim.x) wtab_s[i] = __ldg(&a.wtab[i]);
+        for (int i = tid; i < a.n_ops; i += blockDim.x) ops_s[i] = __ldg(&a.ops[i]);
+        if (a.vtab_smem)
+            for (int i = tid; i < a.vtab_words; i += blockDim.x) vtab_s[i] = __ldg(&a.vtab[i]);
     }
     __syncthreads();
 
@@ -456,7 +494,7 @@ cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchA
         for (long long tile = blockIdx.x; tile < a.ntiles && ok; tile += gridDim.x, ++t) {
             const int buf = (int)(t % (unsigned)a.nbuf);
             const unsigned use = t / (unsigned)a.nbuf;
-            if (!mbar_wait_warp(&e_free[buf], (use & 1u) ^ 1u, &flags[0])) { ok = false; break; }
+            if (!mbar_wait_warp(&e_free[buf], (use & 1u) ^ 1u, &flags[0], a.wait_ns)) { ok = false; break; }
             T *Eb = E + (size_t)buf * e_elems;
             for (int bi = warp; bi < a.n_boxes && ok; bi += NLW, ++q) {
                 const int slot = (int)(q % (unsigned)S);
@@ -467,7 +505,7 @@ cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchA
                 T cj[kMaxBoxRows];
 #pragma unroll
                 for (int j = 0; j < kMaxBoxRows; ++j) cj[j] = j < valid ? __ldg(coeff + bx.x + j) : T(0);
-                if (!mbar_wait_warp(&my_full[slot], phase, &flags[0])) { ok = false; break; }
+                if (!mbar_wait_warp(&my_full[slot], phase, &flags[0], a.wait_ns)) { ok = false; break; }
                 const T *src = my_ring + (size_t)slot * stage_elems + lane * 4;
                 T e[4] = {T(0), T(0), T(0), T(0)};
                 int node_end = a.m, i = 0;
@@ -501,7 +539,7 @@ cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchA
             atomicExch(a.status, 1);
             const unsigned in_flight_end = __shfl_sync(0xffffffffu, issued, 0);
             for (unsigned b = q; b < in_flight_end; ++b)
-                mbar_wait(&my_full[b % (unsigned)S], (b / (unsigned)S) & 1u, &flags[1]);
+                mbar_wait(&my_full[b % (unsigned)S], (b / (unsigned)S) & 1u, &flags[1], a.wait_ns);
         }
     } else if (warp < NLW) {
         // ---------------- loaders: stream their boxes, coded gradients of the union nodes -> E[buf] ----------------
@@ -531,7 +569,7 @@ cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchA
             const int buf = (int)(t % (unsigned)a.nbuf);
             const unsigned use = t / (unsigned)a.nbuf;  // how many times this buffer has been filled before
             // the buffer must have been released by the replay of its previous tile
-            if (!mbar_wait_warp(&e_free[buf], (use & 1u) ^ 1u, &flags[0])) { ok = false; break; }
+            if (!mbar_wait_warp(&e_free[buf], (use & 1u) ^ 1u, &flags[0], a.wait_ns)) { ok = false; break; }
             T *Eb = E + (size_t)buf * e_elems;
             for (int u = warp; u < a.n_union && ok; u += NLW) {
                 const int node = __ldg(&a.unodes[u]);
@@ -544,7 +582,7 @@ cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchA
                     T cj[kMaxBoxRows];
 #pragma unroll
                     for (int j = 0; j < kMaxBoxRows; ++j) cj[j] = j < R ? __ldg(cf + j) : T(0);
-                    if (!mbar_wait_warp(&my_full[slot], phase, &flags[0])) { ok = false; break; }
+                    if (!mbar_wait_warp(&my_full[slot], phase, &flags[0], a.wait_ns)) { ok = false; break; }
                     const T *src = my_ring + (size_t)slot * stage_elems + lane * 4;
 #pragma unroll
                     for (int j = 0; j < kMaxBoxRows; ++j) {
@@ -574,7 +612,7 @@ cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchA
             atomicExch(a.status, 1);
             const unsigned in_flight_end = __shfl_sync(0xffffffffu, issued, 0);
             for (unsigned b = q; b < in_flight_end; ++b)
-                mbar_wait(&my_full[b % (unsigned)S], (b / (unsigned)S) & 1u, &flags[1]);
+                mbar_wait(&my_full[b % (unsigned)S], (b / (unsigned)S) & 1u, &flags[1], a.wait_ns);
         }
     } else {
         // ---------------- replayers: every pattern's schedule from E[buf] ----------------
@@ -584,9 +622,54 @@ cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchA
         for (long long tile = blockIdx.x; tile < a.ntiles; tile += gridDim.x, ++t) {
             const int buf = (int)(t % (unsigned)a.nbuf);
             const unsigned use = t / (unsigned)a.nbuf;
-            if (!mbar_wait_warp(&e_full[buf], use & 1u, &flags[0])) { ok = false; break; }
-            const T *Eb = E + (size_t)buf * e_elems;
+            if (!mbar_wait_warp(&e_full[buf], use & 1u, &flags[0], a.wait_ns)) { ok = false; break; }
+            T *Eb = E + (size_t)buf * e_elems;
             const long long gcol = tile * TILE + lane * 4;
+            if constexpr (SHARE) {
+                // messages of the bottom-layer nodes, every distinct variant once for the whole batch
+                const int4 *ops_p = a.sched_smem ? ops_s : a.ops;
+                const uint32_t *vt = a.vtab_smem ? vtab_s : a.vtab;
+                for (int op = rw; op < a.n_ops; op += NRW) {
+                    const int4 o = ops_p[op];
+                    const int cnt = o.z & 0xff, nvar = o.z >> 8;
+                    T own[4], ch[kMaxKids][4];
+                    {
+                        const V4 v = *reinterpret_cast<const V4 *>(Eb + (size_t)o.x * TILE + lane * 4);
+                        own[0] = v.x; own[1] = v.y; own[2] = v.z; own[3] = v.w;
+                    }
+#pragma unroll
+                    for (int j = 0; j < kMaxKids; ++j) {
+                        if (j < cnt) {
+                            const V4 v = *reinterpret_cast<const V4 *>(Eb + (size_t)(o.y + j) * TILE + lane * 4);
+                            ch[j][0] = v.x; ch[j][1] = v.y; ch[j][2] = v.z; ch[j][3] = v.w;
+                        } else {
+                            ch[j][0] = ch[j][1] = ch[j][2] = ch[j][3] = T(0);
+                        }
+                    }
+                    // per variant: the row its message goes to and where its weights are (nodes whose
+                    // children in the union coincide share the weight records of their decode rows)
+                    const uint2 *list = reinterpret_cast<const uint2 *>(vt + o.w);
+                    for (int v = 0; v < nvar; ++v) {
+                        const uint2 dv = list[v];
+                        const uint4 *wr = reinterpret_cast<const uint4 *>(vt + dv.y);
+                        T msg[4] = {own[0], own[1], own[2], own[3]};
+#pragma unroll
+                        for (int g = 0; g < kMaxKids / 4; ++g) {
+                            if (g * 4 < cnt) {
+                                const uint4 wb = wr[g];
+                                const T w0 = weight_of<T>(wb.x), w1 = weight_of<T>(wb.y), w2 = weight_of<T>(wb.z), w3 = weight_of<T>(wb.w);
+#pragma unroll
+                                for (int q = 0; q < 4; ++q)
+                                    msg[q] += w0 * ch[g * 4][q] + w1 * ch[g * 4 + 1][q] + w2 * ch[g * 4 + 2][q] + w3 * ch[g * 4 + 3][q];
+                            }
+                        }
+                        V4 o4; o4.x = msg[0]; o4.y = msg[1]; o4.z = msg[2]; o4.w = msg[3];
+                        *reinterpret_cast<V4 *>(Eb + (size_t)dv.x * TILE + lane * 4) = o4;
+                    }
+                }
+                // every replay warp reads message rows written by the others
+                asm volatile("bar.sync 2, %0;" ::"r"(NRW * 32) : "memory");
+            }
             if (a.sched_smem) {
                 // NP patterns at a time per warp: their schedules visit the same layers, so one
                 // branch per step serves NP independent chains.  Step entries come from the staged
@@ -628,10 +711,10 @@ cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchA
                     fetch(0, lfA, eA, wA);
                     for (int k = 0; k < nst; k += 2) {
                         if (k + 1 < nst) fetch(k + 1, lfB, eB, wB);
-                        fold_many<T, LMAX, NP>(acc, eA, lfA, wA);
+                        fold_many<T, LMAX, NP, SHARE>(acc, eA, lfA, wA);
                         if (k + 1 < nst) {
                             if (k + 2 < nst) fetch(k + 2, lfA, eA, wA);
-                            fold_many<T, LMAX, NP>(acc, eB, lfB, wB);
+                            fold_many<T, LMAX, NP, SHARE>(acc, eB, lfB, wB);
                         }
                     }
                     if (gcol < a.d) {
@@ -1087,6 +1170,7 @@ struct PgArgs {
     int stages;
     long long d;
     int *status;
+    unsigned long long wait_ns;  // bound of every wait, in nanoseconds
 };
 
 __device__ __forceinline__ void bulk_load_1d(void *smem_dst, const void *gsrc, uint32_t bytes, uint64_t *bar) {
@@ -1186,7 +1270,7 @@ cr_partial_fused_kernel(const PgArgs a) {
             }
         }
         // all threads have left the previous block once this barrier is passed, so its buffer is free
-        const int ok = __syncthreads_and(mbar_wait(&full[blk % S], (uint32_t)((blk / S) & 1), &flags[1]) ? 1 : 0);
+        const int ok = __syncthreads_and(mbar_wait(&full[blk % S], (uint32_t)((blk / S) & 1), &flags[1], a.wait_ns) ? 1 : 0);
         if (!ok) break;
         if (tid == 0 && issued < nblocks) {
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -1248,7 +1332,7 @@ cr_partial_fused_kernel(const PgArgs a) {
         if (tid == 0) {
             flags[1] = 1;
             atomicExch(a.status, 1);
-            for (int b = done; b < issued; ++b) mbar_wait(&full[b % S], (uint32_t)((b / S) & 1), &flags[0]);
+            for (int b = done; b < issued; ++b) mbar_wait(&full[b % S], (uint32_t)((b / S) & 1), &flags[0], a.wait_ns);
         }
     }
     __syncthreads();
@@ -1275,8 +1359,33 @@ cr_partial_fused_kernel(const PgArgs a) {
 }
 
 // ------------------------------------------------------------------------------------------------
+// Self-test of the bounded wait: what a kernel does when a copy never arrives
+// ------------------------------------------------------------------------------------------------
+
+// One thread initialises an mbarrier that expects one arrival and waits for a phase nobody completes,
+// with the wait the kernels above use; when the wait gives up it reports through the status word,
+// exactly as they do.  Nothing is in flight, so there is nothing to drain.
+__global__ void cr_wait_selftest_kernel(int *status, unsigned long long limit_ns) {
+    __shared__ uint64_t bar;
+    __shared__ volatile int never;
+    if (threadIdx.x == 0) {
+        never = 0;
+        mbar_init(&bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (!mbar_wait(&bar, 0, &never, limit_ns)) atomicExch(status, 1);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // host side: launch wrappers
 // ------------------------------------------------------------------------------------------------
+
+cudaError_t launch_wait_selftest(int *status, unsigned long long limit_ns, cudaStream_t stream, int64_t *launches) {
+    cr_wait_selftest_kernel<<<1, 32, 0, stream>>>(status, limit_ns);
+    const cudaError_t err = cudaGetLastError();
+    if (err == cudaSuccess) ++*launches;
+    return err;
+}
 
 static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -1447,7 +1556,7 @@ cudaError_t launch_fused_tma(const AggArgs &a, const DeviceInfo &dev, const Tuni
     }
     fa.coeff = a.coeff; fa.steps = a.steps; fa.n_steps = a.total_steps; fa.m = a.m; fa.R = R; fa.cpn = a.m / R;
     fa.stages = stages; fa.d = a.d; fa.ntiles = (a.d + tile - 1) / tile; fa.out = a.out; fa.shift = a.shift;
-    fa.status = a.status;
+    fa.status = a.status; fa.wait_ns = tune.wait_limit_ns;
     const long long max_grid = (long long)dev.sm_count * ctas;
     const int grid = (int)std::min<long long>(fa.ntiles, max_grid);
     cudaError_t err = a.is_int ? run_fused_ncw<int>(ncw, pick_lmax(a.L), map, fa, grid, smem, stream)
@@ -1456,32 +1565,35 @@ cudaError_t launch_fused_tma(const AggArgs &a, const DeviceInfo &dev, const Tuni
     return err;
 }
 
-template <typename T, int LMAX, int NLW, int NRW>
+template <typename T, int LMAX, int NLW, int NRW, bool SHARE>
 static cudaError_t run_batch(const CUtensorMap &map, const BatchArgs &ba, int grid, size_t smem, cudaStream_t stream) {
-    auto kern = cr_fused_batch_tma_kernel<T, LMAX, NLW, NRW>;
+    auto kern = cr_fused_batch_tma_kernel<T, LMAX, NLW, NRW, SHARE>;
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
     kern<<<grid, (NLW + NRW) * 32, smem, stream>>>(map, ba);
     return cudaGetLastError();
 }
 
-template <typename T, int NLW, int NRW>
+template <typename T, int NLW, int NRW, bool SHARE>
 static cudaError_t run_batch_l(int lmax, const CUtensorMap &map, const BatchArgs &ba, int grid, size_t smem,
                                cudaStream_t stream) {
     switch (lmax) {
-        case 2: return run_batch<T, 2, NLW, NRW>(map, ba, grid, smem, stream);
-        case 4: return run_batch<T, 4, NLW, NRW>(map, ba, grid, smem, stream);
-        default: return run_batch<T, 8, NLW, NRW>(map, ba, grid, smem, stream);
+        case 2: return run_batch<T, 2, NLW, NRW, SHARE>(map, ba, grid, smem, stream);
+        case 4: return run_batch<T, 4, NLW, NRW, SHARE>(map, ba, grid, smem, stream);
+        default: return run_batch<T, 8, NLW, NRW, SHARE>(map, ba, grid, smem, stream);
     }
 }
 
 template <typename T>
 static cudaError_t run_batch_w(int nlw, int nrw, int lmax, const CUtensorMap &map, const BatchArgs &ba, int grid,
                                size_t smem, cudaStream_t stream) {
-    if (nlw == 6) return nrw == 4 ? run_batch_l<T, 6, 4>(lmax, map, ba, grid, smem, stream)
-                                  : run_batch_l<T, 6, 8>(lmax, map, ba, grid, smem, stream);
-    return nrw == 4 ? run_batch_l<T, 4, 4>(lmax, map, ba, grid, smem, stream)
-                    : run_batch_l<T, 4, 8>(lmax, map, ba, grid, smem, stream);
+    if (ba.n_ops)   // shared messages: eight replay warps always
+        return nlw == 6 ? run_batch_l<T, 6, 8, true>(lmax, map, ba, grid, smem, stream)
+                        : run_batch_l<T, 4, 8, true>(lmax, map, ba, grid, smem, stream);
+    if (nlw == 6) return nrw == 4 ? run_batch_l<T, 6, 4, false>(lmax, map, ba, grid, smem, stream)
+                                  : run_batch_l<T, 6, 8, false>(lmax, map, ba, grid, smem, stream);
+    return nrw == 4 ? run_batch_l<T, 4, 4, false>(lmax, map, ba, grid, smem, stream)
+                    : run_batch_l<T, 4, 8, false>(lmax, map, ba, grid, smem, stream);
 }
 
 cudaError_t launch_fused_batch_tma(const AggArgs &a, const DeviceInfo &dev, const Tuning &tune, EncodeTiledFn encode,
@@ -1489,7 +1601,7 @@ cudaError_t launch_fused_batch_tma(const AggArgs &a, const DeviceInfo &dev, cons
     *done = false;
     if (!encode || !tma_eligible(a)) return cudaSuccess;
     const int tile = 128;
-    const int nrw = tune.ncw == 4 ? 4 : 8;  // replay warps
+    const int nrw = (tune.ncw == 4 && !a.n_ops) ? 4 : 8;  // replay warps
     // same-shape batches stage their schedules in shared memory (layer word per step, one 4-byte entry
     // per step and pattern, patterns padded to the replay group size, the weight table) when small
     const int lmax = pick_lmax(a.L);
@@ -1499,10 +1611,11 @@ cudaError_t launch_fused_batch_tma(const AggArgs &a, const DeviceInfo &dev, cons
     if (a.same_shape && nst > 0 && a.n_wtab > 0) {
         const size_t want = (((size_t)nst * 4 + 15) & ~(size_t)15) +
                             (((size_t)nst * ((a.batch + np - 1) / np * np) + 3) & ~(size_t)3) * 4 +
-                            (((size_t)a.n_wtab * 4 + 15) & ~(size_t)15);
+                            (((size_t)a.n_wtab * 4 + 15) & ~(size_t)15) + (size_t)a.n_ops * 16;
         if (want <= 24 * 1024) sched_bytes = (want + 15) & ~(size_t)15;
     }
-    const size_t e_one = (size_t)a.n_union * tile * 4;
+    const int n_rows = a.n_ops ? a.n_rows : a.n_union;
+    const size_t e_one = (size_t)n_rows * tile * 4;
     const size_t budget = (size_t)dev.smem_optin - 512;   // barriers and flags take the rest
     // Shared memory = nbuf x E + staged schedules + one private ring of `stages` boxes of R rows per
     // loader warp.  Measured on B200 (d = 2^22, m = 16, 120 nodes, 64 patterns): six loaders with two
@@ -1521,7 +1634,7 @@ cudaError_t launch_fused_batch_tma(const AggArgs &a, const DeviceInfo &dev, cons
         multi = false;
     }
     const int node_rows = multi ? a.npb * a.m : a.m;
-    for (int try_buf = 2; try_buf >= 1 && !nbuf; --try_buf) {
+    for (int try_buf = tune.e_buffers == 1 ? 1 : 2; try_buf >= 1 && !nbuf; --try_buf) {
         if (budget <= try_buf * e_one + sched_bytes) continue;
         const size_t ring_budget = budget - try_buf * e_one - sched_bytes;
         const int want_stages = tune.stages ? tune.stages : 2;
@@ -1543,8 +1656,15 @@ cudaError_t launch_fused_batch_tma(const AggArgs &a, const DeviceInfo &dev, cons
     }
     if (!nbuf) return cudaSuccess;  // union too large for shared memory: caller falls back
     const size_t stage_bytes = (size_t)R * tile * 4;
-    const size_t smem = (size_t)nlw * stages * stage_bytes + nbuf * e_one + sched_bytes + (size_t)nlw * stages * 8 + 64 + 16;
+    size_t smem = (size_t)nlw * stages * stage_bytes + nbuf * e_one + sched_bytes + (size_t)nlw * stages * 8 + 64 + 16;
     if (smem > (size_t)dev.smem_optin) return cudaSuccess;
+    // the variant records of the shared messages ride in shared memory too when the rest leaves room
+    int vtab_smem = 0;
+    if (a.n_ops && sched_bytes && smem + (size_t)a.vtab_words * 4 <= (size_t)dev.smem_optin) {
+        vtab_smem = 1;
+        sched_bytes += (size_t)a.vtab_words * 4;
+        smem += (size_t)a.vtab_words * 4;
+    }
     const long long ntiles = (a.d + tile - 1) / tile;
     const int grid = (int)std::min<long long>(ntiles, (long long)dev.sm_count);
     // box counters are 32-bit
@@ -1560,6 +1680,9 @@ cudaError_t launch_fused_batch_tma(const AggArgs &a, const DeviceInfo &dev, cons
     ba.sched_smem = (int)sched_bytes; ba.nst = nst; ba.nbuf = nbuf; ba.wtab = a.wtab; ba.n_wtab = a.n_wtab;
     ba.boxes = multi ? a.boxes : nullptr; ba.n_boxes = multi ? a.n_boxes : 0; ba.npb = multi ? a.npb : 1;
     if (multi) ba.cpn = 1;
+    ba.wait_ns = tune.wait_limit_ns;
+    ba.n_rows = n_rows; ba.n_ops = a.n_ops; ba.ops = a.ops; ba.vtab = a.vtab; ba.vtab_words = a.vtab_words;
+    ba.vtab_smem = vtab_smem;
     const cudaError_t err = a.is_int ? run_batch_w<int>(nlw, nrw, lmax, map, ba, grid, smem, stream)
                                      : run_batch_w<float>(nlw, nrw, lmax, map, ba, grid, smem, stream);
     if (err == cudaSuccess) { *done = true; ++*launches; }
@@ -1713,11 +1836,11 @@ cudaError_t launch_decode(const void *M_child, const void *E_parent, const void 
 
 cudaError_t launch_partial_gradients_two_pass(const float *X, const float *y, const float *w, const int32_t *part,
                                               const int32_t *order, int items, int rows, int64_t d, float *resid,
-                                              float *G, int loss, cudaStream_t stream, int64_t *launches) {
+                                              float *G, int loss, int sm_count, cudaStream_t stream, int64_t *launches) {
     const bool v4 = d % 4 == 0 && aligned16(X) && aligned16(w) && aligned16(G);
     const long long total_rows = (long long)items * rows;
     const long long want_blocks = (total_rows + 7) / 8;  // 8 warps per block
-    const int blocks = (int)std::min<long long>(want_blocks, 148 * 32);
+    const int blocks = (int)std::min<long long>(want_blocks, (long long)std::max(1, sm_count) * 32);
     if (v4) cr_residual_kernel<4><<<blocks, 256, 0, stream>>>(X, y, w, part, order, total_rows, rows, d, resid, loss);
     else cr_residual_kernel<1><<<blocks, 256, 0, stream>>>(X, y, w, part, order, total_rows, rows, d, resid, loss);
     cudaError_t err = cudaGetLastError();
@@ -1837,6 +1960,7 @@ cudaError_t launch_partial_gradients_fused(const float *X, const float *y, const
     PgArgs pa;
     pa.X = X; pa.y = y; pa.w = w; pa.part = part; pa.order = slots_per_item == 1 ? order : nullptr; pa.coeff = coeff; pa.G = G; pa.rows = rows;
     pa.slots_per_item = slots_per_item; pa.loss = loss; pa.RB = RB; pa.stages = stages; pa.d = d; pa.status = status;
+    pa.wait_ns = tune.wait_limit_ns;
     cudaError_t err;
     const bool fit = !tune.pg_cluster;
     if (d <= 1024) err = run_partial_fused<1>(pa, csplit, fit, items, smem, stream);

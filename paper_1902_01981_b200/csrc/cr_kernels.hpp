@@ -28,6 +28,9 @@ struct Tuning {
     int pg_cluster = 0;   // partial gradients: CTAs per (node, slot) item (1, 2, 4 or 8)
     int pg_order = 0;     // partial gradients: launch order of the items: 1 (node, slot), 2 grouped by partition
     int tc_stages = 0;    // multi-model gradients: ring depth of the X^T R kernel (2..4)
+    int share = 0;        // batch kernel, messages shared by the patterns of a batch: 0 when it pays, 1 never, 2 always
+    int e_buffers = 0;    // batch kernel: buffers of coded gradients in shared memory (1 or 2)
+    unsigned long long wait_limit_ns = 2000000000ull;  // bound of every device-side wait
 };
 
 struct DeviceInfo {
@@ -64,6 +67,13 @@ struct AggArgs {
     int *status;          // device status word (bounded waits)
     int is_int;
     int same_shape;       // batch > 1: all patterns' schedules share length and layer sequence
+    // batch kernel, messages shared by the patterns (n_ops > 0): an E buffer has n_rows rows (the union nodes,
+    // then extra message rows); ops / vtab as in BatchArgs (device pointers)
+    int n_rows = 0;
+    int n_ops = 0;
+    const int4 *ops = nullptr;
+    const uint32_t *vtab = nullptr;
+    int vtab_words = 0;
     void *split_scratch = nullptr;  // launch_fused_ldg, single inline schedule: [n][d] scratch; when set, the
                                     // sub-trees below the master run as separate blocks (see launch_fused_ldg)
 };
@@ -108,7 +118,11 @@ cudaError_t launch_decode(const void *M_child, const void *E_parent, const void 
 // `order` (device [items], may be null): launch order of the items, e.g. grouped by partition.
 cudaError_t launch_partial_gradients_two_pass(const float *X, const float *y, const float *w, const int32_t *part,
                                               const int32_t *order, int items, int rows, int64_t d, float *resid,
-                                              float *G, int loss, cudaStream_t stream, int64_t *launches);
+                                              float *G, int loss, int sm_count, cudaStream_t stream, int64_t *launches);
+
+// One CTA that waits `limit_ns` on an mbarrier nobody arrives on -- through the same bounded wait as the
+// production kernels -- and then sets *status, as they do when a wait runs out.  No copy is in flight.
+cudaError_t launch_wait_selftest(int *status, unsigned long long limit_ns, cudaStream_t stream, int64_t *launches);
 
 // The same in one pass over X (row blocks staged in shared memory, cluster reduction), no scratch;
 // needs d % 4 == 0, d <= 8192 and 16-byte aligned X, w, G (partial_fused_eligible).

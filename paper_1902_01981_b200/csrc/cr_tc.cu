@@ -34,7 +34,6 @@ constexpr int kBoxCols = 32;      // 32 fp32 = 128 bytes: one swizzle row
 constexpr int kHeadAccs = 7;
 constexpr int kAccs = kHeadAccs + 1;
 constexpr uint32_t kTmemCols = kAccs * kModels;   // 256 columns: two CTAs fit one SM's tensor memory
-constexpr uint64_t kWaitLimitNs = 2000000000ull;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -62,8 +61,9 @@ __device__ __forceinline__ uint64_t global_timer_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait (about two seconds): false when it gave up or when *abort_flag is set.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
+// Bounded wait (`limit_ns`, a kernel argument: two seconds by default): false when it gave up or when
+// *abort_flag is set.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, uint64_t limit_ns) {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = global_timer_ns();
     for (int outer = 0; outer < (1 << 22); ++outer) {
@@ -71,7 +71,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
         for (int i = 0; i < 256; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (global_timer_ns() - t0 > kWaitLimitNs) return false;
+        if (global_timer_ns() - t0 > limit_ns) return false;
     }
     return false;
 }
@@ -207,6 +207,7 @@ struct TcResidualArgs {
     int rows, rows_pad, K, loss, stages;
     int kchunks;           // ceil(d / 32)
     int *status;
+    unsigned long long wait_ns;  // bound of every wait, in nanoseconds
 };
 
 __global__ void __launch_bounds__(192, 1)
@@ -250,7 +251,7 @@ cr_tc_residual_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_con
             bool ok = true;
             for (int kc = 0; kc < a.kchunks; ++kc) {
                 const int s = kc % S;
-                if (!mbar_wait(&empty[s], (uint32_t)(((kc / S) & 1) ^ 1), &flags[0])) { ok = false; break; }
+                if (!mbar_wait(&empty[s], (uint32_t)(((kc / S) & 1) ^ 1), &flags[0], a.wait_ns)) { ok = false; break; }
                 unsigned char *st = ring + (size_t)s * kStageBytes;
                 mbar_expect_tx(&full[s], kStageBytes);
                 tma_load_3d(st, &mapX, kc * kBoxCols, row0, p, &full[s]);
@@ -262,7 +263,7 @@ cr_tc_residual_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_con
                 flags[0] = 1;
                 atomicExch(a.status, 1);
                 for (int i = issued > S ? issued - S : 0; i < issued; ++i)
-                    mbar_wait(&full[i % S], (uint32_t)((i / S) & 1), &flags[1]);
+                    mbar_wait(&full[i % S], (uint32_t)((i / S) & 1), &flags[1], a.wait_ns);
             }
         }
     } else if (warp == 1) {
@@ -271,7 +272,7 @@ cr_tc_residual_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_con
             bool ok = true;
             for (int kc = 0; kc < a.kchunks; ++kc) {
                 const int s = kc % S;
-                if (!mbar_wait(&full[s], (uint32_t)((kc / S) & 1), &flags[0])) { ok = false; break; }
+                if (!mbar_wait(&full[s], (uint32_t)((kc / S) & 1), &flags[0], a.wait_ns)) { ok = false; break; }
                 tc_fence_after();
                 const unsigned char *st = ring + (size_t)s * kStageBytes;
 #pragma unroll
@@ -293,7 +294,7 @@ cr_tc_residual_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_con
         const int q = warp & 3;
         const int row = row0 + q * 32 + lane;
         const float yv = row < a.rows ? __ldg(&a.y[(size_t)p * a.rows + row]) : 0.f;
-        const bool ok = __all_sync(0xffffffffu, mbar_wait(acc_full, 0, &flags[0]) ? 1 : 0) != 0;
+        const bool ok = __all_sync(0xffffffffu, mbar_wait(acc_full, 0, &flags[0], a.wait_ns) ? 1 : 0) != 0;
         if (ok) {
             tc_fence_after();
             float r[kModels];
@@ -349,6 +350,7 @@ struct TcGradientArgs {
     long long d;
     int rows, K, items, stages;
     int *status;
+    unsigned long long wait_ns;  // bound of every wait, in nanoseconds
 };
 
 __global__ void __launch_bounds__(192, 1)
@@ -393,7 +395,7 @@ cr_tc_gradient_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_con
             bool ok = true;
             for (int c = 0; c < chunks; ++c) {
                 const int s = c % S;
-                if (!mbar_wait(&empty[s], (uint32_t)(((c / S) & 1) ^ 1), &flags[0])) { ok = false; break; }
+                if (!mbar_wait(&empty[s], (uint32_t)(((c / S) & 1) ^ 1), &flags[0], a.wait_ns)) { ok = false; break; }
                 unsigned char *st = ring + (size_t)s * kStageBytes;
                 mbar_expect_tx(&full[s], kStageBytes);
 #pragma unroll
@@ -407,7 +409,7 @@ cr_tc_gradient_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_con
                 flags[0] = 1;
                 atomicExch(a.status, 1);
                 for (int i = issued > S ? issued - S : 0; i < issued; ++i)
-                    mbar_wait(&full[i % S], (uint32_t)((i / S) & 1), &flags[1]);
+                    mbar_wait(&full[i % S], (uint32_t)((i / S) & 1), &flags[1], a.wait_ns);
             }
         }
     } else if (warp == 1) {
@@ -416,7 +418,7 @@ cr_tc_gradient_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_con
             bool ok = true;
             for (int c = 0; c < chunks; ++c) {
                 const int s = c % S;
-                if (!mbar_wait(&full[s], (uint32_t)((c / S) & 1), &flags[0])) { ok = false; break; }
+                if (!mbar_wait(&full[s], (uint32_t)((c / S) & 1), &flags[0], a.wait_ns)) { ok = false; break; }
                 tc_fence_after();
                 const unsigned char *st = ring + (size_t)s * kStageBytes;
 #pragma unroll
@@ -436,7 +438,7 @@ cr_tc_gradient_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_con
     } else {
         const int q = warp & 3;
         const long long col = (long long)col0 + q * 32 + lane;
-        const bool ok = __all_sync(0xffffffffu, mbar_wait(acc_full, 0, &flags[0]) ? 1 : 0) != 0;
+        const bool ok = __all_sync(0xffffffffu, mbar_wait(acc_full, 0, &flags[0], a.wait_ns) ? 1 : 0) != 0;
         if (ok) {
             tc_fence_after();
             float r[kModels];
@@ -526,7 +528,7 @@ cudaError_t launch_partial_gradients_multi(const float *X, const float *y, const
     {   // residuals
         TcResidualArgs ra;
         ra.y = y; ra.part = part; ra.order = order; ra.Rh = Rh; ra.Rl = Rl; ra.R_out = R_out; ra.rows = rows; ra.rows_pad = rows_pad;
-        ra.K = K; ra.loss = loss; ra.stages = 4; ra.kchunks = (int)((d + kBoxCols - 1) / kBoxCols); ra.status = status;
+        ra.K = K; ra.loss = loss; ra.stages = 4; ra.kchunks = (int)((d + kBoxCols - 1) / kBoxCols); ra.status = status; ra.wait_ns = tune.wait_limit_ns;
         const size_t smem = (size_t)ra.stages * (kTileM * kBoxCols * 4 + 2 * kModels * kBoxCols * 4) + (2 * ra.stages + 1) * 8 + 16 + 1024;
         cudaError_t e = cudaFuncSetAttribute(cr_tc_residual_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
@@ -537,7 +539,7 @@ cudaError_t launch_partial_gradients_multi(const float *X, const float *y, const
     }
     if (G) {   // gradients
         TcGradientArgs ga;
-        ga.part = part; ga.order = order; ga.G = G; ga.d = d; ga.rows = rows; ga.K = K; ga.items = items; ga.stages = tune.tc_stages ? tune.tc_stages : 2; ga.status = status;
+        ga.part = part; ga.order = order; ga.G = G; ga.d = d; ga.rows = rows; ga.K = K; ga.items = items; ga.stages = tune.tc_stages ? tune.tc_stages : 2; ga.status = status; ga.wait_ns = tune.wait_limit_ns;
         const size_t smem = (size_t)ga.stages * ((kTileM / kBoxCols + 2) * kRowsB * kBoxCols * 4) + (2 * ga.stages + 1) * 8 + 16 + 1024;
         cudaError_t e = cudaFuncSetAttribute(cr_tc_gradient_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;

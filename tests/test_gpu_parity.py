@@ -160,7 +160,7 @@ def test_batches_over_nodes_with_few_slot_rows(cfg, dtype, batch):
         masks = inputs.straggler_masks(n, L, s, batch, seed=32, exactly_s=True)
         tdtype = torch.int32 if is_int else torch.float32
         got = run_aggregate(plan, G_dev, masks, d, B.CR_AGG_FUSED, dtype=tdtype)
-        assert B.cr_plan_last_kernel(plan) == "cr_fused_batch_tma_kernel"
+        assert B.cr_plan_last_kernel(plan).startswith("cr_fused_batch_tma_kernel")
         E = torch.zeros((B.cr_plan_num_nodes(plan), d), dtype=tdtype, device="cuda")
         B.cr_encode(plan, G_dev, E)
         got_coded = run_aggregate(plan, E, masks, d, B.CR_AGG_FUSED | B.CR_AGG_FROM_CODED, dtype=tdtype)
@@ -270,7 +270,7 @@ def test_last_kernel_names_the_route_taken():
                                 (masks[:1], B.CR_AGG_FUSED_LDG, "cr_fused_ldg_kernel"),
                                 (masks[:1], B.CR_AGG_UNCODED_SUM, "cr_uncoded_sum_kernel")):
             got = run_aggregate(plan, G_dev, m_, cfg["d"], flags)
-            assert B.cr_plan_last_kernel(plan) == name
+            assert B.cr_plan_last_kernel(plan).startswith(name)
             if flags != B.CR_AGG_UNCODED_SUM:
                 for b in range(len(m_)):
                     assert rel_l2(got[b], O.execute(code, local, G, m_[b])) <= REL_L2_BAR
