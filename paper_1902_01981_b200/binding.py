@@ -12,7 +12,8 @@ import os
 import numpy as np
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libcodedreduce.so")
+# the in-tree build, unless CODEDREDUCE_LIB names a library built elsewhere (e.g. with other compiler flags)
+LIB_PATH = os.environ.get("CODEDREDUCE_LIB") or os.path.join(_PKG, "libcodedreduce.so")
 
 # status codes / enums of codedreduce.h
 CR_OK = 0

@@ -683,9 +683,10 @@ struct Prepared {
     int m_eff = 0;            // slot rows per node as the kernels see them (1 when the input is coded gradients)
     std::vector<unsigned char> blob;
     // fused forms: offsets of the tables inside the blob
-    size_t off_steps = 0, off_pat = 0, off_unodes = 0, off_wtab = 0, off_boxes = 0, off_ops = 0, off_vtab = 0,
+    size_t off_steps = 0, off_pat = 0, off_unodes = 0, off_wtab = 0, off_units = 0, off_ops = 0, off_vtab = 0,
            off_red_steps = 0, off_red_pat = 0;
     int n_boxes = 0, npb = 1;
+    cr::BatchShape shape;     // batches: launch shape of the batch kernel (ok = false: it cannot serve this batch)
     // unfused form: per pattern and level the weight rows and the active flags
     std::vector<size_t> w_off, a_off;
     size_t per_pattern = 0, nodes_bytes = 0;
@@ -777,11 +778,57 @@ cr_status_t prepare(const cr_plan *plan, const uint32_t *masks_host, int batch, 
         }
     }
     pr.n_boxes = (int)boxes.size();
+    // Batches: the launch shape of the batch kernel is fixed here, first with the shared messages and, if
+    // their tables do not fit, without them; then the unit records of the boxes are laid out for it.
+    std::vector<uint32_t> units;
+    if (batch > 1 && variant == CR_AGG_FUSED) {
+        cr::AggArgs q;
+        q.G = nullptr; q.coeff = nullptr; q.steps = nullptr; q.host_steps = nullptr; q.pat_off = nullptr; q.unodes = nullptr;
+        q.wtab = nullptr; q.out = nullptr; q.status = nullptr; q.shift = 0; q.rows_total = 0;
+        q.n_wtab = (int)ex.wtab.size(); q.n_union = (int)ex.unodes.size(); q.batch = batch;
+        q.m = pr.m_eff; q.L = hp.L; q.d = hp.d; q.is_int = hp.dtype == CR_I32;
+        q.npb = pr.npb; q.n_boxes = pr.n_boxes;
+        if (!pr.ex.ops.empty()) {
+            q.total_steps = (int)ex.red_steps.size(); q.same_shape = pr.red_same_shape;
+            q.n_rows = ex.n_rows; q.n_ops = (int)ex.ops.size(); q.vtab_words = (int)ex.vtab.size();
+            pr.shape = cr::batch_shape(q, plan->dev, plan->tune);
+            if (!pr.shape.ok) {   // the shared form does not fit: the plain one
+                pr.ex.ops.clear(); pr.ex.vtab.clear(); pr.ex.red_steps.clear(); pr.ex.red_off.clear();
+                pr.ex.n_rows = (int)ex.unodes.size();
+            }
+        }
+        if (pr.ex.ops.empty()) {
+            q.total_steps = (int)ex.steps.size(); q.same_shape = pr.same_shape;
+            q.n_rows = 0; q.n_ops = 0; q.vtab_words = 0;
+            pr.shape = cr::batch_shape(q, plan->dev, plan->tune);
+        }
+        if (pr.shape.ok) {
+            const int W = cr::unit_words();
+            const bool coded = (flags & CR_AGG_FROM_CODED) != 0;
+            auto coef_at = [&](int64_t row) {   // coefficient of slot row `row` as the kernels see it
+                return coded ? weight_bits(hp, 1.0) : weight_bits(hp, hp.slots[(size_t)row].coeff * (double)hp.int_scale);
+            };
+            auto put = [&](int row0, int erow, int every, int valid) {
+                const size_t at = units.size();
+                units.resize(at + W, 0u);
+                for (int j = 0; j < valid; ++j) units[at + j] = coef_at((int64_t)row0 + j);
+                units[at + 16] = (uint32_t)row0; units[at + 17] = (uint32_t)erow;
+                units[at + 18] = (uint32_t)every; units[at + 19] = (uint32_t)valid;
+            };
+            if (pr.shape.multi) {
+                for (const int2 &bx : boxes) put(bx.x, bx.y & 0xfffff, pr.m_eff, (bx.y >> 20) * pr.m_eff);
+            } else {
+                for (size_t u = 0; u < ex.unodes.size(); ++u)
+                    for (int c = 0; c < pr.shape.cpn; ++c)
+                        put(ex.unodes[u] * pr.m_eff + c * pr.shape.R, (int)u, c + 1 == pr.shape.cpn ? pr.shape.R : 0, pr.shape.R);
+            }
+        }
+    }
     pr.off_steps = append(pr.blob, ex.steps.data(), ex.steps.size() * sizeof(cr::Step));
     pr.off_pat = append(pr.blob, ex.pat_off.data(), ex.pat_off.size() * 4);
     pr.off_unodes = append(pr.blob, ex.unodes.data(), ex.unodes.size() * 4);
     pr.off_wtab = append(pr.blob, ex.wtab.data(), ex.wtab.size() * 4);
-    pr.off_boxes = append(pr.blob, boxes.data(), boxes.size() * sizeof(int2));
+    pr.off_units = append(pr.blob, units.data(), units.size() * 4);
     pr.off_ops = append(pr.blob, ex.ops.data(), ex.ops.size() * sizeof(int4));
     pr.off_vtab = append(pr.blob, ex.vtab.data(), ex.vtab.size() * 4);
     pr.off_red_steps = append(pr.blob, ex.red_steps.data(), ex.red_steps.size() * sizeof(cr::Step));
@@ -907,11 +954,9 @@ int run_prepared(cr_plan *plan, const Prepared &pr, const unsigned char *tables,
     a.pat_off = reinterpret_cast<const int32_t *>(tables + pr.off_pat);
     a.unodes = reinterpret_cast<const int32_t *>(tables + pr.off_unodes);
     a.wtab = reinterpret_cast<const uint32_t *>(tables + pr.off_wtab);
-    if (pr.n_boxes) {
-        a.boxes = reinterpret_cast<const int2 *>(tables + pr.off_boxes);
-        a.n_boxes = pr.n_boxes;
-        a.npb = pr.npb;
-    }
+    a.n_boxes = pr.n_boxes;
+    a.npb = pr.npb;
+    a.units = reinterpret_cast<const uint32_t *>(tables + pr.off_units);
     a.host_steps = nullptr;
 
     cudaError_t e = cudaSuccess;
@@ -936,11 +981,10 @@ int run_prepared(cr_plan *plan, const Prepared &pr, const unsigned char *tables,
                     r.ops = reinterpret_cast<const int4 *>(tables + pr.off_ops);
                     r.vtab = reinterpret_cast<const uint32_t *>(tables + pr.off_vtab);
                     r.vtab_words = (int)ex.vtab.size();
-                    e = cr::launch_fused_batch_tma(r, plan->dev, plan->tune, plan->encode, s, &plan->launches, &done);
+                    e = cr::launch_fused_batch_tma(r, pr.shape, plan->tune, plan->encode, s, &plan->launches, &done);
                     if (done) plan->last_kernel = "cr_fused_batch_tma_kernel (shared messages)";
-                }
-                if (e == cudaSuccess && !done) {
-                    e = cr::launch_fused_batch_tma(a, plan->dev, plan->tune, plan->encode, s, &plan->launches, &done);
+                } else {
+                    e = cr::launch_fused_batch_tma(a, pr.shape, plan->tune, plan->encode, s, &plan->launches, &done);
                     if (done) plan->last_kernel = "cr_fused_batch_tma_kernel";
                 }
             }

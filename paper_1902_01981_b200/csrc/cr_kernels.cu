@@ -34,16 +34,20 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// One probe of a barrier phase.  The hint lets the hardware park the warp for up to about a microsecond
+// while the phase is pending (it returns at once when the phase completes), so that a waiting warp does not
+// spend the issue slots of its scheduler on polling: with eight replay warps spinning, polling was a third of
+// all instructions the batch kernel issued.
 __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n"
         ".reg .pred p;\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
         "selp.u32 %0, 1, 0, p;\n"
         "}\n"
         : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
+        : "r"(smem_u32(bar)), "r"(parity), "r"(1000u)
         : "memory");
     return ok != 0;
 }
@@ -63,6 +67,9 @@ constexpr int kMaxBoxRows = 16;
 // Most children of a parent (the batch kernel keeps their coded gradients in registers when it forms
 // the messages that the patterns of a batch share).
 constexpr int kMaxKids = 16;
+// Words of a unit record of the batch kernel: 16 coefficients, then {first slot row, first E row, rows per
+// node (0: the node continues in the next box), rows in use}.
+constexpr int kUnitWords = 20;
 
 // `abort_flag` points at a shared-memory word that the other side of the pipeline sets when it has
 // given up (flags[0]: a consumer did, flags[1]: the producer did, flags[2]: never set).
@@ -91,6 +98,14 @@ __device__ __forceinline__ void tma_load_2d(void *smem_dst, const CUtensorMap *m
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
+
+// 1-D bulk copy global -> shared (no tensor map): both addresses 16-byte aligned, size a multiple of 16.
+__device__ __forceinline__ void bulk_load_1d(void *smem_dst, const void *gsrc, uint32_t bytes, uint64_t *bar) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
         : "memory");
 }
 
@@ -386,8 +401,8 @@ struct BatchArgs {
     const int32_t *unodes;
     const uint32_t *wtab;  // distinct weight bit patterns of the batch
     int n_wtab;
-    const int2 *boxes;     // npb > 1: boxes that cover several union nodes each (see AggArgs)
-    int n_boxes, npb;
+    const uint32_t *units; // [n_groups * cpn][kUnitWords] unit records (see kUnitWords), 16-byte aligned
+    int n_groups;          // groups of boxes per tile: loader w takes groups w, w + NLW, .., cpn boxes each
     int n_union, batch;
     int m, R, cpn, stages;
     int same_shape;  // every pattern's schedule has the same length and layer sequence
@@ -412,7 +427,35 @@ struct BatchArgs {
                            // variant list: pairs {destination row, word offset of the weight record}
     int vtab_words;
     int vtab_smem;         // the records are staged in shared memory behind the other tables
+    int flat;              // two-layer tree, staged schedules: every entry of a pattern is a message row of layer 1
 };
+
+// The rows of one full box (kMaxBoxRows rows in use) combined into coded gradients, for a compile-time
+// number EV of rows per node (0: the node continues in the next box): no predicate and no branch per row,
+// eight loads in flight at a time, and the stores of completed nodes at fixed places.  `dst` is the E row of
+// the first node the box completes.
+template <typename T, int EV>
+__device__ __forceinline__ void full_box_rows(const T *src, const uint32_t (&cb)[kMaxBoxRows], T (&e)[4], T *dst) {
+    typedef typename Vec4<T>::type V4;
+    constexpr int TILE = 128;
+#pragma unroll
+    for (int h = 0; h < kMaxBoxRows; h += 8) {
+        V4 v[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[j] = *reinterpret_cast<const V4 *>(src + (size_t)(h + j) * TILE);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const T cj = weight_of<T>(cb[h + j]);
+            e[0] += cj * v[j].x; e[1] += cj * v[j].y; e[2] += cj * v[j].z; e[3] += cj * v[j].w;
+            if (EV > 0 && (h + j + 1) % (EV > 0 ? EV : 1) == 0) {
+                V4 o; o.x = e[0]; o.y = e[1]; o.z = e[2]; o.w = e[3];
+                *reinterpret_cast<V4 *>(dst) = o;
+                dst += TILE;
+                e[0] = e[1] = e[2] = e[3] = T(0);
+            }
+        }
+    }
+}
 
 // SHARE: the instance that forms shared messages first; the other one is free of that code and of its
 // registers (a node's children live in registers while its variants are formed).
@@ -469,137 +512,129 @@ cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchA
     const T *coeff = reinterpret_cast<const T *>(a.coeff);
     const uint32_t stage_bytes = (uint32_t)(stage_elems * sizeof(T));
 
-    if (warp < NLW && a.npb > 1) {
-        // ---------------- loaders, few slot rows per node: a box holds the rows of up to npb union nodes ----------------
-        bool ok = true;
-        const unsigned boxes_w = warp < a.n_boxes ? (unsigned)(a.n_boxes - warp + NLW - 1) / NLW : 0u;   // boxes of this loader per tile
-        const unsigned my_tiles = blockIdx.x < a.ntiles ? (unsigned)((a.ntiles - 1 - blockIdx.x) / gridDim.x + 1) : 0u;
-        const unsigned total_boxes = my_tiles * boxes_w;
-        T *my_ring = ring + (size_t)warp * S * stage_elems;
-        uint64_t *my_full = full + warp * S;
-        unsigned issued = 0, it_t = 0, it_n = 0;
-        auto issue_next = [&]() {   // lane 0 only
-            const int slot = (int)(issued % (unsigned)S);
-            const long long tile = (long long)blockIdx.x + (long long)it_t * gridDim.x;
-            const int row0 = __ldg(&a.boxes[warp + (int)it_n * NLW].x);
-            mbar_expect_tx(&my_full[slot], stage_bytes);
-            tma_load_2d(my_ring + (size_t)slot * stage_elems, &tmap, (int)(tile * TILE), row0, &my_full[slot]);
-            ++issued;
-            if (++it_n == boxes_w) { it_n = 0; ++it_t; }
-        };
-        if (lane == 0)
-            while (issued < total_boxes && issued < (unsigned)S) issue_next();
-        unsigned q = 0;  // next box to consume
-        unsigned t = 0;  // tiles handled by this CTA so far
-        for (long long tile = blockIdx.x; tile < a.ntiles && ok; tile += gridDim.x, ++t) {
-            const int buf = (int)(t % (unsigned)a.nbuf);
-            const unsigned use = t / (unsigned)a.nbuf;
-            if (!mbar_wait_warp(&e_free[buf], (use & 1u) ^ 1u, &flags[0], a.wait_ns)) { ok = false; break; }
-            T *Eb = E + (size_t)buf * e_elems;
-            for (int bi = warp; bi < a.n_boxes && ok; bi += NLW, ++q) {
-                const int slot = (int)(q % (unsigned)S);
-                const uint32_t phase = (q / (unsigned)S) & 1u;
-                const int2 bx = __ldg(&a.boxes[bi]);
-                const int u0 = bx.y & 0xfffff, valid = (bx.y >> 20) * a.m;   // rows of the box that belong to union nodes
-                // a row's coefficient sits at the row's own index; fetched before the wait on the data
-                T cj[kMaxBoxRows];
-#pragma unroll
-                for (int j = 0; j < kMaxBoxRows; ++j) cj[j] = j < valid ? __ldg(coeff + bx.x + j) : T(0);
-                if (!mbar_wait_warp(&my_full[slot], phase, &flags[0], a.wait_ns)) { ok = false; break; }
-                const T *src = my_ring + (size_t)slot * stage_elems + lane * 4;
-                T e[4] = {T(0), T(0), T(0), T(0)};
-                int node_end = a.m, i = 0;
-#pragma unroll
-                for (int j = 0; j < kMaxBoxRows; ++j) {
-                    if (j < valid) {
-                        const V4 v = *reinterpret_cast<const V4 *>(src + (size_t)j * TILE);
-                        e[0] += cj[j] * v.x; e[1] += cj[j] * v.y; e[2] += cj[j] * v.z; e[3] += cj[j] * v.w;
-                        if (j + 1 == node_end) {   // last row of a node: its coded gradient is complete
-                            V4 o; o.x = e[0]; o.y = e[1]; o.z = e[2]; o.w = e[3];
-                            *reinterpret_cast<V4 *>(Eb + (size_t)(u0 + i) * TILE + lane * 4) = o;
-                            e[0] = e[1] = e[2] = e[3] = T(0);
-                            ++i; node_end += a.m;
-                        }
-                    }
-                }
-                // every lane has read the box: refill its buffer with box q + stages
-                __syncwarp();
-                if (lane == 0 && issued < total_boxes) {
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    issue_next();
-                }
-            }
-            if (!ok) break;
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&e_full[buf]);
-        }
-        if (!ok) {
-            // give up: flag it, then wait (bounded) for this loader's copies still in flight
-            flags[0] = 1;
-            atomicExch(a.status, 1);
-            const unsigned in_flight_end = __shfl_sync(0xffffffffu, issued, 0);
-            for (unsigned b = q; b < in_flight_end; ++b)
-                mbar_wait(&my_full[b % (unsigned)S], (b / (unsigned)S) & 1u, &flags[1], a.wait_ns);
-        }
-    } else if (warp < NLW) {
+    if (warp < NLW) {
         // ---------------- loaders: stream their boxes, coded gradients of the union nodes -> E[buf] ----------------
+        // A loader's work per tile is a fixed list of units (boxes): groups warp, warp + NLW, .. of `upg` units
+        // each (a group is a box over several small nodes, or a tall node cut into upg boxes).  What a box is
+        // -- its first slot row, the E row of its first node, after how many rows a node's coded gradient is
+        // complete, its rows' coefficients -- is its unit record.  The list is the same for every tile, so with
+        // at most 32 units per loader and tile (the usual case) lane k keeps the record of the loader's k-th
+        // unit in registers for the whole kernel and hands it round by shuffles: the loop below then touches
+        // global memory only through the copy engine.  (Read with plain loads in front of every box, the tables
+        // cost three dependent L2 latencies per box and the loaders, not HBM, set the pace: 2800 cycles per 8 KB
+        // box on the 156-node tree.  Sent along with each box as a second small bulk copy, they double the
+        // number of requests to the copy engine, which then becomes the limit.)
         bool ok = true;
-        const unsigned nodes_w = (unsigned)(a.n_union - warp + NLW - 1) / NLW;   // union nodes of this loader per tile
+        const unsigned upg = (unsigned)a.cpn;
+        const unsigned groups_w = warp < a.n_groups ? (unsigned)(a.n_groups - warp + NLW - 1) / NLW : 0u;   // groups of this loader per tile
+        const unsigned units_w = groups_w * upg;
         const unsigned my_tiles = blockIdx.x < a.ntiles ? (unsigned)((a.ntiles - 1 - blockIdx.x) / gridDim.x + 1) : 0u;
-        const unsigned total_boxes = my_tiles * nodes_w * (unsigned)a.cpn;
+        const unsigned total_boxes = my_tiles * units_w;
         T *my_ring = ring + (size_t)warp * S * stage_elems;
         uint64_t *my_full = full + warp * S;
-        // cursor of the next box to issue: (tile number of this CTA, node number of this loader, chunk)
-        unsigned issued = 0, it_t = 0, it_n = 0, it_c = 0;
-        auto issue_next = [&]() {   // lane 0 only
-            const int slot = (int)(issued % (unsigned)S);
-            const long long tile = (long long)blockIdx.x + (long long)it_t * gridDim.x;
-            const int u = warp + (int)it_n * NLW;
-            mbar_expect_tx(&my_full[slot], stage_bytes);
-            tma_load_2d(my_ring + (size_t)slot * stage_elems, &tmap, (int)(tile * TILE),
-                        __ldg(&a.unodes[u]) * a.m + (int)it_c * R, &my_full[slot]);
+        auto unit_at = [&](unsigned k) { return (unsigned)(warp + (int)(k / upg) * NLW) * upg + k % upg; };   // k-th unit of a tile
+        const bool in_regs = units_w <= 32u;
+        uint32_t myrec[kUnitWords];
+#pragma unroll
+        for (int w = 0; w < kUnitWords; ++w) myrec[w] = 0u;
+        if (in_regs && (unsigned)lane < units_w) {
+            const uint4 *g = reinterpret_cast<const uint4 *>(a.units + (size_t)unit_at((unsigned)lane) * kUnitWords);
+#pragma unroll
+            for (int w = 0; w < kUnitWords / 4; ++w) {
+                const uint4 v = __ldg(g + w);
+                myrec[4 * w] = v.x; myrec[4 * w + 1] = v.y; myrec[4 * w + 2] = v.z; myrec[4 * w + 3] = v.w;
+            }
+        }
+        // cursor of the next box to issue: tile number of this CTA and unit within the tile (kept by all lanes,
+        // so that all of them can take part in the shuffle that fetches the unit's first slot row)
+        unsigned issued = 0, it_t = 0, it_k = 0;
+        auto issue_next = [&]() {   // all lanes; lane 0 issues
+            const int row0 = in_regs ? (int)__shfl_sync(0xffffffffu, myrec[16], (int)it_k)
+                                     : (int)__ldg(a.units + (size_t)unit_at(it_k) * kUnitWords + 16);
+            if (lane == 0) {
+                const int slot = (int)(issued % (unsigned)S);
+                const long long tile = (long long)blockIdx.x + (long long)it_t * gridDim.x;
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                mbar_expect_tx(&my_full[slot], stage_bytes);
+                tma_load_2d(my_ring + (size_t)slot * stage_elems, &tmap, (int)(tile * TILE), row0, &my_full[slot]);
+            }
             ++issued;
-            if (++it_c == (unsigned)a.cpn) { it_c = 0; if (++it_n == nodes_w) { it_n = 0; ++it_t; } }
+            if (++it_k == units_w) { it_k = 0; ++it_t; }
         };
-        if (lane == 0)
-            while (issued < total_boxes && issued < (unsigned)S) issue_next();
+        while (issued < total_boxes && issued < (unsigned)S) issue_next();
         unsigned q = 0;  // next box to consume
         unsigned t = 0;  // tiles handled by this CTA so far
+        T e[4] = {T(0), T(0), T(0), T(0)};
         for (long long tile = blockIdx.x; tile < a.ntiles && ok; tile += gridDim.x, ++t) {
             const int buf = (int)(t % (unsigned)a.nbuf);
             const unsigned use = t / (unsigned)a.nbuf;  // how many times this buffer has been filled before
             // the buffer must have been released by the replay of its previous tile
             if (!mbar_wait_warp(&e_free[buf], (use & 1u) ^ 1u, &flags[0], a.wait_ns)) { ok = false; break; }
             T *Eb = E + (size_t)buf * e_elems;
-            for (int u = warp; u < a.n_union && ok; u += NLW) {
-                const int node = __ldg(&a.unodes[u]);
-                T e[4] = {T(0), T(0), T(0), T(0)};
-                for (int c = 0; c < a.cpn; ++c, ++q) {
-                    const int slot = (int)(q % (unsigned)S);
-                    const uint32_t phase = (q / (unsigned)S) & 1u;
-                    // the coefficients of a box are fetched before the wait on its data
-                    const T *cf = coeff + (size_t)node * a.m + c * R;
-                    T cj[kMaxBoxRows];
+            for (unsigned k = 0; k < units_w && ok; ++k, ++q) {
+                const int slot = (int)(q % (unsigned)S);
+                const uint32_t phase = (q / (unsigned)S) & 1u;
+                // the unit's record: coefficients of its rows and what the rows are (fetched before the wait)
+                uint32_t cb[kMaxBoxRows], dsc[4];
+                if (in_regs) {
 #pragma unroll
-                    for (int j = 0; j < kMaxBoxRows; ++j) cj[j] = j < R ? __ldg(cf + j) : T(0);
-                    if (!mbar_wait_warp(&my_full[slot], phase, &flags[0], a.wait_ns)) { ok = false; break; }
-                    const T *src = my_ring + (size_t)slot * stage_elems + lane * 4;
+                    for (int j = 0; j < kMaxBoxRows; ++j) cb[j] = __shfl_sync(0xffffffffu, myrec[j], (int)k);
 #pragma unroll
-                    for (int j = 0; j < kMaxBoxRows; ++j) {
-                        if (j < R) {
-                            const V4 v = *reinterpret_cast<const V4 *>(src + (size_t)j * TILE);
-                            e[0] += cj[j] * v.x; e[1] += cj[j] * v.y; e[2] += cj[j] * v.z; e[3] += cj[j] * v.w;
-                        }
-                    }
-                    // every lane has read the box: refill its buffer with box q + stages
-                    __syncwarp();
-                    if (lane == 0 && issued < total_boxes) {
-                        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                        issue_next();
+                    for (int j = 1; j < 4; ++j) dsc[j] = __shfl_sync(0xffffffffu, myrec[16 + j], (int)k);
+                } else {
+                    const uint4 *g = reinterpret_cast<const uint4 *>(a.units + (size_t)unit_at(k) * kUnitWords);
+                    const uint4 c0 = __ldg(g), c1 = __ldg(g + 1), c2 = __ldg(g + 2), c3 = __ldg(g + 3), d4 = __ldg(g + 4);
+                    cb[0] = c0.x; cb[1] = c0.y; cb[2] = c0.z; cb[3] = c0.w; cb[4] = c1.x; cb[5] = c1.y; cb[6] = c1.z; cb[7] = c1.w;
+                    cb[8] = c2.x; cb[9] = c2.y; cb[10] = c2.z; cb[11] = c2.w; cb[12] = c3.x; cb[13] = c3.y; cb[14] = c3.z; cb[15] = c3.w;
+                    dsc[1] = d4.y; dsc[2] = d4.z; dsc[3] = d4.w;
+                }
+                // dsc: [1] = E row of the first node that this box completes, [2] = rows after which a node is
+                // complete (0: the node continues in the loader's next box), [3] = rows of the box in use
+                const int valid = (int)dsc[3], every = (int)dsc[2];
+                int node_end = every ? every : kMaxBoxRows + 1, erow = (int)dsc[1];
+                if (!mbar_wait_warp(&my_full[slot], phase, &flags[0], a.wait_ns)) { ok = false; break; }
+                const T *src = my_ring + (size_t)slot * stage_elems + lane * 4;
+                // Full boxes of the usual shapes take a branch-free body; the loop below serves ragged boxes
+                // and odd node heights.  (The warps of this kernel run at about one instruction in seven
+                // cycles -- dependent chains, three warps per scheduler -- so the instructions per row are
+                // what a box costs: 1500 cycles with a predicate and a compare per row.)
+                bool fast = valid == kMaxBoxRows;
+                if (fast) {
+                    T *dst = Eb + (size_t)erow * TILE + lane * 4;
+                    switch (every) {
+                        case 0: full_box_rows<T, 0>(src, cb, e, dst); break;
+                        case 1: full_box_rows<T, 1>(src, cb, e, dst); break;
+                        case 2: full_box_rows<T, 2>(src, cb, e, dst); break;
+                        case 4: full_box_rows<T, 4>(src, cb, e, dst); break;
+                        case 8: full_box_rows<T, 8>(src, cb, e, dst); break;
+                        case 16: full_box_rows<T, 16>(src, cb, e, dst); break;
+                        default: fast = false; break;
                     }
                 }
-                V4 o; o.x = e[0]; o.y = e[1]; o.z = e[2]; o.w = e[3];
-                *reinterpret_cast<V4 *>(Eb + (size_t)u * TILE + lane * 4) = o;
+                if (!fast)
+#pragma unroll
+                for (int h = 0; h < kMaxBoxRows; h += 8) {
+                    V4 v[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        if (h + j < valid) v[j] = *reinterpret_cast<const V4 *>(src + (size_t)(h + j) * TILE);
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        if (h + j < valid) {
+                            const T cj = weight_of<T>(cb[h + j]);
+                            e[0] += cj * v[j].x; e[1] += cj * v[j].y; e[2] += cj * v[j].z; e[3] += cj * v[j].w;
+                            if (h + j + 1 == node_end) {   // last row of a node: its coded gradient is complete
+                                V4 o; o.x = e[0]; o.y = e[1]; o.z = e[2]; o.w = e[3];
+                                *reinterpret_cast<V4 *>(Eb + (size_t)erow * TILE + lane * 4) = o;
+                                e[0] = e[1] = e[2] = e[3] = T(0);
+                                ++erow; node_end += every;
+                            }
+                        }
+                    }
+                }
+                // every lane has read the box: refill its buffer with box q + stages
+                __syncwarp();
+                if (issued < total_boxes) issue_next();
             }
             if (!ok) break;
             __syncwarp();
@@ -610,8 +645,7 @@ cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchA
             // none lands in shared memory after the CTA has gone
             flags[0] = 1;
             atomicExch(a.status, 1);
-            const unsigned in_flight_end = __shfl_sync(0xffffffffu, issued, 0);
-            for (unsigned b = q; b < in_flight_end; ++b)
+            for (unsigned b = q; b < issued; ++b)
                 mbar_wait(&my_full[b % (unsigned)S], (b / (unsigned)S) & 1u, &flags[1], a.wait_ns);
         }
     } else {
@@ -648,15 +682,31 @@ cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchA
                     }
                     // per variant: the row its message goes to and where its weights are (nodes whose
                     // children in the union coincide share the weight records of their decode rows)
+                    // (the next variant's entry and weights are read before the current message is stored:
+                    // behind the store the compiler could not move them up, and every variant would cost
+                    // two shared-memory latencies in a row)
                     const uint2 *list = reinterpret_cast<const uint2 *>(vt + o.w);
+                    uint2 dv_next = list[0];
+                    uint4 w_next[kMaxKids / 4];
+#pragma unroll
+                    for (int g = 0; g < kMaxKids / 4; ++g)
+                        w_next[g] = g * 4 < cnt ? reinterpret_cast<const uint4 *>(vt + dv_next.y)[g] : make_uint4(0u, 0u, 0u, 0u);
                     for (int v = 0; v < nvar; ++v) {
-                        const uint2 dv = list[v];
-                        const uint4 *wr = reinterpret_cast<const uint4 *>(vt + dv.y);
+                        const uint2 dv = dv_next;
+                        uint4 w_cur[kMaxKids / 4];
+#pragma unroll
+                        for (int g = 0; g < kMaxKids / 4; ++g) w_cur[g] = w_next[g];
+                        if (v + 1 < nvar) {
+                            dv_next = list[v + 1];
+#pragma unroll
+                            for (int g = 0; g < kMaxKids / 4; ++g)
+                                if (g * 4 < cnt) w_next[g] = reinterpret_cast<const uint4 *>(vt + dv_next.y)[g];
+                        }
                         T msg[4] = {own[0], own[1], own[2], own[3]};
 #pragma unroll
                         for (int g = 0; g < kMaxKids / 4; ++g) {
                             if (g * 4 < cnt) {
-                                const uint4 wb = wr[g];
+                                const uint4 wb = w_cur[g];
                                 const T w0 = weight_of<T>(wb.x), w1 = weight_of<T>(wb.y), w2 = weight_of<T>(wb.z), w3 = weight_of<T>(wb.w);
 #pragma unroll
                                 for (int q = 0; q < 4; ++q)
@@ -670,7 +720,50 @@ cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchA
                 // every replay warp reads message rows written by the others
                 asm volatile("bar.sync 2, %0;" ::"r"(NRW * 32) : "memory");
             }
-            if (a.sched_smem) {
+            if (SHARE && a.flat) {
+                // Two-layer tree with shared messages: a pattern's schedule is the master's decode alone, a
+                // weighted sum of n-s message rows.  NP patterns at a time, no layer bookkeeping.
+                const int nst = a.nst;
+                const int ngroups = (a.batch + NP - 1) / NP;
+                const int g0 = ngroups < NRW ? (int)((rw + NRW - (t * (unsigned)ngroups) % NRW) % NRW) : rw;
+                for (int g = g0; g < ngroups; g += NRW) {
+                    T acc[NP][4];
+#pragma unroll
+                    for (int p = 0; p < NP; ++p)
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) acc[p][q] = T(0);
+                    const uint32_t *mine = ent + g * NP;
+#pragma unroll 4
+                    for (int k = 0; k < nst; ++k) {
+                        uint32_t en[NP];
+                        if (NP == 4) {
+                            const uint4 t4 = *reinterpret_cast<const uint4 *>(mine + (size_t)k * batch_pad);
+                            en[0] = t4.x; en[1] = t4.y; en[NP - 2] = t4.z; en[NP - 1] = t4.w;
+                        } else {
+                            const uint2 t2 = *reinterpret_cast<const uint2 *>(mine + (size_t)k * batch_pad);
+                            en[0] = t2.x; en[1] = t2.y;
+                        }
+#pragma unroll
+                        for (int p = 0; p < NP; ++p) {
+                            const T w = weight_of<T>(wtab_s[en[p] >> 12]);
+                            const V4 v = *reinterpret_cast<const V4 *>(Eb + (size_t)(en[p] & 0xfffu) * TILE + lane * 4);
+                            acc[p][0] += w * v.x; acc[p][1] += w * v.y; acc[p][2] += w * v.z; acc[p][3] += w * v.w;
+                        }
+                    }
+                    if (gcol < a.d) {
+#pragma unroll
+                        for (int p = 0; p < NP; ++p) {
+                            const int b = g * NP + p;
+                            if (b < a.batch) {
+                                V4 o;
+                                o.x = finish<T>(acc[p][0], a.shift); o.y = finish<T>(acc[p][1], a.shift);
+                                o.z = finish<T>(acc[p][2], a.shift); o.w = finish<T>(acc[p][3], a.shift);
+                                *reinterpret_cast<V4 *>(reinterpret_cast<T *>(a.out) + (size_t)b * a.d + gcol) = o;
+                            }
+                        }
+                    }
+                }
+            } else if (a.sched_smem) {
                 // NP patterns at a time per warp: their schedules visit the same layers, so one
                 // branch per step serves NP independent chains.  Step entries come from the staged
                 // table (broadcast shared-memory loads); the loop is unrolled by two so that the E rows
@@ -1173,13 +1266,6 @@ struct PgArgs {
     unsigned long long wait_ns;  // bound of every wait, in nanoseconds
 };
 
-__device__ __forceinline__ void bulk_load_1d(void *smem_dst, const void *gsrc, uint32_t bytes, uint64_t *bar) {
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-        ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
-        : "memory");
-}
-
 // RG = rows handled together in pass A (1, 2 or 4; at most the rows of a block).  GENERAL = false is the
 // case of one slot per item without slot coefficient, kept free of the bookkeeping of the general one
 // (measured: 5 % faster on 2048 x 4096 partitions).
@@ -1596,12 +1682,10 @@ static cudaError_t run_batch_w(int nlw, int nrw, int lmax, const CUtensorMap &ma
                     : run_batch_l<T, 4, 8, false>(lmax, map, ba, grid, smem, stream);
 }
 
-cudaError_t launch_fused_batch_tma(const AggArgs &a, const DeviceInfo &dev, const Tuning &tune, EncodeTiledFn encode,
-                                   cudaStream_t stream, int64_t *launches, bool *done) {
-    *done = false;
-    if (!encode || !tma_eligible(a)) return cudaSuccess;
+BatchShape batch_shape(const AggArgs &a, const DeviceInfo &dev, const Tuning &tune) {
+    BatchShape sh;
     const int tile = 128;
-    const int nrw = (tune.ncw == 4 && !a.n_ops) ? 4 : 8;  // replay warps
+    sh.nrw = (tune.ncw == 4 && !a.n_ops) ? 4 : 8;  // replay warps
     // same-shape batches stage their schedules in shared memory (layer word per step, one 4-byte entry
     // per step and pattern, patterns padded to the replay group size, the weight table) when small
     const int lmax = pick_lmax(a.L);
@@ -1617,74 +1701,90 @@ cudaError_t launch_fused_batch_tma(const AggArgs &a, const DeviceInfo &dev, cons
     const int n_rows = a.n_ops ? a.n_rows : a.n_union;
     const size_t e_one = (size_t)n_rows * tile * 4;
     const size_t budget = (size_t)dev.smem_optin - 512;   // barriers and flags take the rest
-    // Shared memory = nbuf x E + staged schedules + one private ring of `stages` boxes of R rows per
-    // loader warp.  Measured on B200 (d = 2^22, m = 16, 120 nodes, 64 patterns): six loaders with two
-    // boxes of 8 KB each stream at the copy bandwidth; four loaders reach 90 % of it, boxes of 4 KB two
-    // thirds, a third box per loader adds nothing.  So: boxes as tall as fit come first, then the
+    // Shared memory = nbuf x E + staged schedules + one private ring of `stages` boxes of R rows per loader warp.  Measured on B200 (d = 2^22, m = 16, 120 nodes, 64 patterns): six
+    // loaders with two boxes of 8 KB each stream at the copy bandwidth; four loaders reach 90 % of it, boxes
+    // of 4 KB two thirds, a third box per loader adds nothing.  So: boxes as tall as fit come first, then the
     // second E buffer, then six loaders rather than four.
     int nbuf = 0, stages = 0, R = 0, nlw = 0;
     const int want_loaders = tune.ctas_per_sm == 4 ? 4 : 6;
     // Few slot rows per node (m <= 8, coded gradients): a box of one node would be 0.5-4 KB, too small for
     // the copy engine.  Then a box takes the rows of npb consecutive union nodes; the selection below sees
     // such a box as one tall node, and falls back to one node per box if tall boxes do not fit beside E.
-    bool multi = a.npb > 1 && a.boxes && a.n_boxes > 0 && a.npb * a.m <= kMaxBoxRows && !tune.rows;
+    bool multi = a.npb > 1 && a.n_boxes > 0 && a.npb * a.m <= kMaxBoxRows && !tune.rows;
     for (int attempt = 0; attempt < 2 && !nbuf; ++attempt) {
-    if (attempt == 1) {
-        if (!multi) break;
-        multi = false;
-    }
-    const int node_rows = multi ? a.npb * a.m : a.m;
-    for (int try_buf = tune.e_buffers == 1 ? 1 : 2; try_buf >= 1 && !nbuf; --try_buf) {
-        if (budget <= try_buf * e_one + sched_bytes) continue;
-        const size_t ring_budget = budget - try_buf * e_one - sched_bytes;
-        const int want_stages = tune.stages ? tune.stages : 2;
-        int best_r = 0, best_depth = 0, best_lw = 0;
-        for (int lw = want_loaders; lw >= 4; lw -= 2) {
-            for (int depth = want_stages; depth >= 2; --depth) {
-                const int cap = (int)std::min<size_t>(kMaxBoxRows, ring_budget / ((size_t)lw * depth * tile * 4));
-                if (cap < 1) continue;
-                const int r = multi ? (node_rows <= cap ? node_rows : 0)
-                                    : (tune.rows && a.m % tune.rows == 0 && tune.rows <= cap ? tune.rows : rows_per_box(a.m, cap));
-                if (r > best_r) { best_r = r; best_depth = depth; best_lw = lw; }
+        if (attempt == 1) {
+            if (!multi) break;
+            multi = false;
+        }
+        const int node_rows = multi ? a.npb * a.m : a.m;
+        for (int try_buf = tune.e_buffers == 1 ? 1 : 2; try_buf >= 1 && !nbuf; --try_buf) {
+            if (budget <= try_buf * e_one + sched_bytes) continue;
+            const size_t ring_budget = budget - try_buf * e_one - sched_bytes;
+            const int want_stages = tune.stages ? tune.stages : 2;
+            int best_r = 0, best_depth = 0, best_lw = 0;
+            for (int lw = want_loaders; lw >= 4; lw -= 2) {
+                for (int depth = want_stages; depth >= 2; --depth) {
+                    const size_t per_row = (size_t)lw * depth * tile * 4, fixed = (size_t)lw * depth * 8;
+                    if (ring_budget <= fixed) continue;
+                    const int cap = (int)std::min<size_t>(kMaxBoxRows, (ring_budget - fixed) / per_row);
+                    if (cap < 1) continue;
+                    const int r = multi ? (node_rows <= cap ? node_rows : 0)
+                                        : (tune.rows && a.m % tune.rows == 0 && tune.rows <= cap ? tune.rows : rows_per_box(a.m, cap));
+                    if (r > best_r) { best_r = r; best_depth = depth; best_lw = lw; }
+                }
+            }
+            // two buffers only if they do not cost more than half of the box height one buffer allows
+            if (best_r && (try_buf == 1 || 2 * best_r >= std::min(node_rows, kMaxBoxRows))) {
+                nbuf = try_buf; R = best_r; stages = best_depth; nlw = best_lw;
             }
         }
-        // two buffers only if they do not cost more than half of the box height one buffer allows
-        if (best_r && (try_buf == 1 || 2 * best_r >= std::min(node_rows, kMaxBoxRows))) {
-            nbuf = try_buf; R = best_r; stages = best_depth; nlw = best_lw;
-        }
     }
-    }
-    if (!nbuf) return cudaSuccess;  // union too large for shared memory: caller falls back
+    if (!nbuf) return sh;  // union too large for shared memory
     const size_t stage_bytes = (size_t)R * tile * 4;
-    size_t smem = (size_t)nlw * stages * stage_bytes + nbuf * e_one + sched_bytes + (size_t)nlw * stages * 8 + 64 + 16;
-    if (smem > (size_t)dev.smem_optin) return cudaSuccess;
+    size_t smem = (size_t)nlw * stages * (stage_bytes + 8) + nbuf * e_one + sched_bytes + 64 + 16;
+    if (smem > (size_t)dev.smem_optin) return sh;
     // the variant records of the shared messages ride in shared memory too when the rest leaves room
-    int vtab_smem = 0;
-    if (a.n_ops && sched_bytes && smem + (size_t)a.vtab_words * 4 <= (size_t)dev.smem_optin) {
-        vtab_smem = 1;
-        sched_bytes += (size_t)a.vtab_words * 4;
-        smem += (size_t)a.vtab_words * 4;
+    const size_t vtab_bytes = ((size_t)a.vtab_words * 4 + 15) & ~(size_t)15;   // what follows stays 16-byte aligned
+    if (a.n_ops && sched_bytes && smem + vtab_bytes <= (size_t)dev.smem_optin) {
+        sh.vtab_smem = 1;
+        sched_bytes += vtab_bytes;
+        smem += vtab_bytes;
     }
     const long long ntiles = (a.d + tile - 1) / tile;
-    const int grid = (int)std::min<long long>(ntiles, (long long)dev.sm_count);
+    const int grid = (int)std::min<long long>(ntiles, (long long)std::max(1, dev.sm_count));
+    sh.cpn = multi ? 1 : a.m / R;
+    sh.n_groups = multi ? a.n_boxes : a.n_union;
     // box counters are 32-bit
-    if ((ntiles / grid + 1) * (long long)a.n_union * (multi ? 1 : a.m / R) >= (1ll << 31)) return cudaSuccess;
+    if ((ntiles / grid + 1) * (long long)sh.n_groups * sh.cpn >= (1ll << 31)) return sh;
+    sh.nbuf = nbuf; sh.stages = stages; sh.R = R; sh.nlw = nlw; sh.multi = multi ? 1 : 0; sh.nst = nst;
+    sh.sched_bytes = sched_bytes; sh.smem = smem; sh.n_rows = n_rows; sh.grid = grid;
+    sh.ok = true;
+    return sh;
+}
 
+int unit_words() { return kUnitWords; }
+
+cudaError_t launch_fused_batch_tma(const AggArgs &a, const BatchShape &sh, const Tuning &tune, EncodeTiledFn encode,
+                                   cudaStream_t stream, int64_t *launches, bool *done) {
+    *done = false;
+    if (!encode || !sh.ok || !a.units || !tma_eligible(a)) return cudaSuccess;
+    const int tile = 128;
     CUtensorMap map;
-    if (make_map(encode, &map, a, tile, R) != CUDA_SUCCESS) return cudaSuccess;
+    if (make_map(encode, &map, a, tile, sh.R) != CUDA_SUCCESS) return cudaSuccess;
 
     BatchArgs ba;
     ba.coeff = a.coeff; ba.steps = a.steps; ba.pat_off = a.pat_off; ba.unodes = a.unodes; ba.n_union = a.n_union;
-    ba.batch = a.batch; ba.same_shape = a.same_shape; ba.m = a.m; ba.R = R; ba.cpn = a.m / R; ba.stages = stages;
-    ba.d = a.d; ba.ntiles = ntiles; ba.out = a.out; ba.shift = a.shift; ba.status = a.status;
-    ba.sched_smem = (int)sched_bytes; ba.nst = nst; ba.nbuf = nbuf; ba.wtab = a.wtab; ba.n_wtab = a.n_wtab;
-    ba.boxes = multi ? a.boxes : nullptr; ba.n_boxes = multi ? a.n_boxes : 0; ba.npb = multi ? a.npb : 1;
-    if (multi) ba.cpn = 1;
+    ba.batch = a.batch; ba.same_shape = a.same_shape; ba.m = a.m; ba.R = sh.R; ba.cpn = sh.cpn; ba.stages = sh.stages;
+    ba.d = a.d; ba.ntiles = (a.d + tile - 1) / tile; ba.out = a.out; ba.shift = a.shift; ba.status = a.status;
+    ba.sched_smem = (int)sh.sched_bytes; ba.nst = sh.nst; ba.nbuf = sh.nbuf; ba.wtab = a.wtab; ba.n_wtab = a.n_wtab;
+    ba.units = a.units; ba.n_groups = sh.n_groups;
     ba.wait_ns = tune.wait_limit_ns;
-    ba.n_rows = n_rows; ba.n_ops = a.n_ops; ba.ops = a.ops; ba.vtab = a.vtab; ba.vtab_words = a.vtab_words;
-    ba.vtab_smem = vtab_smem;
-    const cudaError_t err = a.is_int ? run_batch_w<int>(nlw, nrw, lmax, map, ba, grid, smem, stream)
-                                     : run_batch_w<float>(nlw, nrw, lmax, map, ba, grid, smem, stream);
+    ba.n_rows = sh.n_rows; ba.n_ops = a.n_ops; ba.ops = a.ops; ba.vtab = a.vtab; ba.vtab_words = a.vtab_words;
+    ba.vtab_smem = sh.vtab_smem;
+    ba.flat = (a.n_ops && a.L == 2 && sh.sched_bytes) ? 1 : 0;
+    const int lmax = pick_lmax(a.L);
+    const cudaError_t err = a.is_int ? run_batch_w<int>(sh.nlw, sh.nrw, lmax, map, ba, sh.grid, sh.smem, stream)
+                                     : run_batch_w<float>(sh.nlw, sh.nrw, lmax, map, ba, sh.grid, sh.smem, stream);
     if (err == cudaSuccess) { *done = true; ++*launches; }
     return err;
 }

@@ -49,12 +49,13 @@ struct AggArgs {
     const int32_t *unodes;   // device [n_union]: union of used nodes (batch kernel)
     const uint32_t *wtab;    // device [n_wtab]: distinct weight bit patterns of the batch (n_wtab = 0: none)
     int n_wtab;
-    // batch kernel, few slot rows per node: device [n_boxes] TMA boxes that each cover up to `npb` union
-    // nodes with consecutive ids (their slot rows are contiguous).  x = first slot row, y = position of the
-    // first node in the union list (bits 0..19) | number of union nodes covered (bits 20..).  npb <= 1: unused.
-    const int2 *boxes = nullptr;
+    // batch kernel, few slot rows per node: n_boxes TMA boxes that each cover up to `npb` union nodes with
+    // consecutive ids (their slot rows are contiguous); npb <= 1: one node per box.
     int n_boxes = 0;
     int npb = 0;
+    // batch kernel: device table of unit records, one per box of a tile, laid out for the BatchShape the
+    // launch uses (16-byte aligned)
+    const uint32_t *units = nullptr;
     int n_union;
     int batch;
     int total_steps;
@@ -90,7 +91,29 @@ int inline_schedule_limit();
 
 cudaError_t launch_fused_tma(const AggArgs &a, const DeviceInfo &dev, const Tuning &tune, EncodeTiledFn encode,
                              cudaStream_t stream, int64_t *launches, bool *done);
-cudaError_t launch_fused_batch_tma(const AggArgs &a, const DeviceInfo &dev, const Tuning &tune, EncodeTiledFn encode,
+// Launch shape of the batch kernel for one expanded batch: depends on the tree, the union, the tables and the
+// device, not on any pointer, so it is fixed when the batch is expanded (the unit records are laid out for it).
+struct BatchShape {
+    bool ok = false;       // false: the union does not fit shared memory, the batch kernel cannot serve this batch
+    int nbuf = 0;          // buffers of coded gradients
+    int stages = 0;        // boxes per loader ring
+    int R = 0;             // slot rows per box
+    int nlw = 0, nrw = 0;  // loader and replay warps
+    int multi = 0;         // a box covers several small nodes
+    int cpn = 1;           // boxes per group (a tall node cut into cpn boxes)
+    int n_groups = 0;      // groups of boxes per tile
+    int nst = 0;           // same-shape batches: entries per schedule
+    int n_rows = 0;        // rows of a buffer of coded gradients
+    int vtab_smem = 0;
+    int grid = 0;
+    size_t sched_bytes = 0, smem = 0;
+};
+BatchShape batch_shape(const AggArgs &a, const DeviceInfo &dev, const Tuning &tune);
+// Words of a unit record: 16 coefficients (zero beyond the rows in use), then {first slot row of the box, E row
+// of the first node the box completes, rows after which a node is complete (0: it continues in the next box of
+// the group), rows of the box in use}.
+int unit_words();
+cudaError_t launch_fused_batch_tma(const AggArgs &a, const BatchShape &shape, const Tuning &tune, EncodeTiledFn encode,
                                    cudaStream_t stream, int64_t *launches, bool *done);
 // With a.split_scratch the schedule of a single pattern is cut at the master's children: every layer-1
 // sub-tree is folded by its own blocks into a row of the scratch, and a second small kernel adds the
