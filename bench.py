@@ -35,11 +35,39 @@ METRIC = "CR aggregation GB/s (fraction of HBM peak) and coded iterations/sec"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the timed kernel, from the ncu capture
-# summarised under profiles/ (absent = no capture of the current kernel on that workload).
-# cfg4: 917.5 MB measured at d = 2^21, scaled by 8 to d = 2^24 (traffic is proportional to d).
-# cfg5: 2076.0 MB measured at d = 2^18, scaled by 16 to d = 2^22.
-NCU_TRAFFIC_BYTES = {("cfg4", "f32", 1 << 24): 8 * 917.46e6, ("cfg5", "f32", 1 << 22): 16 * 2076.03e6}
+TRAFFIC_TABLE = os.path.join(ROOT, "profiles", "ncu_dram_traffic.txt")
+KERNEL_SOURCES = [os.path.join(ROOT, "paper_1902_01981_b200", "csrc", f) for f in ("cr_kernels.cu", "cr_tc.cu")]
+
+
+def kernel_source_digest() -> str:
+    """Short digest of the kernel sources: a DRAM-traffic figure taken under ncu is quoted only for the
+    very sources it was measured on."""
+    import hashlib
+    h = hashlib.sha256()
+    for path in KERNEL_SOURCES:
+        with open(path, "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(workload: str, dtype: str, d: int, kernel: str):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch of `kernel` on `workload`, from the table of
+    ncu captures under profiles/ (one line per capture: workload, dtype, captured d, kernel as the library
+    names it, DRAM bytes per launch at the captured d, digest of the kernel sources, summary file).  The
+    captures are small cases; traffic grows in proportion to d, so the figure is scaled by d / captured d.
+    None when there is no capture, when another kernel served the call, or when the kernel sources have
+    changed since the capture."""
+    try:
+        rows = [ln.split("|") for ln in open(TRAFFIC_TABLE) if ln.strip() and not ln.startswith("#")]
+    except OSError:
+        return None
+    digest = kernel_source_digest()
+    for r in rows:
+        r = [c.strip() for c in r]
+        if len(r) >= 7 and r[0] == workload and r[1] == dtype and r[3] == kernel and r[5] == digest:
+            return {"bytes": float(r[4]) * d / float(r[2]), "captured_d": int(r[2]), "summary": r[6],
+                    "note": "ncu capture of a small case, scaled by d / captured d"}
+    return None
 
 
 def peak_hbm():
@@ -146,10 +174,13 @@ class L2Flush:
 
 # ----------------------------------------------------------------------------- CPU oracle legs
 
-def oracle_sample(cfg, d_sample: int, steps: int, warmup: int, G=None):
+def oracle_sample(cfg, d_sample: int, steps: int, warmup: int, G=None, threads: int = 1):
     """Times the CPU oracle, as it stands, on `d_sample` columns of the workload (the array G
-    [P, d_sample] if given, else freshly drawn ones).
+    [P, d_sample] if given, else freshly drawn ones).  With threads > 1 the columns are cut into chunks
+    and the oracle's CR.Execute runs on the chunks side by side (a thread pool; NumPy releases the
+    interpreter lock inside its array operations) -- the oracle's code is the same either way.
     Returns (seconds per step, algorithmic bytes per step, results of the last step, masks used)."""
+    from concurrent.futures import ThreadPoolExecutor
     from oracle import cr_oracle as O
     from oracle import cr_setup
     code, local, _ = cr_setup.setup(cfg)
@@ -159,10 +190,20 @@ def oracle_sample(cfg, d_sample: int, steps: int, warmup: int, G=None):
     masks = inputs.straggler_masks(cfg["n"], cfg["L"], cfg["s"], (steps + warmup) * batch, cfg["mask_seed"],
                                    cfg.get("exactly_s", False)).reshape(steps + warmup, batch, -1)
     m = len(local[0])
+    threads = max(1, min(threads, d_sample // 1024))
+    bounds = np.linspace(0, d_sample, 4 * threads + 1).astype(int) if threads > 1 else None
+    chunks = [np.ascontiguousarray(G[:, a:b]) for a, b in zip(bounds[:-1], bounds[1:])] if threads > 1 else None
+    pool = ThreadPoolExecutor(threads) if threads > 1 else None
+
+    def execute_all(mk):
+        if pool is None:
+            return O.execute(code, local, G, mk)
+        return np.concatenate(list(pool.map(lambda c: O.execute(code, local, c, mk), chunks)))
+
     times, nbytes, last = [], [], None
     for it in range(steps + warmup):
         t0 = time.perf_counter()
-        last = [O.execute(code, local, G, masks[it, b]) for b in range(batch)]
+        last = [execute_all(masks[it, b]) for b in range(batch)]
         dt = time.perf_counter() - t0
         if it >= warmup:
             times.append(dt)
@@ -170,17 +211,29 @@ def oracle_sample(cfg, d_sample: int, steps: int, warmup: int, G=None):
             for b in range(batch):
                 union |= set(O.used_nodes(code, masks[it, b]))
             nbytes.append(4 * d_sample * (m * len(union) + batch))
+    if pool is not None:
+        pool.shutdown()
     return float(np.mean(times)), float(np.mean(nbytes)), last, masks[-1]
 
 
-def calibrated_columns(cfg, steps: int, seconds: float, max_cols: int) -> int:
+def calibrated_columns(cfg, steps: int, seconds: float, max_cols: int, threads: int = 1) -> int:
     """Largest power-of-two column count (>= 4096, <= max_cols) for which `steps` oracle steps take
-    about `seconds`, from one timed step on 4096 columns."""
+    about `seconds` on `threads` threads, from one timed single-thread step on 4096 columns (taken as if
+    the threads scaled perfectly: the sample then errs on the short side)."""
     sec, _, _, _ = oracle_sample(cfg, 4096, 1, 0)
     cols = 4096
-    while cols * 2 <= max_cols and sec * (cols * 2 / 4096.0) * steps <= seconds:
+    while cols * 2 <= max_cols and sec * (cols * 2 / 4096.0) * steps / threads <= seconds:
         cols *= 2
     return cols
+
+
+def blas_threads() -> int:
+    """Threads NumPy's BLAS uses for a matrix product (1 if that cannot be told)."""
+    try:
+        from threadpoolctl import threadpool_info
+        return max([int(i.get("num_threads", 1)) for i in threadpool_info() if i.get("user_api") == "blas"] or [1])
+    except Exception:
+        return 1
 
 
 def host_threads() -> int:
@@ -196,18 +249,19 @@ def run_reference(args, cfg):
     if rank != 0:
         return
     # bounded sample: calibrate the oracle on 4096 columns, then size the sample for about a minute
-    d_sample = calibrated_columns(cfg, args.steps + args.warmup, 60.0, min(args.ref_columns, cfg["d"]))
-    sec, nbytes, _, _ = oracle_sample(cfg, d_sample, args.steps, args.warmup)
+    cores = host_threads()
+    d_sample = calibrated_columns(cfg, args.steps + args.warmup, 60.0, min(args.ref_columns, cfg["d"]), cores)
+    sec, nbytes, _, _ = oracle_sample(cfg, d_sample, args.steps, args.warmup, threads=cores)
     value = nbytes / sec / 1e9
-    sample = f"first {d_sample} of {cfg['d']} columns, every step a fresh straggler pattern"
+    sample = (f"first {d_sample} of {cfg['d']} columns, every step a fresh straggler pattern, NumPy fp64, "
+              f"column chunks on {cores} threads")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": workload_config(args.workload, cfg, None),
         "iterations_per_s": 1.0 / sec,
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
-                         "host_threads_available": host_threads()},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -274,8 +328,8 @@ def run_reference_regression(args, cfg):
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": regression_workload_name(args.workload, cfg)},
         "iterations_per_s": 1.0 / sec,
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
-                         "host_threads_available": host_threads()},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                         "sample": sample + "; the matrix products run on NumPy's BLAS threads (the count given), CR.Execute on one"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -292,6 +346,224 @@ def workload_config(name, cfg, extra):
     if extra:
         out.update(extra)
     return out
+
+
+CODE_IDS = {"printed_3_1": "CR_CODE_PAPER_3_1", "cyclic": "CR_CODE_CYCLIC_RANDOM", "repetition": "CR_CODE_FRACTIONAL_REPETITION"}
+
+
+class AggregateSetup:
+    """An aggregation workload resident on one GPU: plan, slot buffer, output, straggler patterns."""
+
+    def __init__(self, torch, B, cfg, dtype, dev, seed_offset=0, patterns=256):
+        self.torch, self.B, self.cfg, self.dev = torch, B, cfg, dev
+        self.is_int = dtype == "int32"
+        self.plan = B.cr_plan_create(cfg["n"], cfg["L"], cfg["s"], cfg["P"], cfg["d"], code=getattr(B, CODE_IDS[cfg["code"]]),
+                                     dtype=B.CR_I32 if self.is_int else B.CR_F32, seed=0, device=dev.index or 0)
+        self.N, self.m, self.groups = B.cr_plan_num_nodes(self.plan), B.cr_plan_load(self.plan), B.cr_plan_num_groups(self.plan)
+        self.d, self.batch = cfg["d"], cfg.get("batch", 1)
+        self.tdtype = torch.int32 if self.is_int else torch.float32
+        # synthetic inputs: one vector per partition on the host, replicated into the slots on the device
+        if self.is_int:
+            self.G_parts = inputs.integer_gradients(cfg["P"], self.d, cfg["seed"] + seed_offset, cfg.get("int_bound", 1 << 10))
+        else:
+            self.G_parts = inputs.partition_gradients(cfg["P"], self.d, cfg["seed"] + seed_offset, cfg.get("std", 1.0))
+        part = torch.from_numpy(B.slot_partitions(self.plan).astype(np.int64).reshape(-1)).to(dev)
+        parts_dev = torch.from_numpy(self.G_parts).to(dev)
+        self.G_slots = torch.empty((self.N * self.m, self.d), dtype=self.tdtype, device=dev)
+        step_rows = max(1, (1 << 30) // (4 * self.d))
+        for r0 in range(0, self.N * self.m, step_rows):
+            torch.index_select(parts_dev, 0, part[r0:r0 + step_rows], out=self.G_slots[r0:r0 + step_rows])
+        del parts_dev
+        self.out = torch.zeros((self.batch, self.d), dtype=self.tdtype, device=dev)
+        self.total = patterns                       # distinct straggler patterns, cycled over the steps
+        self.masks = inputs.straggler_masks(cfg["n"], cfg["L"], cfg["s"], self.total * self.batch, cfg["mask_seed"],
+                                            cfg.get("exactly_s", False)).reshape(self.total, self.batch, self.groups)
+        self.step_bytes = [B.cr_aggregate_bytes(self.plan, self.masks[i])[0] for i in range(self.total)]
+        self.need_flush = self.d * 4 * cfg["P"] <= 126e6
+        self.flush = L2Flush(torch, dev) if self.need_flush else None
+        self.stream = torch.cuda.current_stream()
+
+    def timed(self, flags, steps, warmup, ws=None, dist=None, first=0):
+        """`steps` calls of cr_aggregate, a CUDA-event pair around each on the launching stream.
+        Returns (seconds per step [steps], seconds of the whole region on the device, host window)."""
+        torch, B = self.torch, self.B
+        starts = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        stops = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        for i in range(warmup):
+            B.cr_aggregate(self.plan, self.G_slots, self.masks[(first + i) % self.total], self.out, flags, ws, self.stream)
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+        t0 = time.time()
+        n0 = B.cr_plan_launch_count(self.plan)
+        for i in range(steps):
+            if self.flush is not None:
+                self.flush(i)
+            starts[i].record(self.stream)
+            B.cr_aggregate(self.plan, self.G_slots, self.masks[(first + warmup + i) % self.total], self.out, flags, ws, self.stream)
+            stops[i].record(self.stream)
+        torch.cuda.synchronize()
+        t1 = time.time()
+        self.launches = B.cr_plan_launch_count(self.plan) - n0
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+        per = np.array([a.elapsed_time(b) for a, b in zip(starts, stops)]) * 1e-3
+        span = starts[0].elapsed_time(stops[-1]) * 1e-3
+        return per, (span if self.flush is None else float(per.sum())), (t0, t1)
+
+    def bytes_of(self, steps, warmup, first=0):
+        return float(sum(self.step_bytes[(first + warmup + i) % self.total] for i in range(steps)))
+
+    def host_cost_us(self, flags, calls=200):
+        """Host time of one call with the stream idle (median over `calls`): the direct form, which expands
+        the masks, and the form with a schedule made beforehand, given plain addresses."""
+        torch, B = self.torch, self.B
+        sched = B.cr_schedule_create(self.plan, self.masks[0], flags)
+        g, o, st = self.G_slots.data_ptr(), self.out.data_ptr(), self.stream.cuda_stream
+        direct, scheduled = [], []
+        for i in range(calls):
+            torch.cuda.synchronize()
+            t0 = time.perf_counter_ns()
+            B.cr_aggregate(self.plan, self.G_slots, self.masks[0], self.out, flags, None, self.stream)
+            t1 = time.perf_counter_ns()
+            torch.cuda.synchronize()
+            t2 = time.perf_counter_ns()
+            B.cr_aggregate_scheduled(self.plan, g, sched, o, (0, 0), st)
+            t3 = time.perf_counter_ns()
+            direct.append(t1 - t0)
+            scheduled.append(t3 - t2)
+        torch.cuda.synchronize()
+        B.cr_schedule_destroy(sched)
+        return {"cr_aggregate": float(np.median(direct)) * 1e-3, "cr_aggregate_scheduled": float(np.median(scheduled)) * 1e-3,
+                "note": "host clock around the call through the Python binding, stream idle, median of %d" % calls}
+
+    def parity_on_sample(self, cols, flags, patterns=2):
+        """The GPU result on the first `cols` columns against the CPU oracle for the last straggler patterns:
+        worst relative L2 error (fp32) or exact equality (int32)."""
+        from oracle import cr_oracle as O
+        from oracle import cr_setup
+        torch, B = self.torch, self.B
+        code, local, _ = cr_setup.setup(self.cfg)
+        mk = self.masks[self.total - 1]
+        B.cr_aggregate(self.plan, self.G_slots, mk, self.out, flags, None, self.stream)
+        torch.cuda.synchronize()
+        got = self.out[:, :cols].cpu().numpy()
+        G = np.ascontiguousarray(self.G_parts[:, :cols])
+        picks = sorted(set(np.linspace(0, self.batch - 1, min(patterns, self.batch)).astype(int).tolist()))
+        if self.is_int:
+            exact = G.astype(np.int64).sum(0)
+            ok = all(np.array_equal(got[b].astype(np.int64), exact) and
+                     np.array_equal(O.execute_integer(code, local, G, mk[b]), exact) for b in picks)
+            return {"bit_exact_on_sample": bool(ok), "columns": cols, "patterns": len(picks)}
+        worst = 0.0
+        for b in picks:
+            want = O.execute(code, local, G, mk[b])
+            worst = max(worst, float(np.linalg.norm(got[b].astype(np.float64) - want) / np.linalg.norm(want)))
+        return {"gpu_rel_l2_on_sample": worst, "columns": cols, "patterns": len(picks)}
+
+    def close(self):
+        self.B.cr_plan_destroy(self.plan)
+        del self.G_slots, self.out, self.G_parts
+        self.flush = None
+        self.torch.cuda.empty_cache()
+
+
+def other_aggregate(torch, B, dev, name, dtype, steps, overrides=None):
+    """One more workload measured in the same process: value, time, kernel, parity against the oracle on a
+    column sample.  Kept short; the headline region is not touched."""
+    cfg = dict(inputs.CONFIGS[name])
+    cfg.update(overrides or {})
+    ws = AggregateSetup(torch, B, cfg, dtype, dev, patterns=min(64, steps + 3))
+    try:
+        per, wall, _ = ws.timed(B.CR_AGG_FUSED, steps, 3)
+        kernel = B.cr_plan_last_kernel(ws.plan)
+        nbytes = ws.bytes_of(steps, 3)
+        assert B.cr_plan_device_status(ws.plan) == B.CR_OK, "a device-side wait timed out"
+        peak, peak_kind = peak_hbm()
+        value = nbytes / wall / 1e9
+        out = {"workload": workload_config(name, cfg, None)["workload"], "dtype": "int32" if ws.is_int else "f32",
+               "value": value, "unit": UNIT, "ms_per_step": wall / steps * 1e3, "median_launch_ms": float(np.median(per)) * 1e3,
+               "steps": steps, "kernel": kernel,
+               "algorithmic_bytes_per_step": nbytes / steps, "frac": value / peak, "peak_kind": f"of {peak_kind}",
+               "l2": "flushed between steps" if ws.need_flush else "inputs larger than L2"}
+        out.update(ws.parity_on_sample(min(cfg["d"], 1 << 15), B.CR_AGG_FUSED))
+        return out
+    finally:
+        ws.close()
+
+
+def other_regression(torch, B, name, steps):
+    """cfg3-like regression step measured in the same process: partial gradients of every slot, fused aggregation,
+    model update; the aggregated gradient of the last step checked against the oracle's (fp64 partial gradients
+    from the definition, then CR.Execute)."""
+    from oracle import cr_oracle as O
+    from oracle import cr_setup
+    cfg = dict(inputs.CONFIGS[name])
+    n, L, s, P, d, rows = cfg["n"], cfg["L"], cfg["s"], cfg["P"], cfg["d"], cfg["rows"]
+    plan = B.cr_plan_create(n, L, s, P, d, code=getattr(B, CODE_IDS[cfg["code"]]), device=0)
+    try:
+        N, m = B.cr_plan_num_nodes(plan), B.cr_plan_load(plan)
+        logistic = cfg["kind"] == "logistic"
+        loss = B.CR_LOSS_LOGISTIC if logistic else B.CR_LOSS_SQUARED
+        X, y, _ = (inputs.logistic_partitions(P, rows, d, cfg["seed"], cfg["x_std"]) if logistic else
+                   inputs.linreg_partitions(P, rows, d, cfg["seed"], cfg["x_std"], cfg["noise_std"]))
+        X_dev, y_dev = torch.from_numpy(X).cuda(), torch.from_numpy(y).cuda()
+        w_dev = torch.zeros(d, device="cuda")
+        G_slots = torch.zeros((N, m, d), device="cuda")
+        ws = torch.empty(max(16, B.cr_partial_gradients_workspace_bytes(plan, rows)), dtype=torch.uint8, device="cuda")
+        out = torch.zeros((1, d), device="cuda")
+        masks = inputs.straggler_masks(n, L, s, steps + 3, cfg.get("mask_seed", 1))
+        lr_eff = cfg["lr"] / P
+        flush = L2Flush(torch, "cuda") if X.nbytes <= 126e6 else None
+        stream = torch.cuda.current_stream()
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+        w_before = None
+        for i in range(steps + 3):
+            if i >= 3:
+                if flush is not None:
+                    flush(i)
+                ev[i - 3][0].record(stream)
+            if i == steps + 2:
+                w_before = w_dev.clone()
+            B.cr_partial_gradients_loss(plan, loss, X_dev, y_dev, rows, w_dev, G_slots, ws, stream)
+            if i >= 3:
+                ev[i - 3][1].record(stream)
+            B.cr_aggregate(plan, G_slots, masks[i], out, B.CR_AGG_FUSED, None, stream)
+            w_dev.sub_(out[0], alpha=lr_eff)
+            if i >= 3:
+                ev[i - 3][2].record(stream)
+        torch.cuda.synchronize()
+        t_grad = np.array([e[0].elapsed_time(e[1]) for e in ev]) * 1e-3
+        t_step = np.array([e[0].elapsed_time(e[2]) for e in ev]) * 1e-3
+        grad_bytes = 4.0 * rows * d * N * m
+        agg_bytes = float(np.mean([B.cr_aggregate_bytes(plan, masks[i])[0] for i in range(3, steps + 3)]))
+        peak, peak_kind = peak_hbm()
+        # parity of the last step's aggregated gradient
+        code, local, _ = cr_setup.setup(cfg)
+        w_h = w_before.cpu().numpy()
+        grad = O.partial_gradient_logistic if logistic else O.partial_gradient_linreg
+        G_parts = np.stack([grad(X[p], y[p], w_h) for p in range(P)])
+        want = O.execute(code, local, G_parts, masks[steps + 2])
+        got = out[0].cpu().numpy().astype(np.float64)
+        value = (grad_bytes + agg_bytes) / float(t_step.mean()) / 1e9
+        traffic = ncu_traffic(name, "f32", d, "partial gradients")
+        res = {"workload": regression_workload_name(name, cfg), "dtype": "f32", "value": value, "unit": UNIT,
+               "ms_per_step": float(t_step.mean()) * 1e3, "gradient_ms": float(t_grad.mean()) * 1e3, "steps": steps,
+               "kernel": "partial gradients (one pass) + " + B.cr_plan_last_kernel(plan),
+               "algorithmic_bytes_per_step": grad_bytes + agg_bytes, "frac": value / peak, "peak_kind": f"of {peak_kind}",
+               "gradient_GBs_algorithmic": grad_bytes / float(t_grad.mean()) / 1e9,
+               "l2": "flushed between steps" if flush is not None else "inputs larger than L2",
+               "gpu_rel_l2_of_aggregated_gradient": float(np.linalg.norm(got - want) / np.linalg.norm(want))}
+        if traffic:
+            res["gradient_dram_frac"] = traffic["bytes"] / float(t_grad.mean()) / 1e9 / peak
+            res["gradient_dram_note"] = ("DRAM bytes of an ncu capture over time over peak: slots that hold the same partition "
+                                         "share its rows through L2, so DRAM sees less than the algorithmic bytes")
+        return res
+    finally:
+        B.cr_plan_destroy(plan)
+        torch.cuda.empty_cache()
 
 
 def run_ours(args, cfg):
@@ -316,67 +588,12 @@ def run_ours(args, cfg):
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
 
-    is_int = args.dtype == "int32"
-    code_id = {"printed_3_1": B.CR_CODE_PAPER_3_1, "cyclic": B.CR_CODE_CYCLIC_RANDOM,
-               "repetition": B.CR_CODE_FRACTIONAL_REPETITION}[cfg["code"]]
-    plan = B.cr_plan_create(cfg["n"], cfg["L"], cfg["s"], cfg["P"], cfg["d"], code=code_id,
-                            dtype=B.CR_I32 if is_int else B.CR_F32, seed=0, device=local_rank)
+    ws0 = AggregateSetup(torch, B, cfg, args.dtype, dev, seed_offset=rank, patterns=min(args.steps + args.warmup, 256))
+    plan, is_int, d, batch, N, m = ws0.plan, ws0.is_int, ws0.d, ws0.batch, ws0.N, ws0.m
     if args.tune:
         B.cr_plan_tune(plan, *[int(x) for x in args.tune.split(",")])
     if args.share or args.e_buffers:
         B.cr_plan_tune_batch(plan, args.share, args.e_buffers)
-    N, m, groups = B.cr_plan_num_nodes(plan), B.cr_plan_load(plan), B.cr_plan_num_groups(plan)
-    d, batch = cfg["d"], cfg.get("batch", 1)
-    tdtype = torch.int32 if is_int else torch.float32
-
-    # synthetic inputs: one vector per partition on the host, replicated into the slots on the device
-    if is_int:
-        G_parts = inputs.integer_gradients(cfg["P"], d, cfg["seed"] + rank, cfg.get("int_bound", 1 << 10))
-    else:
-        G_parts = inputs.partition_gradients(cfg["P"], d, cfg["seed"] + rank, cfg.get("std", 1.0))
-    part = torch.from_numpy(B.slot_partitions(plan).astype(np.int64).reshape(-1)).to(dev)
-    parts_dev = torch.from_numpy(G_parts).to(dev)
-    G_slots = torch.empty((N * m, d), dtype=tdtype, device=dev)
-    step_rows = max(1, (1 << 30) // (4 * d))
-    for r0 in range(0, N * m, step_rows):
-        torch.index_select(parts_dev, 0, part[r0:r0 + step_rows], out=G_slots[r0:r0 + step_rows])
-    del parts_dev
-    out = torch.zeros((batch, d), dtype=tdtype, device=dev)
-    total = min(args.steps + args.warmup, 256)       # distinct straggler patterns, cycled over the steps
-    masks = inputs.straggler_masks(cfg["n"], cfg["L"], cfg["s"], total * batch, cfg["mask_seed"],
-                                   cfg.get("exactly_s", False)).reshape(total, batch, groups)
-    step_bytes = [B.cr_aggregate_bytes(plan, masks[i])[0] for i in range(total)]
-    need_flush = d * 4 * cfg["P"] <= 126e6
-    flush_buf = L2Flush(torch, dev) if need_flush else None
-    stream = torch.cuda.current_stream()
-
-    def timed_run(flags, ws=None, steps=args.steps, warmup=args.warmup):
-        starts = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
-        stops = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
-        for i in range(warmup):
-            B.cr_aggregate(plan, G_slots, masks[i], out, flags, ws, stream)
-        torch.cuda.synchronize()
-        if dist is not None:
-            dist.barrier()
-            torch.cuda.synchronize()
-        t0 = time.time()
-        n0 = B.cr_plan_launch_count(plan)
-        for i in range(steps):
-            if flush_buf is not None:
-                flush_buf(i)
-            starts[i].record(stream)
-            B.cr_aggregate(plan, G_slots, masks[(warmup + i) % total], out, flags, ws, stream)
-            stops[i].record(stream)
-        torch.cuda.synchronize()
-        t1 = time.time()
-        timed_run.launches = B.cr_plan_launch_count(plan) - n0
-        timed_run.window = (t0, t1)
-        if dist is not None:
-            dist.barrier()
-            torch.cuda.synchronize()
-        per = np.array([a.elapsed_time(b) for a, b in zip(starts, stops)]) * 1e-3
-        span = starts[0].elapsed_time(stops[-1]) * 1e-3
-        return per, (span if flush_buf is None else float(per.sum()))
 
     # ---- the timed region: K steps of the fused kernel
     try:
@@ -385,60 +602,76 @@ def run_ours(args, cfg):
         gpu_id = local_rank
     sampler = ClockSampler(gpu_id)
     sampler.wait_first_sample()
-    per, wall = timed_run(B.CR_AGG_FUSED)
-    launches = timed_run.launches
+    per, wall, window = ws0.timed(B.CR_AGG_FUSED, args.steps, args.warmup, dist=dist)
+    launches = ws0.launches
     timed_kernel = B.cr_plan_last_kernel(plan)
-    clocks = sampler.stop(timed_run.window)
+    clocks = sampler.stop(window)
     assert B.cr_plan_device_status(plan) == B.CR_OK, "a device-side wait timed out"
     # device time of the K steps: first start event to last stop event on the launching stream (with
     # an L2 flush between steps: the sum of the per-step intervals, which leaves the flushes out)
     elapsed = float(wall)
-    units = float(sum(step_bytes[(args.warmup + i) % total] for i in range(args.steps)))
+    units = ws0.bytes_of(args.steps, args.warmup)
     elapsed_all, units_all = combine_ranks(elapsed, units, world, dist, dev)
     value = units_all / elapsed_all / 1e9
-    result_last = out.clone()
+
+    # ---- a sustained leg of the same call, long enough for the clock samples to fall inside it (the
+    # K-step region above can be shorter than one sampling period); rank 0 only
+    sustained = None
+    if rank == 0 and not args.no_sustained and world == 1:
+        s_steps = int(min(20000, max(args.steps, np.ceil(args.sustain_seconds / max(float(per.mean()), 1e-6)))))
+        sampler2 = ClockSampler(gpu_id)
+        sampler2.wait_first_sample()
+        per2, wall2, window2 = ws0.timed(B.CR_AGG_FUSED, s_steps, 3)
+        clocks2 = sampler2.stop(window2)
+        bytes2 = ws0.bytes_of(s_steps, 3)
+        sustained = {"value": bytes2 / wall2 / 1e9, "unit": UNIT, "steps": s_steps, "seconds": wall2,
+                     "ms_per_step": wall2 / s_steps * 1e3, "clocks": clocks2,
+                     "ms_times_sm_mhz": (wall2 / s_steps * 1e3) * (clocks2.get("sm_mhz") or 0.0)}
+        if not clocks.get("samples_in_timed_region"):
+            clocks["note"] = ("the timed region is shorter than the sampling period: these samples lie around it; "
+                              "the sustained leg carries samples taken inside its own region")
 
     # ---- comparators on the same slots (rank 0 only, outside the timed region)
     extras = {}
+    host_cost = None
     if rank == 0 and not args.no_extras:
         ksteps = min(args.steps, 50)
-        bytes_k = float(np.mean([step_bytes[(args.warmup + i) % total] for i in range(ksteps)]))
+        bytes_k = ws0.bytes_of(ksteps, args.warmup) / ksteps
         for name, flags in (("fused_plain_loads", B.CR_AGG_FUSED_LDG), ("uncoded_sum_same_bytes", B.CR_AGG_UNCODED_SUM)):
-            p2, _ = timed_run(flags, steps=ksteps)
+            p2, _, _ = ws0.timed(flags, ksteps, args.warmup)
             extras[name] = {"GB/s": bytes_k / float(p2.mean()) / 1e9, "ms_per_step": float(p2.mean()) * 1e3}
         nws = B.cr_aggregate_workspace_bytes(plan, batch, B.CR_AGG_UNFUSED)
         free, _ = torch.cuda.mem_get_info()
         if nws < free - (2 << 30):
-            ws = torch.empty(nws, dtype=torch.uint8, device=dev)
-            p2, _ = timed_run(B.CR_AGG_UNFUSED, ws, steps=min(ksteps, 5))
+            wsb = torch.empty(nws, dtype=torch.uint8, device=dev)
+            p2, _, _ = ws0.timed(B.CR_AGG_UNFUSED, min(ksteps, 5), args.warmup, ws=wsb)
             extras["unfused_per_level"] = {"GB/s": bytes_k / float(p2.mean()) / 1e9, "ms_per_step": float(p2.mean()) * 1e3}
-            del ws
-        B.cr_aggregate(plan, G_slots, masks[total - 1], out, B.CR_AGG_FUSED, None, stream)
-        torch.cuda.synchronize()
+            del wsb
+        host_cost = ws0.host_cost_us(B.CR_AGG_FUSED)
 
     # ---- end to end through the host-buffer entry point: H2D of the slots and D2H of the result
     # inside the timed region
     e2e = None
     if not args.no_e2e:
         e2e_steps = max(1, min(args.e2e_steps, args.steps))
-        host_slots = torch.empty((N * m, d), dtype=tdtype, pin_memory=True)
-        host_slots.copy_(G_slots)
-        host_out = torch.empty((batch, d), dtype=tdtype, pin_memory=True)
+        host_slots = torch.empty((N * m, d), dtype=ws0.tdtype, pin_memory=True)
+        host_slots.copy_(ws0.G_slots)
+        host_out = torch.empty((batch, d), dtype=ws0.tdtype, pin_memory=True)
         torch.cuda.synchronize()
-        B.cr_aggregate_host(plan, host_slots, masks[0], host_out, G_slots, out, B.CR_AGG_FUSED, None, stream)
+        B.cr_aggregate_host(plan, host_slots, ws0.masks[0], host_out, ws0.G_slots, ws0.out, B.CR_AGG_FUSED, None, ws0.stream)
         if dist is not None:
             dist.barrier()
         t0 = time.perf_counter()
         for i in range(e2e_steps):
-            B.cr_aggregate_host(plan, host_slots, masks[(args.warmup + i) % total], host_out, G_slots, out,
-                                B.CR_AGG_FUSED, None, stream)
+            B.cr_aggregate_host(plan, host_slots, ws0.masks[(args.warmup + i) % ws0.total], host_out, ws0.G_slots, ws0.out,
+                                B.CR_AGG_FUSED, None, ws0.stream)
         torch.cuda.synchronize()
         e2e_elapsed = time.perf_counter() - t0
-        e2e_units = float(sum(step_bytes[(args.warmup + i) % total] for i in range(e2e_steps)))
+        e2e_units = ws0.bytes_of(e2e_steps, args.warmup)
         e2e_elapsed, e2e_units = combine_ranks(e2e_elapsed, e2e_units, world, dist, dev)
         e2e = {"value": e2e_units / e2e_elapsed / 1e9, "unit": UNIT,
                # cr_aggregate_host sends the slots of the consumed nodes only (stragglers are not waited for)
-               "h2d_bytes_per_step": int(e2e_units / e2e_steps / world - batch * d * 4 + masks[0].nbytes),
+               "h2d_bytes_per_step": int(e2e_units / e2e_steps / world - batch * d * 4 + ws0.masks[0].nbytes),
                "d2h_bytes_per_step": int(batch * d * 4),
                "steps": e2e_steps, "ms_per_step": e2e_elapsed / e2e_steps * 1e3}
         del host_slots
@@ -448,40 +681,55 @@ def run_ours(args, cfg):
         avg_launch = float(per.mean())
         avg_bytes = units / args.steps
         achieved = avg_bytes / avg_launch / 1e9
-        kern = timed_kernel
-        traffic = NCU_TRAFFIC_BYTES.get((args.workload, args.dtype, d)) if not args.tune else None
-        roofline = {"bound": "hbm", "kernel": kern, "achieved": achieved, "peak": peak, "unit": "GB/s",
-                    "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_nominal_8TBs": achieved / 8000.0,
-                    "traffic": traffic, "algorithmic_bytes_per_launch": avg_bytes,
+        dtype_name = "int32" if is_int else "f32"
+        traffic = ncu_traffic(args.workload, dtype_name, d, timed_kernel) if not (args.tune or args.tree) else None
+        roofline = {"bound": "hbm", "kernel": timed_kernel, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                    "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                    "frac_note": "the peak is a measured copy (read + write); a read-mostly stream can exceed it slightly",
+                    "frac_of_nominal_8TBs": achieved / 8000.0,
+                    "traffic": traffic["bytes"] if traffic else None, "traffic_source": traffic,
+                    "algorithmic_bytes_per_launch": avg_bytes,
                     "avg_launch_ms": avg_launch * 1e3, "best_launch_ms": float(per.min()) * 1e3}
         cpu = None
-        if not args.no_cpu_baseline:
-            d_sample = calibrated_columns(cfg, args.cpu_steps + 1, 15.0, min(d, args.cpu_columns))
-            sec, nbytes, last, last_masks = oracle_sample(
-                cfg, d_sample, args.cpu_steps, 1, np.ascontiguousarray(G_parts[:, :d_sample])) \
-                if not is_int else (None, None, None, None)
-            if sec is not None:
-                cpu = {"value": nbytes / sec / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
-                       "sample": f"first {d_sample} of {d} columns, {args.cpu_steps} steps, NumPy fp64",
-                       "ms_per_step_on_sample": sec * 1e3, "host_threads_available": host_threads()}
-                # by-product: the GPU result for the same masks on those columns against the oracle
-                B.cr_aggregate(plan, G_slots, last_masks, out, B.CR_AGG_FUSED, None, stream)
-                torch.cuda.synchronize()
-                got = out[:, :d_sample].cpu().numpy().astype(np.float64)
-                worst = max(float(np.linalg.norm(got[b] - last[b]) / np.linalg.norm(last[b])) for b in range(batch))
-                cpu["gpu_rel_l2_on_sample"] = worst
+        if not args.no_cpu_baseline and not is_int:
+            cores = host_threads()
+            d_sample = calibrated_columns(cfg, args.cpu_steps + 1, 15.0, min(d, args.cpu_columns), cores)
+            sec, nbytes, last, last_masks = oracle_sample(cfg, d_sample, args.cpu_steps, 1,
+                                                          np.ascontiguousarray(ws0.G_parts[:, :d_sample]), threads=cores)
+            cpu = {"value": nbytes / sec / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
+                   "sample": f"first {d_sample} of {d} columns, {args.cpu_steps} steps, NumPy fp64, column chunks on {cores} threads",
+                   "ms_per_step_on_sample": sec * 1e3}
+            # by-product: the GPU result for the same masks on those columns against the oracle
+            B.cr_aggregate(plan, ws0.G_slots, last_masks, ws0.out, B.CR_AGG_FUSED, None, ws0.stream)
+            torch.cuda.synchronize()
+            got = ws0.out[:, :d_sample].cpu().numpy().astype(np.float64)
+            worst = max(float(np.linalg.norm(got[b] - last[b]) / np.linalg.norm(last[b])) for b in range(batch))
+            cpu["gpu_rel_l2_on_sample"] = worst
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": elapsed_all / args.steps * 1e3, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "int32" if is_int else "f32", "data": "synthetic",
-            "config": workload_config(args.workload, cfg, {"slots_gb": N * m * d * 4 / 1e9, "tune": args.tune or "auto"}),
+            "scaling": "weak", "vs_baseline": None, "dtype": dtype_name, "data": "synthetic",
+            "config": workload_config(args.workload, cfg, None),
             "iterations_per_s": world * args.steps / elapsed_all,
             "patterns_per_s": world * args.steps * batch / elapsed_all,
             "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
-            "clocks": clocks, "comparators": extras,
+            "clocks": clocks, "sustained": sustained, "comparators": extras, "host_us_per_call": host_cost,
+            "slots_gb": N * m * d * 4 / 1e9, "tune": args.tune or "auto",
         }
+    ws0.close()
+    # ---- the other workloads of the results table, measured in the same process (default run, one GPU)
+    if rank == 0 and world == 1 and args.others and not (args.tune or args.tree or args.d or args.batch):
+        others = []
+        for name, dtype, steps, over in (("cfg5", "f32", 8, None), ("cfg5", "int32", 8, None), ("cfg2", "f32", 100, None),
+                                         ("cfg_tree12", "f32", 20, None),
+                                         ("cfg_tree12", "f32", 20, {"batch": 64, "d": 1 << 20}), ("cfg_cnn", "f32", 100, None)):
+            if name == args.workload and dtype == args.dtype and not over:
+                continue
+            others.append(other_aggregate(torch, B, dev, name, dtype, steps, over))
+        others.append(other_regression(torch, B, "cfg3", 20))
+        line["other_workloads"] = others
+    if rank == 0:
         print(json.dumps(line), flush=True)
-    B.cr_plan_destroy(plan)
     if dist is not None:
         dist.destroy_process_group()
 
@@ -585,8 +833,10 @@ def run_linreg(args, cfg):
     cpu = None
     if not args.no_cpu_baseline:
         sec, nbytes, sample = oracle_regression_sample(args.workload, cfg, args.cpu_steps, 1, 15.0)
-        cpu = {"value": nbytes / sec / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
-               "ms_per_step_on_sample": sec * 1e3, "host_threads_available": host_threads()}
+        cpu = {"value": nbytes / sec / 1e9, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+               "sample": sample + "; the matrix products run on NumPy's BLAS threads (the count given), CR.Execute on one",
+               "ms_per_step_on_sample": sec * 1e3}
+    traffic = ncu_traffic(args.workload, "f32", d, "partial gradients") if not args.tune_gradients else None
     line = {
         "metric": METRIC, "value": step_bytes * args.steps / elapsed / 1e9, "unit": UNIT, "n_gpus": 1,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": elapsed / args.steps * 1e3,
@@ -598,7 +848,11 @@ def run_linreg(args, cfg):
                    "l2": "inputs larger than L2 (no flush needed)" if flush is None else "L2 flushed between steps (256 MB written, then 256 MB read)"},
         "iterations_per_s": args.steps / elapsed,
         "roofline": {"bound": "hbm", "kernel": "partial gradients", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                     "frac": achieved / peak, "peak_kind": f"of {peak_kind}",
+                     "frac_note": "algorithmic bytes count every (node, slot) item reading its partition; items that hold the "
+                                  "same partition share its rows through L2, so this fraction can exceed 1 (see dram_frac)",
+                     "traffic": traffic["bytes"] if traffic else None, "traffic_source": traffic,
+                     "dram_frac": (traffic["bytes"] / float(t_grad.mean()) / 1e9 / peak) if traffic else None,
                      "algorithmic_bytes_per_launch": grad_bytes, "avg_launch_ms": float(t_grad.mean()) * 1e3,
                      "aggregate_ms": float((t_step - t_grad).mean()) * 1e3},
         "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
@@ -727,6 +981,11 @@ def main():
     ap.add_argument("--coded", action="store_true", help="regression workloads: gradient + encode in one kernel")
     ap.add_argument("--models", type=int, default=0, help="regression workloads: gradients of K models per pass (1..32)")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-sustained", action="store_true", help="skip the sustained leg of the headline call")
+    ap.add_argument("--sustain-seconds", type=float, default=2.0)
+    ap.add_argument("--others", dest="others", action="store_true", default=None,
+                    help="also measure the other workloads of the results table (default for the plain cfg4 run)")
+    ap.add_argument("--no-others", dest="others", action="store_false")
     ap.add_argument("--no-extras", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=3)
@@ -736,6 +995,8 @@ def main():
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
+    if args.others is None:
+        args.others = args.workload == "cfg4" and not (args.no_extras or args.no_e2e or args.no_cpu_baseline)
     cfg = dict(inputs.CONFIGS[args.workload])
     if args.d:
         cfg["d"] = args.d

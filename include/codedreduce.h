@@ -123,10 +123,10 @@ typedef enum {
  * solves, in fp64, the decode row a (a B = 1, supported on the lowest-indexed n-s non-stragglers)
  * for every straggler mask with at most s bits, per level.  With device >= 0 it makes that device
  * current for the call and allocates small device mirrors of the tables and a ring of eight staging
- * buffers (pinned host + device, 64 KB each or 64 bytes per node if that is more), through which
- * cr_aggregate and cr_decode send the expanded straggler patterns.  A call whose tables exceed a slot
- * (a large batch) re-allocates that slot once, which synchronises the device; cr_schedule_create keeps
- * even that out of a loop.  cr_plan_destroy frees everything.  *out is written only on CR_OK. */
+ * buffers (pinned host + device; 64 KB to 1 MB each, sized for batches of 64 patterns), through which
+ * cr_aggregate and cr_decode send the expanded straggler patterns.  The first call whose tables exceed a
+ * buffer (a larger batch) re-allocates the ring once, which synchronises the device; cr_schedule_create
+ * keeps even that out of a loop.  cr_plan_destroy frees everything.  *out is written only on CR_OK. */
 cr_status_t cr_plan_create(const cr_plan_desc_t *desc, cr_plan_t **out);
 cr_status_t cr_plan_destroy(cr_plan_t *plan);
 

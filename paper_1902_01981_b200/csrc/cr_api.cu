@@ -71,22 +71,31 @@ struct cr_plan {
 
 namespace {
 
-// Takes the next staging slot, waiting for the work that last used it, and makes it large enough.
+// Takes the next staging slot, waiting for the work that last used it.  A call whose tables do not fit
+// the slots grows the whole ring at once (every slot to twice the size asked for), so that this happens
+// once and not again for each of the eight slots as the loop reaches them: freeing and allocating pinned
+// memory waits for the device and can take milliseconds.
 cr_status_t stage_acquire(cr_plan *p, size_t bytes, StageSlot **out) {
+    if (p->ring[p->next].bytes < bytes) {
+        const size_t cap = std::max<size_t>(align16(bytes) * 2, 4096);
+        for (StageSlot &s : p->ring) {
+            if (s.pending) {
+                CR_CUDA(cudaEventSynchronize(s.ev));
+                s.pending = false;
+            }
+            if (s.host) cudaFreeHost(s.host);
+            if (s.dev) cudaFree(s.dev);
+            s.host = nullptr; s.dev = nullptr; s.bytes = 0;
+            CR_CUDA(cudaMallocHost(reinterpret_cast<void **>(&s.host), cap));
+            CR_CUDA(cudaMalloc(reinterpret_cast<void **>(&s.dev), cap));
+            s.bytes = cap;
+        }
+    }
     StageSlot &s = p->ring[p->next];
     p->next = (p->next + 1) % kRing;
     if (s.pending) {
         CR_CUDA(cudaEventSynchronize(s.ev));
         s.pending = false;
-    }
-    if (s.bytes < bytes) {
-        if (s.host) cudaFreeHost(s.host);
-        if (s.dev) cudaFree(s.dev);
-        s.host = nullptr; s.dev = nullptr; s.bytes = 0;
-        const size_t cap = std::max<size_t>(align16(bytes) * 2, 4096);
-        CR_CUDA(cudaMallocHost(reinterpret_cast<void **>(&s.host), cap));
-        CR_CUDA(cudaMalloc(reinterpret_cast<void **>(&s.dev), cap));
-        s.bytes = cap;
     }
     if (!s.ev) CR_CUDA(cudaEventCreateWithFlags(&s.ev, cudaEventDisableTiming));
     *out = &s;
@@ -380,7 +389,9 @@ cr_status_t cr_plan_create(const cr_plan_desc_t *desc, cr_plan_t **out) {
         // staging ring for the expanded schedules: sized here for single patterns and small batches, so
         // that the device calls of an ordinary loop never allocate (a larger batch grows its slot once)
         {
-            const size_t cap = std::max<size_t>(64 * 1024, align16((size_t)p->hp.N * 64));
+            // room for a batch of 64 patterns over the whole tree (two schedules of 16-byte entries per pattern
+            // and node), within 64 KB .. 1 MB per slot
+            const size_t cap = std::min<size_t>(1u << 20, std::max<size_t>(64 * 1024, align16((size_t)p->hp.N * 64 * 40)));
             for (StageSlot &s : p->ring) {
                 CR_CUDA_P(cudaMallocHost(reinterpret_cast<void **>(&s.host), cap));
                 CR_CUDA_P(cudaMalloc(reinterpret_cast<void **>(&s.dev), cap));

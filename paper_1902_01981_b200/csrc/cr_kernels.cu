@@ -34,20 +34,18 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
-// One probe of a barrier phase.  The hint lets the hardware park the warp for up to about a microsecond
-// while the phase is pending (it returns at once when the phase completes), so that a waiting warp does not
-// spend the issue slots of its scheduler on polling: with eight replay warps spinning, polling was a third of
-// all instructions the batch kernel issued.
+// One probe of a barrier phase.  (A suspend-time hint on the probe, 200 ns or 1 us, changed nothing measurable
+// in any kernel here and is not used.)
 __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
         "{\n"
         ".reg .pred p;\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
         "selp.u32 %0, 1, 0, p;\n"
         "}\n"
         : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity), "r"(1000u)
+        : "r"(smem_u32(bar)), "r"(parity)
         : "memory");
     return ok != 0;
 }
@@ -1090,9 +1088,10 @@ cr_uncoded_sum_kernel(const T *__restrict__ G, const Step *__restrict__ steps, c
 
 template <typename T, int V>
 __global__ void __launch_bounds__(256)
-cr_encode_kernel(const T *__restrict__ G, const T *__restrict__ coeff, const int32_t *__restrict__ nodes, int m,
+cr_encode_kernel(const T *__restrict__ G, const T *__restrict__ coeff, const int32_t *__restrict__ nodes, int y0, int m,
                  long long d, T *__restrict__ E) {
-    const int v = nodes ? __ldg(&nodes[blockIdx.y]) : (int)blockIdx.y;
+    // (y0: first entry served by this launch; a grid has at most 65535 rows of blocks)
+    const int v = nodes ? __ldg(&nodes[y0 + blockIdx.y]) : y0 + (int)blockIdx.y;
     const long long col = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * V;
     if (col >= d) return;
     const T *row = G + (size_t)v * m * d + col;
@@ -1113,8 +1112,8 @@ cr_encode_kernel(const T *__restrict__ G, const T *__restrict__ coeff, const int
 template <typename T, int V>
 __global__ void __launch_bounds__(256)
 cr_decode_kernel(const T *__restrict__ M_child, const T *__restrict__ E_parent, const T *__restrict__ W,
-                 const int32_t *__restrict__ active, int n, long long d, T *__restrict__ M_parent, int shift) {
-    const int i = blockIdx.y;
+                 const int32_t *__restrict__ active, int y0, int n, long long d, T *__restrict__ M_parent, int shift) {
+    const int i = y0 + (int)blockIdx.y;
     if (active && __ldg(&active[i]) == 0) return;
     const long long col = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * V;
     if (col >= d) return;
@@ -1202,8 +1201,8 @@ cr_residual_kernel(const float *__restrict__ X, const float *__restrict__ y, con
 template <int V>
 __global__ void __launch_bounds__(128)
 cr_xt_r_kernel(const float *__restrict__ X, const int32_t *__restrict__ part, const int32_t *__restrict__ order,
-               const float *__restrict__ resid, int rows, long long d, float *__restrict__ G) {
-    const long long item = order ? (long long)__ldg(&order[blockIdx.y]) : (long long)blockIdx.y;
+               const float *__restrict__ resid, int y0, int rows, long long d, float *__restrict__ G) {
+    const long long item = order ? (long long)__ldg(&order[y0 + blockIdx.y]) : (long long)y0 + blockIdx.y;
     const long long col = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * V;
     if (col >= d) return;
     const int p = __ldg(&part[item]);
@@ -1472,6 +1471,9 @@ cudaError_t launch_wait_selftest(int *status, unsigned long long limit_ns, cudaS
     if (err == cudaSuccess) ++*launches;
     return err;
 }
+
+// Most rows of blocks in a grid: launches over more items (nodes, parents, slot items) go in chunks.
+constexpr int kMaxGridY = 65535;
 
 static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -1890,10 +1892,14 @@ template <typename T, int V>
 static cudaError_t run_encode(const void *G, const void *coeff, const int32_t *nodes, int count, int m, int64_t d,
                               void *E, cudaStream_t stream) {
     const long long threads = (d + V - 1) / V;
-    dim3 grid((unsigned)((threads + 255) / 256), (unsigned)count);
-    cr_encode_kernel<T, V><<<grid, 256, 0, stream>>>(reinterpret_cast<const T *>(G), reinterpret_cast<const T *>(coeff),
-                                                     nodes, m, d, reinterpret_cast<T *>(E));
-    return cudaGetLastError();
+    for (int y0 = 0; y0 < count; y0 += kMaxGridY) {
+        dim3 grid((unsigned)((threads + 255) / 256), (unsigned)std::min(kMaxGridY, count - y0));
+        cr_encode_kernel<T, V><<<grid, 256, 0, stream>>>(reinterpret_cast<const T *>(G), reinterpret_cast<const T *>(coeff),
+                                                         nodes, y0, m, d, reinterpret_cast<T *>(E));
+        const cudaError_t err = cudaGetLastError();
+        if (err != cudaSuccess) return err;
+    }
+    return cudaSuccess;
 }
 
 cudaError_t launch_encode(const void *G, const void *coeff, const int32_t *nodes, int count, int m, int64_t d,
@@ -1913,12 +1919,16 @@ template <typename T, int V>
 static cudaError_t run_decode(const void *M_child, const void *E_parent, const void *W, const int32_t *active,
                               int parents, int n, int64_t d, void *M_parent, int shift, cudaStream_t stream) {
     const long long threads = (d + V - 1) / V;
-    dim3 grid((unsigned)((threads + 255) / 256), (unsigned)parents);
-    cr_decode_kernel<T, V><<<grid, 256, 0, stream>>>(reinterpret_cast<const T *>(M_child),
-                                                     reinterpret_cast<const T *>(E_parent),
-                                                     reinterpret_cast<const T *>(W), active, n, d,
-                                                     reinterpret_cast<T *>(M_parent), shift);
-    return cudaGetLastError();
+    for (int y0 = 0; y0 < parents; y0 += kMaxGridY) {
+        dim3 grid((unsigned)((threads + 255) / 256), (unsigned)std::min(kMaxGridY, parents - y0));
+        cr_decode_kernel<T, V><<<grid, 256, 0, stream>>>(reinterpret_cast<const T *>(M_child),
+                                                         reinterpret_cast<const T *>(E_parent),
+                                                         reinterpret_cast<const T *>(W), active, y0, n, d,
+                                                         reinterpret_cast<T *>(M_parent), shift);
+        const cudaError_t err = cudaGetLastError();
+        if (err != cudaSuccess) return err;
+    }
+    return cudaSuccess;
 }
 
 cudaError_t launch_decode(const void *M_child, const void *E_parent, const void *W, const int32_t *active,
@@ -1946,15 +1956,18 @@ cudaError_t launch_partial_gradients_two_pass(const float *X, const float *y, co
     cudaError_t err = cudaGetLastError();
     if (err != cudaSuccess) return err;
     ++*launches;
-    if (v4) {
-        dim3 grid((unsigned)((d / 4 + 127) / 128), (unsigned)items);
-        cr_xt_r_kernel<4><<<grid, 128, 0, stream>>>(X, part, order, resid, rows, d, G);
-    } else {
-        dim3 grid((unsigned)((d + 127) / 128), (unsigned)items);
-        cr_xt_r_kernel<1><<<grid, 128, 0, stream>>>(X, part, order, resid, rows, d, G);
+    for (int y0 = 0; y0 < items && err == cudaSuccess; y0 += kMaxGridY) {
+        const unsigned gy = (unsigned)std::min(kMaxGridY, items - y0);
+        if (v4) {
+            dim3 grid((unsigned)((d / 4 + 127) / 128), gy);
+            cr_xt_r_kernel<4><<<grid, 128, 0, stream>>>(X, part, order, resid, y0, rows, d, G);
+        } else {
+            dim3 grid((unsigned)((d + 127) / 128), gy);
+            cr_xt_r_kernel<1><<<grid, 128, 0, stream>>>(X, part, order, resid, y0, rows, d, G);
+        }
+        err = cudaGetLastError();
+        if (err == cudaSuccess) ++*launches;
     }
-    err = cudaGetLastError();
-    if (err == cudaSuccess) ++*launches;
     return err;
 }
 

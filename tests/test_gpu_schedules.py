@@ -244,3 +244,44 @@ def test_a_wait_that_runs_out_sets_the_status_and_harms_nothing():
         assert rel_l2(out[2].cpu().numpy(), O.execute(code, local, G, masks[2])) <= REL_L2_BAR
     finally:
         B.cr_plan_destroy(plan)
+
+
+# ------------------------------------------------------------------ more items than a grid has rows
+
+def test_more_nodes_than_a_grid_has_rows_of_blocks():
+    """(16,4) tree without redundancy: 69904 nodes, one slot each.  The per-node and per-slot launches
+    (encode, partial gradients) then exceed the 65535 rows of blocks of a grid and go in chunks."""
+    n, L, s, d, rows = 16, 4, 0, 8, 2
+    P = O.partition_quantum(n, L, s)
+    assert P == 69904
+    cfg = tree(n, L, s, "cyclic", d)
+    plan = make_plan(cfg)
+    try:
+        code, local = check_slot_table(plan, cfg)
+        N, m = B.cr_plan_num_nodes(plan), B.cr_plan_load(plan)
+        assert N == 69904 and m == 1
+        X, y, _ = inputs.linreg_partitions(P, rows, d, seed=61)
+        w = inputs.model_vector(d, seed=62)
+        G_slots = torch.full((N, m, d), float("nan"), device="cuda")
+        ws = torch.empty(B.cr_partial_gradients_workspace_bytes(plan, rows), dtype=torch.uint8, device="cuda")
+        B.cr_partial_gradients(plan, torch.from_numpy(X).cuda(), torch.from_numpy(y).cuda(), rows, torch.from_numpy(w).cuda(), G_slots, ws)
+        torch.cuda.synchronize()
+        G_parts = np.stack([O.partial_gradient_linreg(X[p], y[p], w) for p in range(P)])
+        part = B.slot_partitions(plan)
+        got = G_slots.cpu().numpy()
+        for v in (0, 1, 65534, 65535, 65536, N - 1):
+            assert rel_l2(got[v, 0], G_parts[part[v, 0]]) <= REL_L2_BAR
+        assert np.isfinite(got).all()
+        masks = np.zeros((1, B.cr_plan_num_groups(plan)), dtype=np.uint32)
+        want = G_parts.sum(0)                                   # s = 0: the plain tree sum
+        flags = B.CR_AGG_UNFUSED | B.CR_AGG_ALL_NODES
+        wsu = torch.empty(B.cr_aggregate_workspace_bytes(plan, 1, flags), dtype=torch.uint8, device="cuda")
+        out = torch.zeros((1, d), device="cuda")
+        B.cr_aggregate(plan, G_slots, masks, out, flags, wsu)
+        torch.cuda.synchronize()
+        assert rel_l2(out[0].cpu().numpy(), want) <= REL_L2_BAR
+        B.cr_aggregate(plan, G_slots, masks, out, B.CR_AGG_FUSED)
+        torch.cuda.synchronize()
+        assert rel_l2(out[0].cpu().numpy(), want) <= REL_L2_BAR
+    finally:
+        B.cr_plan_destroy(plan)
