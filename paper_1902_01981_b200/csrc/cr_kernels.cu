@@ -1265,24 +1265,32 @@ struct PgArgs {
     unsigned long long wait_ns;  // bound of every wait, in nanoseconds
 };
 
-// RG = rows handled together in pass A (1, 2 or 4; at most the rows of a block).  GENERAL = false is the
-// case of one slot per item without slot coefficient, kept free of the bookkeeping of the general one
-// (measured: 5 % faster on 2048 x 4096 partitions).
-template <int KPT, int RG, bool GENERAL, bool LOGISTIC>
+// Rows of a block: as many as a thread can keep in registers (its KPT column groups of each row).
+__host__ __device__ constexpr int pg_block_rows(int kpt) { return 12 / kpt > 0 ? 12 / kpt : 1; }
+
+// GENERAL = false is the case of one slot per item without slot coefficient, kept free of the bookkeeping of
+// the general one (measured: 5 % faster on 2048 x 4096 partitions).
+// Per block a thread reads its share of every row from shared memory ONCE, into registers: the same
+// values serve the residuals (pass A) and, once the residuals are known, the gradient update (pass B).
+// Every thread then folds the eight per-warp partial sums of each row itself, so one CTA-wide barrier
+// per block is all the synchronisation there is -- it also tells that everybody has read the buffer, so
+// the copy of block blk + S goes into it at once.  (The first version read X from shared memory in both
+// passes and took three barriers per block: shared-memory wavefronts 48 %, DRAM 48 % of peak.)
+template <int KPT, bool GENERAL, bool LOGISTIC>
 __global__ void __launch_bounds__(256, 2)
 cr_partial_fused_kernel(const PgArgs a) {
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
+    constexpr int RBC = pg_block_rows(KPT);
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const long long d = a.d;
-    const int RB = a.RB, S = a.stages;
+    const int RB = a.RB, S = a.stages;   // RB <= RBC
     const size_t stage_elems = (size_t)RB * d;
     float *ring = reinterpret_cast<float *>(smem_raw);
     float *gpart = ring + (size_t)S * stage_elems;          // [d] this CTA's partial gradient
-    float *red = gpart + d;                                 // [RB][8] per-warp partial residuals
-    float *rfin = red + (size_t)RB * 8;                     // [RB] residuals of the block
-    uint64_t *full = reinterpret_cast<uint64_t *>(rfin + ((RB + 3) & ~3));
+    float *red = gpart + d;                                 // [2][RBC][8] per-warp partial residuals, double buffered
+    uint64_t *full = reinterpret_cast<uint64_t *>(red + 2 * RBC * 8);
     volatile int *flags = reinterpret_cast<volatile int *>(full + S);
 
     if (tid == 0) {
@@ -1305,7 +1313,7 @@ cr_partial_fused_kernel(const PgArgs a) {
     const int nblocks = min(total_blocks, b0 + per_cta) - b0;
     // Position in the list, kept incrementally (no division and no dependent load per block): slot
     // within the item, block within the slot, the slot's partition; one copy for the thread that
-    // issues the copies (it runs S - 1 blocks ahead), one for the consumers.
+    // issues the copies (it runs S blocks ahead), one for the consumers.
     const int slot0 = b0 / bps;
     int i_slot = slot0, i_bi = b0 - slot0 * bps, c_slot = slot0, c_bi = i_bi;
     int i_p = 0, c_p = 0;
@@ -1338,13 +1346,15 @@ cr_partial_fused_kernel(const PgArgs a) {
         }
     };
     if (tid == 0)
-        for (; issued < nblocks && issued < S - 1; ++issued) issue(issued);
+        for (; issued < nblocks && issued < S; ++issued) issue(issued);
 
     int done = 0;
     for (int blk = 0; blk < nblocks; ++blk) {
         const int nr = min(RB, a.rows - c_bi * RB);
-        // label of this thread's row, fetched before the wait so that its latency hides behind it
-        const float yv = tid < nr ? __ldg(a.y + (size_t)c_p * a.rows + (size_t)c_bi * RB + tid) : 0.f;
+        // labels of the block's rows, fetched before the wait so that their latency hides behind it
+        float yv[RBC];
+#pragma unroll
+        for (int r = 0; r < RBC; ++r) yv[r] = r < nr ? __ldg(a.y + (size_t)c_p * a.rows + (size_t)c_bi * RB + r) : 0.f;
         const float scale = c_scale;
         ++c_bi;
         if (GENERAL && c_bi == bps) {     // the next block opens the next slot of the item
@@ -1354,58 +1364,49 @@ cr_partial_fused_kernel(const PgArgs a) {
                 if (a.coeff) c_scale = __ldg(&a.coeff[item * spi + c_slot]);
             }
         }
-        // all threads have left the previous block once this barrier is passed, so its buffer is free
-        const int ok = __syncthreads_and(mbar_wait(&full[blk % S], (uint32_t)((blk / S) & 1), &flags[1], a.wait_ns) ? 1 : 0);
-        if (!ok) break;
+        const int ok = mbar_wait(&full[blk % S], (uint32_t)((blk / S) & 1), &flags[1], a.wait_ns) ? 1 : 0;
+        const float *Xb = ring + (size_t)(blk % S) * stage_elems;
+        // this thread's share of the block, read once; pass A: partial residuals
+        float4 xf[RBC][KPT];
+        float part[RBC];
+#pragma unroll
+        for (int r = 0; r < RBC; ++r) {
+            part[r] = 0.f;
+#pragma unroll
+            for (int k = 0; k < KPT; ++k) {
+                const long long col = 4ll * tid + 1024ll * k;
+                xf[r][k] = (r < nr && col < d) ? *reinterpret_cast<const float4 *>(Xb + (size_t)r * d + col)
+                                               : make_float4(0.f, 0.f, 0.f, 0.f);
+                part[r] += xf[r][k].x * wv[k].x + xf[r][k].y * wv[k].y + xf[r][k].z * wv[k].z + xf[r][k].w * wv[k].w;
+            }
+        }
+        float *redb = red + (blk & 1) * (RBC * 8);
+#pragma unroll
+        for (int r = 0; r < RBC; ++r) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) part[r] += __shfl_xor_sync(0xffffffffu, part[r], o);
+            if (lane == 0) redb[r * 8 + warp] = part[r];
+        }
+        // the one barrier of the block: the partial sums are visible, and everybody has read the buffer
+        if (!__syncthreads_and(ok)) break;
         if (tid == 0 && issued < nblocks) {
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             issue(issued);
             ++issued;
         }
-        const float *Xb = ring + (size_t)(blk % S) * stage_elems;
-        // pass A: residual partials, RG rows at a time
-        for (int rg = 0; rg < nr; rg += RG) {
-            float part[RG];
+        // pass B from the registers: acc += r[row] * X_b[row, cols]
 #pragma unroll
-            for (int i = 0; i < RG; ++i) part[i] = 0.f;
+        for (int r = 0; r < RBC; ++r) {
+            if (r < nr) {
+                const float4 p0 = *reinterpret_cast<const float4 *>(redb + r * 8);
+                const float4 p1 = *reinterpret_cast<const float4 *>(redb + r * 8 + 4);
+                float z = ((p0.x + p0.y) + (p0.z + p0.w)) + ((p1.x + p1.y) + (p1.z + p1.w));
+                if (LOGISTIC) z = 1.f / (1.f + expf(-z));
+                const float rr = GENERAL ? scale * (z - yv[r]) : z - yv[r];
 #pragma unroll
-            for (int k = 0; k < KPT; ++k) {
-                const long long col = 4ll * tid + 1024ll * k;
-                if (col < d) {
-#pragma unroll
-                    for (int i = 0; i < RG; ++i) {
-                        if (rg + i < nr) {
-                            const float4 x = *reinterpret_cast<const float4 *>(Xb + (size_t)(rg + i) * d + col);
-                            part[i] += x.x * wv[k].x + x.y * wv[k].y + x.z * wv[k].z + x.w * wv[k].w;
-                        }
-                    }
-                }
-            }
-#pragma unroll
-            for (int i = 0; i < RG; ++i) {
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) part[i] += __shfl_xor_sync(0xffffffffu, part[i], o);
-                if (lane == 0 && rg + i < nr) red[(rg + i) * 8 + warp] = part[i];
-            }
-        }
-        __syncthreads();
-        if (tid < nr) {
-            float z = 0.f;
-#pragma unroll
-            for (int w8 = 0; w8 < 8; ++w8) z += red[tid * 8 + w8];
-            if (LOGISTIC) z = 1.f / (1.f + expf(-z));
-            rfin[tid] = GENERAL ? scale * (z - yv) : z - yv;
-        }
-        __syncthreads();
-        // pass B: acc += r[row] * X_b[row, cols]
-        for (int row = 0; row < nr; ++row) {
-            const float r = rfin[row];
-#pragma unroll
-            for (int k = 0; k < KPT; ++k) {
-                const long long col = 4ll * tid + 1024ll * k;
-                if (col < d) {
-                    const float4 x = *reinterpret_cast<const float4 *>(Xb + (size_t)row * d + col);
-                    acc[k].x += r * x.x; acc[k].y += r * x.y; acc[k].z += r * x.z; acc[k].w += r * x.w;
+                for (int k = 0; k < KPT; ++k) {
+                    acc[k].x += rr * xf[r][k].x; acc[k].y += rr * xf[r][k].y;
+                    acc[k].z += rr * xf[r][k].z; acc[k].w += rr * xf[r][k].w;
                 }
             }
         }
@@ -1971,12 +1972,12 @@ cudaError_t launch_partial_gradients_two_pass(const float *X, const float *y, co
     return err;
 }
 
-template <int KPT, int RG>
-static cudaError_t run_partial_fused_rg(const PgArgs &pa, int csplit, bool fit_one_wave, int items, size_t smem,
-                                        cudaStream_t stream) {
+template <int KPT>
+static cudaError_t run_partial_fused(const PgArgs &pa, int csplit, bool fit_one_wave, int items, size_t smem,
+                                     cudaStream_t stream) {
     const bool general = pa.slots_per_item != 1 || pa.coeff != nullptr;
-    auto kern = general ? (pa.loss == 1 ? cr_partial_fused_kernel<KPT, RG, true, true> : cr_partial_fused_kernel<KPT, RG, true, false>)
-                        : (pa.loss == 1 ? cr_partial_fused_kernel<KPT, RG, false, true> : cr_partial_fused_kernel<KPT, RG, false, false>);
+    auto kern = general ? (pa.loss == 1 ? cr_partial_fused_kernel<KPT, true, true> : cr_partial_fused_kernel<KPT, true, false>)
+                        : (pa.loss == 1 ? cr_partial_fused_kernel<KPT, false, true> : cr_partial_fused_kernel<KPT, false, false>);
     cudaError_t err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (err != cudaSuccess) return err;
     if (csplit > 8) {
@@ -2026,14 +2027,6 @@ static cudaError_t run_partial_fused_rg(const PgArgs &pa, int csplit, bool fit_o
     return cudaLaunchKernelEx(&cfg, kern, pa);
 }
 
-template <int KPT>
-static cudaError_t run_partial_fused(const PgArgs &pa, int csplit, bool fit_one_wave, int items, size_t smem,
-                                     cudaStream_t stream) {
-    if (pa.RB >= 4) return run_partial_fused_rg<KPT, 4>(pa, csplit, fit_one_wave, items, smem, stream);
-    if (pa.RB >= 2) return run_partial_fused_rg<KPT, 2>(pa, csplit, fit_one_wave, items, smem, stream);
-    return run_partial_fused_rg<KPT, 1>(pa, csplit, fit_one_wave, items, smem, stream);
-}
-
 bool partial_fused_eligible(const float *X, const float *w, const float *G, int64_t d, int items) {
     return d % 4 == 0 && d <= 8192 && aligned16(X) && aligned16(w) && aligned16(G) && items <= 65535;
 }
@@ -2051,7 +2044,10 @@ cudaError_t launch_partial_gradients_fused(const float *X, const float *y, const
     const int stages = tune.pg_stages ? tune.pg_stages : 2;
     int64_t rb = tune.pg_block_kb ? ((int64_t)tune.pg_block_kb * 1024) / (d * 4)
                                   : ((int64_t)per_cta - d * 4 - 512) / ((int64_t)stages * d * 4);
-    const int RB = (int)std::max<int64_t>(1, std::min<int64_t>(32, rb));
+    // ... and no more rows than a thread keeps in registers
+    const int kpt = d <= 1024 ? 1 : (d <= 2048 ? 2 : (d <= 4096 ? 4 : (int)((d + 1023) / 1024)));   // as the instances below
+    const int rbc = pg_block_rows(kpt);
+    const int RB = (int)std::max<int64_t>(1, std::min<int64_t>(rbc, rb));
     // the row blocks of one item are split over a cluster of up to 8 CTAs, each with at least 4 blocks
     const int item_blocks = slots_per_item * ((rows + RB - 1) / RB);
     int csplit = 1;
@@ -2067,8 +2063,7 @@ cudaError_t launch_partial_gradients_fused(const float *X, const float *y, const
     // few items (coded gradients of a small tree): a cluster of 16 fills more of the GPU
     if (csplit == 8 && items * 8 < 2 * dev.sm_count && item_blocks / 16 >= 4) csplit = 16;
     if (tune.pg_cluster) csplit = tune.pg_cluster;
-    const size_t smem = (size_t)stages * RB * d * 4 + (size_t)d * 4 + (size_t)RB * 8 * 4 + (size_t)((RB + 3) & ~3) * 4 +
-                        (size_t)stages * 8 + 16;
+    const size_t smem = (size_t)stages * RB * d * 4 + (size_t)d * 4 + (size_t)2 * rbc * 8 * 4 + (size_t)stages * 8 + 16;
     if (smem > (size_t)dev.smem_optin) return cudaErrorInvalidConfiguration;
     PgArgs pa;
     pa.X = X; pa.y = y; pa.w = w; pa.part = part; pa.order = slots_per_item == 1 ? order : nullptr; pa.coeff = coeff; pa.G = G; pa.rows = rows;
