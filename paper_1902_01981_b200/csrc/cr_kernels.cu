@@ -917,6 +917,9 @@ __global__ void __launch_bounds__(256, (LMAX <= 2 && PIPE == 5) ? (std::is_float
 cr_fused_ldg_kernel(const T *__restrict__ G, const T *__restrict__ coeff, const Step *__restrict__ steps,
                     const int32_t *__restrict__ pat_off, int m, long long d, T *__restrict__ out, int shift,
                     const __grid_constant__ InlineSchedule inl) {
+    // The split form launches the kernel that adds the sub-trees' rows as a programmatic dependent: it may be
+    // set up while this grid still runs (it waits for this grid's completion before it reads anything).
+    asm volatile("griddepcontrol.launch_dependents;");
     const int b = blockIdx.y;
     const long long col = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * V;
     if (col >= d) return;
@@ -1043,6 +1046,9 @@ template <typename T>
 __global__ void __launch_bounds__(256)
 cr_sum_rows_kernel(const T *__restrict__ rows, int nrows, long long d, T *__restrict__ out, int shift) {
     const long long col = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    // launched as a programmatic dependent of the kernel that writes `rows`: wait until that grid has
+    // completed and its writes are visible (returns at once when there is no such dependency)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (col >= d) return;
     T sum = T(0);
     for (int r = 0; r < nrows; ++r) sum += rows[(size_t)r * d + col];
@@ -1855,9 +1861,19 @@ static cudaError_t run_ldg(const AggArgs &a, cudaStream_t stream, int64_t *launc
     if (err != cudaSuccess) return err;
     ++*launches;
     if (inl.nseg) {
-        cr_sum_rows_kernel<T><<<(unsigned)((a.d + 255) / 256), 256, 0, stream>>>(reinterpret_cast<const T *>(a.split_scratch), inl.nseg,
-                                                                             a.d, reinterpret_cast<T *>(a.out), a.shift);
-        err = cudaGetLastError();
+        // a programmatic dependent launch: the set-up of this small grid overlaps the run of the first one
+        // (two back-to-back launches cost a few microseconds between them, a fifth of these short calls)
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)((a.d + 255) / 256), 1, 1);
+        cfg.blockDim = dim3(256, 1, 1);
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        err = cudaLaunchKernelEx(&cfg, cr_sum_rows_kernel<T>, reinterpret_cast<const T *>(a.split_scratch), inl.nseg,
+                                 (long long)a.d, reinterpret_cast<T *>(a.out), a.shift);
         if (err == cudaSuccess) ++*launches;
     }
     return err;

@@ -15,6 +15,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstdint>
 #include <cstdio>
 
@@ -42,6 +43,9 @@ __device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
 }
 __device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
     uint32_t ok;
@@ -204,6 +208,9 @@ struct TcResidualArgs {
     const int32_t *order;  // [items] or null: launch order of the items (same partition side by side)
     float *Rh, *Rl;        // [items][rows_pad][32]
     float *R_out;          // optional [items][rows][K]
+    int items;
+    int ipt;               // items per 128-row tile: 1, or 128 / sub_rows for partitions of few rows
+    int sub_rows;          // ipt > 1: rows of a tile that one item takes (its rows rounded up to a multiple of 8)
     int rows, rows_pad, K, loss, stages;
     int kchunks;           // ceil(d / 32)
     int *status;
@@ -227,10 +234,14 @@ cr_tc_residual_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_con
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_full + 1);
     volatile int *flags = reinterpret_cast<volatile int *>(tmem_slot + 1);   // [0] someone gave up, [1] never set
 
+    // Partitions of few rows (the paper's logistic run has 39 per partition) would leave most of a 128-row
+    // tile empty and drag the two W tiles through shared memory once per item.  Then `ipt` items share a
+    // tile: item j of the group takes tile rows j * sub_rows .. (its box is sub_rows rows high, rows beyond
+    // the partition are zero-filled by the copy engine), and W is fetched once for all of them.
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int item = a.order ? __ldg(&a.order[blockIdx.y]) : (int)blockIdx.y;
-    const int row0 = blockIdx.x * kTileM;
-    const int p = __ldg(&a.part[item]);
+    const int first = (int)blockIdx.y * a.ipt;                       // first item of this CTA's group (launch order)
+    const int in_group = min(a.ipt, a.items - first);
+    const int row0 = blockIdx.x * kTileM;                            // ipt == 1: tile of the partition's rows
 
     if (tid == 0) {
         for (int s = 0; s < S; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
@@ -249,12 +260,24 @@ cr_tc_residual_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_con
         if (lane == 0) {
             int issued = 0;
             bool ok = true;
+            int parts[kTileM / 8];
+            for (int j = 0; j < in_group; ++j) {
+                const int it = a.order ? __ldg(&a.order[first + j]) : first + j;
+                parts[j] = __ldg(&a.part[it]);
+            }
+            const uint32_t sub_bytes = (uint32_t)a.sub_rows * kBoxCols * 4;
+            const uint32_t x_bytes = a.ipt > 1 ? (uint32_t)in_group * sub_bytes : kXBytes;
             for (int kc = 0; kc < a.kchunks; ++kc) {
                 const int s = kc % S;
                 if (!mbar_wait(&empty[s], (uint32_t)(((kc / S) & 1) ^ 1), &flags[0], a.wait_ns)) { ok = false; break; }
                 unsigned char *st = ring + (size_t)s * kStageBytes;
-                mbar_expect_tx(&full[s], kStageBytes);
-                tma_load_3d(st, &mapX, kc * kBoxCols, row0, p, &full[s]);
+                mbar_expect_tx(&full[s], x_bytes + 2 * kWBytes);
+                if (a.ipt > 1) {
+                    for (int j = 0; j < in_group; ++j)
+                        tma_load_3d(st + (size_t)j * sub_bytes, &mapX, kc * kBoxCols, 0, parts[j], &full[s]);
+                } else {
+                    tma_load_3d(st, &mapX, kc * kBoxCols, row0, parts[0], &full[s]);
+                }
                 tma_load_2d(st + kXBytes, &mapWh, kc * kBoxCols, 0, &full[s]);
                 tma_load_2d(st + kXBytes + kWBytes, &mapWl, kc * kBoxCols, 0, &full[s]);
                 ++issued;
@@ -292,14 +315,19 @@ cr_tc_residual_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_con
     } else {
         // epilogue: quarter (warp % 4) of the 128 accumulator lanes, one row per thread
         const int q = warp & 3;
-        const int row = row0 + q * 32 + lane;
-        const float yv = row < a.rows ? __ldg(&a.y[(size_t)p * a.rows + row]) : 0.f;
+        const int trow = q * 32 + lane;                                  // row of the tile
+        const int j = a.ipt > 1 ? trow / a.sub_rows : 0;                 // which item of the group
+        const int row = a.ipt > 1 ? trow - j * a.sub_rows : row0 + trow; // row of that item's partition
+        const bool mine = j < in_group && (a.ipt == 1 || row < a.sub_rows);
+        const int item = mine ? (a.order ? __ldg(&a.order[first + j]) : first + j) : 0;
+        const int p = mine ? __ldg(&a.part[item]) : 0;
+        const float yv = (mine && row < a.rows) ? __ldg(&a.y[(size_t)p * a.rows + row]) : 0.f;
         const bool ok = __all_sync(0xffffffffu, mbar_wait(acc_full, 0, &flags[0], a.wait_ns) ? 1 : 0) != 0;
         if (ok) {
             tc_fence_after();
             float r[kModels];
             tmem_sum_accs(tmem_acc + ((uint32_t)(q * 32) << 16), a.kchunks * (kBoxCols / 8), r);
-            if (row < a.rows_pad) {
+            if (mine && row < a.rows_pad) {
                 float4 *dh = reinterpret_cast<float4 *>(a.Rh + ((size_t)item * a.rows_pad + row) * kModels);
                 float4 *dl = reinterpret_cast<float4 *>(a.Rl + ((size_t)item * a.rows_pad + row) * kModels);
 #pragma unroll
@@ -458,6 +486,129 @@ cr_tc_gradient_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_con
     if (warp == 1) tmem_free(tmem_acc, kTmemCols);
 }
 
+// The same contraction for partitions of at most kRowsB rows, where the kernel above would be one small MMA
+// group between a launch, a tensor-memory allocation and an epilogue per (column tile, item).  Here a CTA
+// keeps an item: its residual tiles are fetched once, the column tiles stream through a ring of X stages,
+// and two sets of accumulators alternate so that the epilogue of one tile runs under the MMAs of the next.
+// grid (CTAs per item, items), 192 threads, same roles; all 512 columns of tensor memory (one CTA per SM).
+__global__ void __launch_bounds__(192, 1)
+cr_tc_gradient_short_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapRh,
+                            const __grid_constant__ CUtensorMap mapRl, const TcGradientArgs a) {
+    using namespace tc;
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    constexpr uint32_t kBoxBytes = kRowsB * kBoxCols * 4;          // 8 KB: kRowsB rows of 128 bytes
+    constexpr uint32_t kXBytes = (kTileM / kBoxCols) * kBoxBytes;  // 32 KB: one column tile
+    constexpr uint32_t kSetCols = kAccs * kModels;                 // accumulator columns of one set
+    const int S = a.stages;
+    unsigned char *ring = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    unsigned char *rtile = ring + (size_t)S * kXBytes;             // residuals: head then tail, 8 KB each
+    uint64_t *full = reinterpret_cast<uint64_t *>(rtile + 2 * kBoxBytes);
+    uint64_t *empty = full + S;
+    uint64_t *r_full = empty + S;
+    uint64_t *acc_full = r_full + 1;     // [2]
+    uint64_t *acc_empty = acc_full + 2;  // [2]
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(acc_empty + 2);
+    volatile int *flags = reinterpret_cast<volatile int *>(tmem_slot + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int item = a.order ? __ldg(&a.order[blockIdx.y]) : (int)blockIdx.y;
+    const int p = __ldg(&a.part[item]);
+    const int ntiles = (int)((a.d + kTileM - 1) / kTileM);
+    const int my_tiles = (int)blockIdx.x < ntiles ? (ntiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+    const int ksteps = (a.rows + 7) / 8;   // <= kRowsB / 8
+
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        mbar_init(r_full, 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(&acc_full[b], 1); mbar_init(&acc_empty[b], 4); }
+        flags[0] = 0; flags[1] = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(tmem_slot, 2 * kSetCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_acc = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int issued = 0;
+            bool ok = true;
+            mbar_expect_tx(r_full, 2 * kBoxBytes);
+            tma_load_3d(rtile, &mapRh, 0, 0, item, r_full);
+            tma_load_3d(rtile + kBoxBytes, &mapRl, 0, 0, item, r_full);
+            for (int i = 0; i < my_tiles; ++i) {
+                const int s = i % S;
+                const int col0 = ((int)blockIdx.x + i * (int)gridDim.x) * kTileM;
+                if (!mbar_wait(&empty[s], (uint32_t)(((i / S) & 1) ^ 1), &flags[0], a.wait_ns)) { ok = false; break; }
+                unsigned char *st = ring + (size_t)s * kXBytes;
+                mbar_expect_tx(&full[s], kXBytes);
+#pragma unroll
+                for (int b = 0; b < kTileM / kBoxCols; ++b)
+                    tma_load_3d(st + b * kBoxBytes, &mapX, col0 + b * kBoxCols, 0, p, &full[s]);
+                ++issued;
+            }
+            if (!ok) {
+                flags[0] = 1;
+                atomicExch(a.status, 1);
+                mbar_wait(r_full, 0, &flags[1], a.wait_ns);
+                for (int i = issued > S ? issued - S : 0; i < issued; ++i)
+                    mbar_wait(&full[i % S], (uint32_t)((i / S) & 1), &flags[1], a.wait_ns);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = instr_desc_tf32(kTileM, kModels, 1, 1);
+            bool ok = mbar_wait(r_full, 0, &flags[0], a.wait_ns);
+            for (int i = 0; i < my_tiles && ok; ++i) {
+                const int s = i % S, set = i & 1;
+                if (!mbar_wait(&full[s], (uint32_t)((i / S) & 1), &flags[0], a.wait_ns)) { ok = false; break; }
+                // the accumulator set must have been read by the epilogue of the tile before last
+                if (!mbar_wait(&acc_empty[set], (uint32_t)(((i >> 1) & 1) ^ 1), &flags[0], a.wait_ns)) { ok = false; break; }
+                tc_fence_after();
+                const unsigned char *st = ring + (size_t)s * kXBytes;
+                const uint32_t acc0 = tmem_acc + (uint32_t)set * kSetCols;
+                for (int ks = 0; ks < ksteps; ++ks) {
+                    const uint64_t da = smem_desc(st + ks * 1024, kBoxBytes, 512, kLayoutSw128Base32);
+                    const uint64_t dh = smem_desc(rtile + ks * 1024, kBoxBytes, 512, kLayoutSw128Base32);
+                    const uint64_t dl = smem_desc(rtile + kBoxBytes + ks * 1024, kBoxBytes, 512, kLayoutSw128Base32);
+                    mma_tf32(acc0 + (uint32_t)((ks % kHeadAccs) * kModels), da, dh, idesc, ks >= kHeadAccs ? 1u : 0u);
+                    mma_tf32(acc0 + (uint32_t)(kHeadAccs * kModels), da, dl, idesc, ks > 0 ? 1u : 0u);
+                }
+                mma_commit(&empty[s]);          // the X stage may be refilled once these MMAs have read it
+                mma_commit(&acc_full[set]);     // and the epilogue may read the set
+            }
+            if (!ok) { flags[0] = 1; atomicExch(a.status, 1); }
+        }
+    } else {
+        const int q = warp & 3;
+        bool ok = true;
+        for (int i = 0; i < my_tiles; ++i) {
+            const int set = i & 1;
+            const long long col = (long long)((int)blockIdx.x + i * (int)gridDim.x) * kTileM + q * 32 + lane;
+            ok = __all_sync(0xffffffffu, mbar_wait(&acc_full[set], (uint32_t)((i >> 1) & 1), &flags[0], a.wait_ns) ? 1 : 0) != 0;
+            if (!ok) break;
+            tc_fence_after();
+            float r[kModels];
+            tmem_sum_accs(tmem_acc + (uint32_t)set * kSetCols + ((uint32_t)(q * 32) << 16), ksteps, r);
+            // the set is in registers: hand it back before the stores
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_empty[set]);
+            if (col < a.d) {
+#pragma unroll
+                for (int k = 0; k < kModels; ++k)
+                    if (k < a.K) a.G[((size_t)k * a.items + item) * a.d + col] = r[k];
+            }
+        }
+        if (!ok && lane == 0) { flags[0] = 1; atomicExch(a.status, 1); }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_free(tmem_acc, 2 * kSetCols);
+}
+
 // ------------------------------------------------------------------------------------------------
 // host side
 // ------------------------------------------------------------------------------------------------
@@ -488,6 +639,11 @@ cudaError_t launch_partial_gradients_multi(const float *X, const float *y, const
                                            cudaStream_t stream, int64_t *launches) {
     using namespace tc;
     const int rows_pad = (rows + kTileM - 1) / kTileM * kTileM;
+    // partitions of at most kRowsB rows: several items share a 128-row tile of the residual kernel, and the
+    // gradient kernel keeps an item per CTA (see the kernels)
+    const bool few_rows = rows <= kRowsB;
+    const int sub_rows = (rows + 7) / 8 * 8;
+    const int ipt = few_rows ? kTileM / sub_rows : 1;
     float *Wh = reinterpret_cast<float *>(workspace);
     float *Wl = Wh + (size_t)kModels * d;
     float *Rh = Wl + (size_t)kModels * d;
@@ -505,7 +661,7 @@ cudaError_t launch_partial_gradients_multi(const float *X, const float *y, const
     {
         const cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)rows, (cuuint64_t)P};
         const cuuint64_t strides[2] = {(cuuint64_t)d * 4, (cuuint64_t)rows * (cuuint64_t)d * 4};
-        const cuuint32_t boxA[3] = {kBoxCols, kTileM, 1};
+        const cuuint32_t boxA[3] = {kBoxCols, (cuuint32_t)(ipt > 1 ? sub_rows : kTileM), 1};
         const cuuint32_t boxB[3] = {kBoxCols, kRowsB, 1};
         if (encode_sw128(encode, &mapX, X, 3, dims, strides, boxA, CU_TENSOR_MAP_SWIZZLE_128B) != CUDA_SUCCESS) return cudaErrorInvalidValue;
         if (encode_sw128(encode, &mapXg, X, 3, dims, strides, boxB, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B) != CUDA_SUCCESS) return cudaErrorInvalidValue;
@@ -528,11 +684,13 @@ cudaError_t launch_partial_gradients_multi(const float *X, const float *y, const
     {   // residuals
         TcResidualArgs ra;
         ra.y = y; ra.part = part; ra.order = order; ra.Rh = Rh; ra.Rl = Rl; ra.R_out = R_out; ra.rows = rows; ra.rows_pad = rows_pad;
+        ra.items = items; ra.ipt = ipt; ra.sub_rows = sub_rows;
         ra.K = K; ra.loss = loss; ra.stages = 4; ra.kchunks = (int)((d + kBoxCols - 1) / kBoxCols); ra.status = status; ra.wait_ns = tune.wait_limit_ns;
         const size_t smem = (size_t)ra.stages * (kTileM * kBoxCols * 4 + 2 * kModels * kBoxCols * 4) + (2 * ra.stages + 1) * 8 + 16 + 1024;
         cudaError_t e = cudaFuncSetAttribute(cr_tc_residual_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        cr_tc_residual_kernel<<<dim3((unsigned)(rows_pad / kTileM), (unsigned)items), 192, smem, stream>>>(mapX, mapWh, mapWl, ra);
+        const dim3 grid = ipt > 1 ? dim3(1, (unsigned)((items + ipt - 1) / ipt)) : dim3((unsigned)(rows_pad / kTileM), (unsigned)items);
+        cr_tc_residual_kernel<<<grid, 192, smem, stream>>>(mapX, mapWh, mapWl, ra);
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         ++*launches;
@@ -540,8 +698,27 @@ cudaError_t launch_partial_gradients_multi(const float *X, const float *y, const
     if (G) {   // gradients
         TcGradientArgs ga;
         ga.part = part; ga.order = order; ga.G = G; ga.d = d; ga.rows = rows; ga.K = K; ga.items = items; ga.stages = tune.tc_stages ? tune.tc_stages : 2; ga.status = status; ga.wait_ns = tune.wait_limit_ns;
+        cudaError_t e;
+        if (few_rows) {
+            ga.stages = tune.tc_stages ? tune.tc_stages : 4;
+            const size_t smem = (size_t)ga.stages * (kTileM / kBoxCols) * kRowsB * kBoxCols * 4 + 2 * kRowsB * kBoxCols * 4 +
+                                (2 * ga.stages + 5) * 8 + 16 + 1024;
+            e = cudaFuncSetAttribute(cr_tc_gradient_short_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e != cudaSuccess) return e;
+            // CTAs per item: enough to give every SM about two CTAs, each with several column tiles
+            int dev = 0, sms = 148;
+            if (cudaGetDevice(&dev) == cudaSuccess) (void)cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+            const int ntiles = (int)((d + kTileM - 1) / kTileM);
+            int per_item = (2 * sms + items - 1) / items;
+            per_item = std::max(1, std::min(per_item, (ntiles + 3) / 4));
+            cr_tc_gradient_short_kernel<<<dim3((unsigned)per_item, (unsigned)items), 192, smem, stream>>>(mapXg, mapRh, mapRl, ga);
+            e = cudaGetLastError();
+            if (e != cudaSuccess) return e;
+            ++*launches;
+            return cudaSuccess;
+        }
         const size_t smem = (size_t)ga.stages * ((kTileM / kBoxCols + 2) * kRowsB * kBoxCols * 4) + (2 * ga.stages + 1) * 8 + 16 + 1024;
-        cudaError_t e = cudaFuncSetAttribute(cr_tc_gradient_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        e = cudaFuncSetAttribute(cr_tc_gradient_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         cr_tc_gradient_kernel<<<dim3((unsigned)((d + kTileM - 1) / kTileM), (unsigned)items), 192, smem, stream>>>(mapXg, mapRh, mapRl, ga);
         e = cudaGetLastError();

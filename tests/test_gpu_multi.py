@@ -44,7 +44,13 @@ CASES = [dict(n=3, L=1, s=1, P=6, d=256, code="printed_3_1", rows=64, K=3),     
          dict(n=3, L=2, s=1, P=15, d=36, code="printed_3_1", rows=9, K=1),       # smallest shapes
          dict(n=4, L=2, s=1, P=24, d=5004, code="cyclic", rows=39, K=8),         # shape of the logistic run
          dict(n=4, L=2, s=1, P=48, d=4096, code="cyclic", rows=512, K=16),
-         dict(n=3, L=1, s=1, P=6, d=16384, code="printed_3_1", rows=24, K=2)]     # long contraction over d
+         dict(n=3, L=1, s=1, P=6, d=16384, code="printed_3_1", rows=24, K=2),     # long contraction over d
+         # partitions of few rows: several items share a 128-row tile (five of 24 rows here, 48 items: a ragged
+         # last group), one CTA walks the column tiles of an item
+         dict(n=3, L=2, s=1, P=15, d=300, code="printed_3_1", rows=20, K=5),
+         dict(n=3, L=1, s=1, P=6, d=520, code="printed_3_1", rows=60, K=4),       # eight k-steps: the head accumulators wrap
+         dict(n=12, L=2, s=1, P=168, d=1028, code="cyclic", rows=39, K=32),       # 624 items of 39 rows, three per tile
+         dict(n=3, L=1, s=1, P=6, d=132, code="printed_3_1", rows=65, K=2)]       # just above: the general kernels
 
 
 @pytest.mark.parametrize("loss", [B.CR_LOSS_SQUARED, B.CR_LOSS_LOGISTIC])
