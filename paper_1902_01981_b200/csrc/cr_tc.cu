@@ -490,15 +490,19 @@ cr_tc_gradient_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_con
 // group between a launch, a tensor-memory allocation and an epilogue per (column tile, item).  Here a CTA
 // keeps an item: its residual tiles are fetched once, the column tiles stream through a ring of X stages,
 // and two sets of accumulators alternate so that the epilogue of one tile runs under the MMAs of the next.
-// grid (CTAs per item, items), 192 threads, same roles; all 512 columns of tensor memory (one CTA per SM).
-__global__ void __launch_bounds__(192, 1)
+// With at most eight k-steps the truncation of the tensor core's accumulator is no concern (about 1.5e-8 of
+// the sum per addition), so a set is two accumulators only, head products and tail products: the epilogue
+// reads 64 columns per tile, not 256 (which made it, not the loads, the pace of the first version: 262 us
+// on the logistic shape).  grid (CTAs per item, items), 192 threads, same roles; 128 columns of tensor memory
+// and two X stages, so that two CTAs share an SM.
+__global__ void __launch_bounds__(192, 2)
 cr_tc_gradient_short_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapRh,
                             const __grid_constant__ CUtensorMap mapRl, const TcGradientArgs a) {
     using namespace tc;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     constexpr uint32_t kBoxBytes = kRowsB * kBoxCols * 4;          // 8 KB: kRowsB rows of 128 bytes
     constexpr uint32_t kXBytes = (kTileM / kBoxCols) * kBoxBytes;  // 32 KB: one column tile
-    constexpr uint32_t kSetCols = kAccs * kModels;                 // accumulator columns of one set
+    constexpr uint32_t kSetCols = 2 * kModels;                     // accumulator columns of one set: head, tail
     const int S = a.stages;
     unsigned char *ring = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     unsigned char *rtile = ring + (size_t)S * kXBytes;             // residuals: head then tail, 8 KB each
@@ -573,8 +577,8 @@ cr_tc_gradient_short_kernel(const __grid_constant__ CUtensorMap mapX, const __gr
                     const uint64_t da = smem_desc(st + ks * 1024, kBoxBytes, 512, kLayoutSw128Base32);
                     const uint64_t dh = smem_desc(rtile + ks * 1024, kBoxBytes, 512, kLayoutSw128Base32);
                     const uint64_t dl = smem_desc(rtile + kBoxBytes + ks * 1024, kBoxBytes, 512, kLayoutSw128Base32);
-                    mma_tf32(acc0 + (uint32_t)((ks % kHeadAccs) * kModels), da, dh, idesc, ks >= kHeadAccs ? 1u : 0u);
-                    mma_tf32(acc0 + (uint32_t)(kHeadAccs * kModels), da, dl, idesc, ks > 0 ? 1u : 0u);
+                    mma_tf32(acc0, da, dh, idesc, ks > 0 ? 1u : 0u);
+                    mma_tf32(acc0 + (uint32_t)kModels, da, dl, idesc, ks > 0 ? 1u : 0u);
                 }
                 mma_commit(&empty[s]);          // the X stage may be refilled once these MMAs have read it
                 mma_commit(&acc_full[set]);     // and the epilogue may read the set
@@ -591,7 +595,14 @@ cr_tc_gradient_short_kernel(const __grid_constant__ CUtensorMap mapX, const __gr
             if (!ok) break;
             tc_fence_after();
             float r[kModels];
-            tmem_sum_accs(tmem_acc + (uint32_t)set * kSetCols + ((uint32_t)(q * 32) << 16), ksteps, r);
+            {
+                uint32_t h[32], t[32];
+                const uint32_t lane_base = tmem_acc + (uint32_t)set * kSetCols + ((uint32_t)(q * 32) << 16);
+                tmem_load_32(lane_base, h);
+                tmem_load_32(lane_base + (uint32_t)kModels, t);
+#pragma unroll
+                for (int k = 0; k < kModels; ++k) r[k] = __uint_as_float(h[k]) + __uint_as_float(t[k]);
+            }
             // the set is in registers: hand it back before the stores
             tc_fence_before();
             __syncwarp();
@@ -700,7 +711,7 @@ cudaError_t launch_partial_gradients_multi(const float *X, const float *y, const
         ga.part = part; ga.order = order; ga.G = G; ga.d = d; ga.rows = rows; ga.K = K; ga.items = items; ga.stages = tune.tc_stages ? tune.tc_stages : 2; ga.status = status; ga.wait_ns = tune.wait_limit_ns;
         cudaError_t e;
         if (few_rows) {
-            ga.stages = tune.tc_stages ? tune.tc_stages : 4;
+            ga.stages = tune.tc_stages ? tune.tc_stages : 2;
             const size_t smem = (size_t)ga.stages * (kTileM / kBoxCols) * kRowsB * kBoxCols * 4 + 2 * kRowsB * kBoxCols * 4 +
                                 (2 * ga.stages + 5) * 8 + 16 + 1024;
             e = cudaFuncSetAttribute(cr_tc_gradient_short_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
