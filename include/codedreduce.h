@@ -334,6 +334,15 @@ cr_status_t cr_plan_tune(cr_plan_t *plan, int32_t consumer_warps, int32_t stages
  * shared memory, 0 = built-in choice (two when they fit beside tall boxes), 1 or 2; one buffer leaves
  * room for more and deeper loader rings (cr_plan_tune). */
 cr_status_t cr_plan_tune_batch(cr_plan_t *plan, int32_t share_messages, int32_t e_buffers);
+/* Host work only (also on host-only plans): what the expansion of `batch` patterns (masks_host
+ * [batch][num_groups]) amounts to under the sharing rule `share_messages` (as above).  stats[0] = entries of the
+ * patterns' schedules (consumed nodes, summed over the batch), [1] = nodes in the union, [2] = nodes of layer L-1
+ * whose messages are shared (0: the batch does not share), [3] = distinct message variants over those nodes
+ * (a variant = a distinct decode row over the node's children in the union), [4] = entries of the reduced
+ * schedules (a consumed node of layer L-1 counts once, its leaves not at all), [5] = rows of a buffer of coded
+ * gradients in the batch kernel (the union, plus variants that found no dead row to reuse). */
+cr_status_t cr_plan_batch_stats(const cr_plan_t *plan, const uint32_t *masks_host, int32_t batch, int32_t share_messages,
+                                int64_t *stats);
 
 /* Launch shape of the one-pass partial-gradient kernel; 0 keeps the built-in choice for that field.
  * block_kb = KB of X per staged row block (1..128), stages = row-block buffers per CTA (2..8),

@@ -66,6 +66,7 @@ _SIGNATURES = {
     "cr_plan_set_wait_limit": (C.c_int, [C.c_void_p, C.c_uint64]),
     "cr_selftest_wait": (C.c_int, [C.c_void_p, C.c_uint64, C.c_void_p]),
     "cr_plan_tune_batch": (C.c_int, [C.c_void_p, C.c_int32, C.c_int32]),
+    "cr_plan_batch_stats": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]),
     "cr_schedule_create": (C.c_int, [C.c_void_p, C.c_void_p, C.c_int32, C.c_uint32, C.POINTER(C.c_void_p)]),
     "cr_schedule_destroy": (C.c_int, [C.c_void_p]),
     "cr_schedule_bytes": (C.c_int, [C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_int32)]),
@@ -273,6 +274,14 @@ def cr_selftest_wait(plan: int, limit_ns: int, stream=None) -> None:
 
 def cr_plan_tune_batch(plan: int, share_messages: int = 0, e_buffers: int = 0) -> None:
     _check(lib().cr_plan_tune_batch(plan, share_messages, e_buffers), "cr_plan_tune_batch")
+
+
+def cr_plan_batch_stats(plan: int, masks, share_messages: int = 0) -> dict:
+    """Host-side figures of the expansion of a batch (see codedreduce.h)."""
+    mk = _masks(masks, cr_plan_num_groups(plan))
+    st = np.zeros(6, dtype=np.int64)
+    _check(lib().cr_plan_batch_stats(plan, mk.ctypes.data, mk.shape[0], share_messages, st.ctypes.data), "cr_plan_batch_stats")
+    return dict(zip(("entries", "union", "shared_nodes", "variants", "reduced_entries", "rows"), (int(x) for x in st)))
 
 
 def cr_plan_tune(plan: int, consumer_warps: int = 0, stages: int = 0, ctas_per_sm: int = 0,

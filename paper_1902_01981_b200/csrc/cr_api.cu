@@ -523,6 +523,24 @@ cr_status_t cr_selftest_wait(cr_plan_t *plan, uint64_t limit_ns, void *stream) {
     return CR_OK;
 }
 
+cr_status_t cr_plan_batch_stats(const cr_plan_t *plan, const uint32_t *masks_host, int32_t batch, int32_t share_messages,
+                                int64_t *stats) {
+    if (!plan || !masks_host || !stats || batch < 1 || batch > (1 << 16) || share_messages < 0 || share_messages > 2)
+        return CR_ERR_INVALID_ARG;
+    Expanded ex;
+    cr_status_t st = expand_all(plan->hp, masks_host, batch, share_messages, ex);
+    if (st != CR_OK) return st;
+    int64_t variants = 0;
+    for (const int4 &op : ex.ops) variants += op.z >> 8;
+    stats[0] = (int64_t)ex.steps.size();
+    stats[1] = (int64_t)ex.unodes.size();
+    stats[2] = (int64_t)ex.ops.size();
+    stats[3] = variants;
+    stats[4] = (int64_t)ex.red_steps.size();
+    stats[5] = ex.n_rows;
+    return CR_OK;
+}
+
 cr_status_t cr_plan_tune_batch(cr_plan_t *plan, int32_t share_messages, int32_t e_buffers) {
     if (!plan || share_messages < 0 || share_messages > 2 || e_buffers < 0 || e_buffers > 2) return CR_ERR_INVALID_ARG;
     plan->tune.share = share_messages;

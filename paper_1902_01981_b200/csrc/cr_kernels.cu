@@ -214,6 +214,7 @@ struct FusedArgs {
     int n_inline;           // entries of steps_inline in use (0: read `steps`)
     Step steps_inline[kInlineSteps];
     int n_steps;
+    int steps_smem;         // a staged schedule (n_inline == 0) is copied into shared memory at the start
     int m, R, cpn, stages;
     long long d;
     long long ntiles;
@@ -222,6 +223,11 @@ struct FusedArgs {
     int *status;
     unsigned long long wait_ns;  // bound of every wait, in nanoseconds
 };
+
+// Longest staged schedule that the single-pattern kernel copies into shared memory (16 KB).  Read from global
+// memory instead, the node id in front of every box is a dependent L2 latency on the producer's path: a
+// 182-node pattern ran at 1.9 TB/s where the plain-load kernel reaches 4.4.
+constexpr int kSmemSteps = 1024;
 
 // (Four 160-thread CTAs per SM need at most 96 registers per thread; the L <= 4 instances sit at 97 without
 // the bound and lose nothing to it.)
@@ -240,6 +246,7 @@ cr_fused_tma_kernel(const __grid_constant__ CUtensorMap tmap, const FusedArgs a)
     uint64_t *full = reinterpret_cast<uint64_t *>(smem_raw + (size_t)S * stage_elems * sizeof(T));
     uint64_t *empty = full + S;
     volatile int *flags = reinterpret_cast<volatile int *>(empty + S);
+    Step *steps_s = reinterpret_cast<Step *>(smem_raw + (((size_t)S * stage_elems * sizeof(T) + (size_t)S * 16 + 32 + 15) & ~(size_t)15));
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     if (tid == 0) {
@@ -248,6 +255,9 @@ cr_fused_tma_kernel(const __grid_constant__ CUtensorMap tmap, const FusedArgs a)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    if (a.steps_smem)
+        for (int k = tid; k < a.n_steps; k += blockDim.x)
+            reinterpret_cast<int4 *>(steps_s)[k] = __ldg(reinterpret_cast<const int4 *>(a.steps) + k);
     __syncthreads();
 
     const T *coeff = reinterpret_cast<const T *>(a.coeff);
@@ -263,7 +273,7 @@ cr_fused_tma_kernel(const __grid_constant__ CUtensorMap tmap, const FusedArgs a)
             for (long long tile = blockIdx.x; tile < a.ntiles && ok; tile += gridDim.x) {
                 const int x0 = (int)(tile * TILE);
                 for (int k = 0; k < a.n_steps && ok; ++k) {
-                    const int row0 = (a.n_inline ? a.steps_inline[k].node : __ldg(&a.steps[k].node)) * a.m;
+                    const int row0 = (a.n_inline ? a.steps_inline[k].node : (a.steps_smem ? steps_s[k].node : __ldg(&a.steps[k].node))) * a.m;
                     for (int c = 0; c < a.cpn; ++c) {
                         if (!mbar_wait(&empty[stage], phase ^ 1u, &flags[0], a.wait_ns)) { ok = false; break; }
                         mbar_expect_tx(&full[stage], stage_bytes);
@@ -301,6 +311,7 @@ cr_fused_tma_kernel(const __grid_constant__ CUtensorMap tmap, const FusedArgs a)
         bool ok = true;
         auto step_at = [&](int k) {
             if (a.n_inline) { Step t = a.steps_inline[k]; t.layer &= 0xff; return t; }
+            if (a.steps_smem) { Step t = steps_s[k]; t.layer &= 0xff; return t; }
             return load_step(&a.steps[k]);
         };
         Step st_next = step_at(0);
@@ -1601,8 +1612,19 @@ cudaError_t launch_fused_tma(const AggArgs &a, const DeviceInfo &dev, const Tuni
     // one.  So: boxes of at most ~18 KB (R = a divisor of m), three CTAs per SM, and as many stages
     // as bring the total to ~36 KB per CTA, at least two.
     const int cap = std::min(kMaxBoxRows, std::max(1, (18 * 1024) / (tile * 4)));
-    const int R = tune.rows && a.m % tune.rows == 0 && tune.rows <= kMaxBoxRows ? tune.rows : rows_per_box(a.m, cap);
+    int R = tune.rows && a.m % tune.rows == 0 && tune.rows <= kMaxBoxRows ? tune.rows : rows_per_box(a.m, cap);
+    // A box holds a divisor of m rows.  When m has no divisor under the soft cap but one row (m = 11 or 13 with
+    // 512-column tiles), a box of one row is 2 KB and the copy engine, not HBM, sets the pace (1.9 TB/s
+    // measured): take the taller box if there is one, and leave nodes that only split into thin boxes to the
+    // plain-load kernel.
+    if (!tune.rows && R < 4 && a.m > R) {
+        R = rows_per_box(a.m, kMaxBoxRows);
+        if (R < 4) return cudaSuccess;
+    }
     const size_t stage_bytes = (size_t)R * tile * 4;
+    // a schedule too long for the kernel parameters rides in shared memory when it is short enough for that
+    const bool inline_ok = a.host_steps && a.total_steps <= kInlineSteps;
+    const size_t steps_bytes = (!inline_ok && a.total_steps <= kSmemSteps) ? (size_t)a.total_steps * sizeof(Step) + 16 : 0;
     int ctas = tune.ctas_per_sm ? tune.ctas_per_sm : 3;
     int stages = tune.stages ? tune.stages
                              : std::max(2, std::min(8, (int)((36 * 1024 + stage_bytes / 2) / stage_bytes)));
@@ -1625,7 +1647,7 @@ cudaError_t launch_fused_tma(const AggArgs &a, const DeviceInfo &dev, const Tuni
         double best_fill = fill(ctas);
         for (int c = ctas + 1; c <= 6; ++c) {
             const int thin = tune.stages ? stages : std::max(2, stages * ctas / c);
-            if (fused_resident_any(a.is_int, ncw, pick_lmax(a.L), (size_t)thin * stage_bytes + (size_t)thin * 16 + 32) < c) break;
+            if (fused_resident_any(a.is_int, ncw, pick_lmax(a.L), (size_t)thin * stage_bytes + (size_t)thin * 16 + 32 + steps_bytes) < c) break;
             if (fill(c) > best_fill + 0.03) { best = c; best_stages = thin; best_fill = fill(c); }
             if ((long long)dev.sm_count * c >= tiles_now) break;
         }
@@ -1633,9 +1655,9 @@ cudaError_t launch_fused_tma(const AggArgs &a, const DeviceInfo &dev, const Tuni
         stages = best_stages;
     }
     const size_t usable = (size_t)dev.smem_per_sm - 2048;  // leave room for the per-CTA reserve
-    while (ctas > 1 && ((size_t)stages * stage_bytes + 1024 + 256) * ctas > usable) --ctas;
-    while (stages > 2 && (size_t)stages * stage_bytes + 256 > (size_t)dev.smem_optin) --stages;
-    const size_t smem = (size_t)stages * stage_bytes + (size_t)stages * 16 + 32;
+    while (ctas > 1 && ((size_t)stages * stage_bytes + steps_bytes + 1024 + 256) * ctas > usable) --ctas;
+    while (stages > 2 && (size_t)stages * stage_bytes + steps_bytes + 256 > (size_t)dev.smem_optin) --stages;
+    const size_t smem = (size_t)stages * stage_bytes + (size_t)stages * 16 + 32 + steps_bytes;
     if (smem > (size_t)dev.smem_optin) return cudaSuccess;  // does not fit: caller falls back to plain loads
 
     CUtensorMap map;
@@ -1643,7 +1665,8 @@ cudaError_t launch_fused_tma(const AggArgs &a, const DeviceInfo &dev, const Tuni
 
     FusedArgs fa;
     fa.n_inline = 0;
-    if (a.host_steps && a.total_steps <= kInlineSteps) {
+    fa.steps_smem = steps_bytes ? 1 : 0;
+    if (inline_ok) {
         fa.n_inline = a.total_steps;
         for (int k = 0; k < a.total_steps; ++k) fa.steps_inline[k] = a.host_steps[k];
     } else if (!a.steps) {

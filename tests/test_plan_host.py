@@ -220,3 +220,46 @@ def test_baseline_config_sizes():
         assert (B.cr_plan_num_nodes(plan), B.cr_plan_num_groups(plan), B.cr_plan_load(plan)) == (N, groups, m)
         assert B.cr_plan_load(plan) == O.computation_load(n, L, s) * P
         B.cr_plan_destroy(plan)
+
+
+@pytest.mark.parametrize("n,L,s,code,batch,exactly", [(12, 2, 1, B.CR_CODE_CYCLIC_RANDOM, 64, True), (4, 3, 1, B.CR_CODE_CYCLIC_RANDOM, 40, False),
+                                                      (3, 4, 1, B.CR_CODE_PAPER_3_1, 64, False), (5, 2, 2, B.CR_CODE_CYCLIC_RANDOM, 30, True),
+                                                      (6, 2, 2, B.CR_CODE_FRACTIONAL_REPETITION, 16, True)])
+def test_shared_message_tables_against_a_count_from_the_oracle(n, L, s, code, batch, exactly):
+    """The batch kernel shares the messages of the nodes above the leaves among the patterns of a batch.
+    What the host derives for that -- the union, the distinct (node, decode row) variants, the lengths of the
+    full and the reduced schedules -- is recounted here from the oracle's own decode rows."""
+    plan = host_plan(n, L, s, code=code)
+    try:
+        if code == B.CR_CODE_CYCLIC_RANDOM:
+            Bm, _ = O.cyclic_random_code(n, s, 0, 100.0)
+            ocode = O.Code(n, L, s, [Bm] * L, kind="solve")
+        else:
+            ocode = oracle_code(plan, code, n, L, s)
+        masks = inputs.straggler_masks(n, L, s, batch, seed=71, exactly_s=exactly)
+        used = [O.used_nodes(ocode, masks[b]) for b in range(batch)]
+        union = sorted(set(v for u in used for v in u))
+        lo, hi = O.layer_offset(n, L - 1), O.layer_offset(n, L)          # flat indices of layer L-1
+        variants, reduced = set(), 0
+        for b in range(batch):
+            for v in used[b]:
+                if lo <= v < hi:
+                    reduced += 1
+                    i = v - lo + 1                                        # node (L-1, i)
+                    a = ocode.decode(L - 1, int(masks[b][O.group_of_parent(n, L - 1, i)]))
+                    kids = O.children_of(n, L, L - 1, i)
+                    row = tuple(np.float32(a[j]) if kids[j] in union else None for j in range(n))
+                    variants.add((v, tuple(x for x in row if x is not None)))
+                elif v < lo:
+                    reduced += 1
+        st = B.cr_plan_batch_stats(plan, masks, 2)
+        assert st["entries"] == sum(len(u) for u in used)
+        assert st["union"] == len(union)
+        assert st["shared_nodes"] == len({v for v, _ in variants})
+        assert st["variants"] == len(variants)
+        assert st["reduced_entries"] == reduced
+        assert st["rows"] >= st["union"]
+        off = B.cr_plan_batch_stats(plan, masks, 1)
+        assert off["shared_nodes"] == 0 and off["entries"] == st["entries"] and off["rows"] == off["union"]
+    finally:
+        B.cr_plan_destroy(plan)
