@@ -202,7 +202,7 @@ cr_status_t cr_partial_gradients_loss(cr_plan_t *plan, int32_t loss, const float
                                       const float *w, float *G_slots, void *workspace, size_t workspace_bytes,
                                       void *stream);
 
-/* ---- CR.Execute, "all nodes compute their local partial CODED gradients" in one step -----------
+/* ---- CR.Execute step 1 in coded form: every node's local coded gradient in one pass (Section III-A) ----
  * E[v][:] = g_{D(l,i)} = sum_j c_{v,j} * X_p^T r_p with p the partition of slot j of node v
  * (Section III-A: D(l,i) carries the combining coefficients along with its data points), r_p the
  * residuals of `loss` at w.  The slot gradients are never written: each node's cluster of CTAs walks
