@@ -436,7 +436,14 @@ class AggregateSetup:
             scheduled.append(t3 - t2)
         torch.cuda.synchronize()
         B.cr_schedule_destroy(sched)
+        # what the binding itself costs: a call through ctypes that does nothing on the device
+        trivial = []
+        for i in range(calls):
+            t0 = time.perf_counter_ns()
+            B.cr_plan_launch_count(self.plan)
+            trivial.append(time.perf_counter_ns() - t0)
         return {"cr_aggregate": float(np.median(direct)) * 1e-3, "cr_aggregate_scheduled": float(np.median(scheduled)) * 1e-3,
+                "ctypes_call_that_launches_nothing": float(np.median(trivial)) * 1e-3,
                 "note": "host clock around the call through the Python binding, stream idle, median of %d" % calls}
 
     def parity_on_sample(self, cols, flags, patterns=2):

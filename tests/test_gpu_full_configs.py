@@ -101,6 +101,20 @@ def test_paper_cluster_trees_d_2_22(name):
         assert rel_l2(got[0], O.full_gradient(G_cols)) <= REL_L2_BAR
 
 
+@pytest.mark.parametrize("name", ["cfg_tree12", "cfg_tree43"])
+def test_paper_cluster_trees_batches_of_64_d_2_20(name):
+    """Batches of 64 patterns on the paper's trees at d = 2^20, as `bench.py --batch 64 --d 1048576` times
+    them: the patterns share the messages of the layer above the leaves.  Every pattern against the plain
+    sum, a spread of them against CR.Execute."""
+    cfg = dict(inputs.CONFIGS[name], d=1 << 20, batch=64)
+    for code, local, got, G_cols, masks in aggregate_full(cfg, B.CR_F32, 2):
+        want_sum = O.full_gradient(G_cols)
+        for b in range(64):
+            assert rel_l2(got[b], want_sum) <= REL_L2_BAR
+        for b in range(0, 64, 9):
+            assert rel_l2(got[b], O.execute(code, local, G_cols, masks[b])) <= REL_L2_BAR
+
+
 @pytest.mark.parametrize("n,s,code", [(12, 1, "cyclic"), (12, 3, "repetition"), (3, 1, "printed_3_1")])
 def test_flat_gradient_coding_d_2_22(n, s, code):
     """L = 1: CodedReduce is flat gradient coding (master and n workers, m = s + 1 slot rows per worker).

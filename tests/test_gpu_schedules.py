@@ -172,6 +172,39 @@ def test_scheduled_call_equals_the_direct_call(cfg, batch, dtype, flags):
         B.cr_plan_destroy(plan)
 
 
+@pytest.mark.parametrize("cfg,batch", [(tree(3, 1, 1, "printed_3_1", 1001), 1), (tree(3, 1, 1, "printed_3_1", 1001), 5),
+                                       (tree(4, 2, 1, "cyclic", 3), 4), (tree(5, 1, 2, "cyclic", 1 << 16), 1),
+                                       (tree(13, 2, 0, "cyclic", 2048, P=182 * 11), 1)])
+def test_schedules_at_the_edges(cfg, batch):
+    """Flat gradient coding (L = 1), lengths that are not multiples of four (the scalar plain-load path), a
+    length of 3, a pattern of 182 consumed nodes with 11 slot rows each (a schedule too long for the kernel
+    parameters, a slot count without a small divisor): scheduled call, direct call, oracle; also from coded
+    gradients."""
+    n, L, s, d = cfg["n"], cfg["L"], cfg["s"], cfg["d"]
+    plan = make_plan(cfg)
+    try:
+        code, local = check_slot_table(plan, cfg)
+        G = inputs.partition_gradients(cfg["P"], d, seed=81)
+        G_dev = slots_on_device(plan, G, torch)
+        masks = inputs.straggler_masks(n, L, s, batch, seed=82)
+        E = torch.zeros((B.cr_plan_num_nodes(plan), d), device="cuda")
+        B.cr_encode(plan, G_dev, E)
+        for flags, src in ((B.CR_AGG_FUSED, G_dev), (B.CR_AGG_FUSED | B.CR_AGG_FROM_CODED, E)):
+            sched = B.cr_schedule_create(plan, masks, flags)
+            got = torch.full((batch, d), 5.0, device="cuda")
+            direct = torch.full((batch, d), 6.0, device="cuda")
+            B.cr_aggregate_scheduled(plan, src, sched, got)
+            B.cr_aggregate(plan, src, masks, direct, flags)
+            torch.cuda.synchronize()
+            assert torch.equal(got, direct)
+            for b in range(batch):
+                assert rel_l2(got[b].cpu().numpy(), O.execute(code, local, G, masks[b])) <= REL_L2_BAR
+            B.cr_schedule_destroy(sched)
+        assert B.cr_plan_device_status(plan) == B.CR_OK
+    finally:
+        B.cr_plan_destroy(plan)
+
+
 def test_schedule_errors_and_raw_pointers():
     cfg = tree(4, 2, 1, "cyclic", 1024)
     plan, other = make_plan(cfg), make_plan(cfg)
