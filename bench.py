@@ -757,6 +757,8 @@ def run_linreg(args, cfg):
     plan = B.cr_plan_create(n, L, s, P, d, code=code_id, device=0)
     if args.tune_gradients:
         B.cr_plan_tune_gradients(plan, *[int(x) for x in args.tune_gradients.split(",")])
+    if args.item_order:
+        B.cr_plan_tune_items(plan, args.item_order, 0)
     N, m, groups = B.cr_plan_num_nodes(plan), B.cr_plan_load(plan), B.cr_plan_num_groups(plan)
     logistic = cfg["kind"] == "logistic"
     loss = B.CR_LOSS_LOGISTIC if logistic else B.CR_LOSS_SQUARED
@@ -985,6 +987,8 @@ def main():
     ap.add_argument("--share", type=int, default=0, help="batches: messages shared by the patterns: 0 built-in choice, "
                     "1 never, 2 whenever possible")
     ap.add_argument("--e-buffers", type=int, default=0, help="batches: buffers of coded gradients in shared memory (1, 2)")
+    ap.add_argument("--item-order", type=int, default=0, help="regression workloads: launch order of the (node, slot) items: "
+                    "1 by node then slot, 2 grouped by partition (0: built-in choice)")
     ap.add_argument("--coded", action="store_true", help="regression workloads: gradient + encode in one kernel")
     ap.add_argument("--models", type=int, default=0, help="regression workloads: gradients of K models per pass (1..32)")
     ap.add_argument("--no-e2e", action="store_true")

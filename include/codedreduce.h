@@ -353,7 +353,8 @@ cr_status_t cr_plan_tune_gradients(cr_plan_t *plan, int32_t block_kb, int32_t st
 /* Order in which the partial-gradient kernels launch the (node, slot) items, and ring depth of the
  * second kernel of cr_partial_gradients_multi; 0 keeps the built-in choice for that field.
  * item_order: 1 = by node, then slot; 2 = grouped by partition (items that hold the same partition
- * run side by side and share its rows through L2).  multi_stages: 2..4 (2 lets two CTAs share an SM). */
+ * run side by side and share its rows through L2; the built-in choice of every partial-gradient kernel).
+ * multi_stages: 2..4 (2 lets two CTAs share an SM). */
 cr_status_t cr_plan_tune_items(cr_plan_t *plan, int32_t item_order, int32_t multi_stages);
 
 /* Kernel launches enqueued by this plan's device calls so far. */

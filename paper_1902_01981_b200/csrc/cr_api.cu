@@ -574,8 +574,11 @@ cr_status_t cr_partial_gradients_loss(cr_plan_t *plan, int32_t loss, const float
     const int items = plan->hp.N * plan->hp.m;
     cudaError_t e;
     if (cr::partial_fused_eligible(X, w, G_slots, plan->hp.d, items)) {
-        // one pass over X, no scratch
-        e = cr::launch_partial_gradients_fused(X, y, w, plan->d_part, plan->tune.pg_order == 2 ? plan->d_order : nullptr, nullptr, items, 1, rows, plan->hp.d, G_slots, loss,
+        // one pass over X, no scratch; items grouped by partition unless the caller asked for (node, slot) order:
+        // the clusters that hold the same partition then run side by side and share its rows through L2 (since
+        // the kernel reads shared memory once per block it is close to the DRAM bound and gains from that:
+        // 2048 x 4096 partitions 0.557 -> 0.533 ms)
+        e = cr::launch_partial_gradients_fused(X, y, w, plan->d_part, plan->tune.pg_order == 1 ? nullptr : plan->d_order, nullptr, items, 1, rows, plan->hp.d, G_slots, loss,
                                                plan->d_status, plan->dev, plan->tune,
                                                reinterpret_cast<cudaStream_t>(stream), &plan->launches);
     } else {
