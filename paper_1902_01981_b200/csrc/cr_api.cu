@@ -823,7 +823,9 @@ cr_status_t prepare(const cr_plan *plan, const uint32_t *masks_host, int batch, 
         if (!pr.ex.ops.empty()) {
             q.total_steps = (int)ex.red_steps.size(); q.same_shape = pr.red_same_shape;
             q.n_rows = ex.n_rows; q.n_ops = (int)ex.ops.size(); q.vtab_words = (int)ex.vtab.size();
+            q.L = hp.L - 1;   // the reduced schedules end at the layer above the leaves
             pr.shape = cr::batch_shape(q, plan->dev, plan->tune);
+            q.L = hp.L;
             if (!pr.shape.ok) {   // the shared form does not fit: the plain one
                 pr.ex.ops.clear(); pr.ex.vtab.clear(); pr.ex.red_steps.clear(); pr.ex.red_off.clear();
                 pr.ex.n_rows = (int)ex.unodes.size();
@@ -1009,6 +1011,7 @@ int run_prepared(cr_plan *plan, const Prepared &pr, const unsigned char *tables,
                     r.pat_off = reinterpret_cast<const int32_t *>(tables + pr.off_red_pat);
                     r.total_steps = (int)ex.red_steps.size();
                     r.same_shape = pr.red_same_shape;
+                    r.L = hp.L - 1;   // depth of the reduced schedules: the kernel instance for that depth serves them
                     r.n_rows = ex.n_rows; r.n_ops = (int)ex.ops.size();
                     r.ops = reinterpret_cast<const int4 *>(tables + pr.off_ops);
                     r.vtab = reinterpret_cast<const uint32_t *>(tables + pr.off_vtab);

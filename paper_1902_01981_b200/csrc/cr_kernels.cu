@@ -1813,7 +1813,7 @@ cudaError_t launch_fused_batch_tma(const AggArgs &a, const BatchShape &sh, const
     ba.wait_ns = tune.wait_limit_ns;
     ba.n_rows = sh.n_rows; ba.n_ops = a.n_ops; ba.ops = a.ops; ba.vtab = a.vtab; ba.vtab_words = a.vtab_words;
     ba.vtab_smem = sh.vtab_smem;
-    ba.flat = (a.n_ops && a.L == 2 && sh.sched_bytes) ? 1 : 0;
+    ba.flat = (a.n_ops && a.L == 1 && sh.sched_bytes) ? 1 : 0;   // a.L: depth of the (reduced) schedules
     const int lmax = pick_lmax(a.L);
     const cudaError_t err = a.is_int ? run_batch_w<int>(sh.nlw, sh.nrw, lmax, map, ba, sh.grid, sh.smem, stream)
                                      : run_batch_w<float>(sh.nlw, sh.nrw, lmax, map, ba, sh.grid, sh.smem, stream);

@@ -60,7 +60,7 @@ struct AggArgs {
     int batch;
     int total_steps;
     int m;
-    int L;
+    int L;                // layers of the schedules (with shared messages: of the reduced ones, one less than the tree's)
     int64_t d;
     int64_t rows_total;   // N*m
     void *out;            // [batch][d]
