@@ -1284,30 +1284,98 @@ struct PgArgs {
 
 // Rows of a block: as many as a thread can keep in registers (its KPT column groups of each row).
 __host__ __device__ constexpr int pg_block_rows(int kpt) { return 12 / kpt > 0 ? 12 / kpt : 1; }
+// Words of one buffer of per-warp partial residuals: chunks of four rows, [row in chunk][warp].
+__host__ __device__ constexpr int pg_red_words(int kpt) { return (pg_block_rows(kpt) + 3) / 4 * 32; }
+
+__device__ __forceinline__ float4 lds128(uint32_t addr) {
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr));
+    return v;
+}
+
+// Sums over the warp of R per-lane values, four rows at a time: the first two exchange steps halve the
+// number of values instead of repeating the butterfly per row (6 shuffles for 4 rows against 20), after which
+// lane class (lane >> 3) holds row 2 * (bit 3) + (bit 4) of the chunk.  One lane per class stores the warp's
+// sum at red[chunk][row][warp].
+template <int R>
+__device__ __forceinline__ void pg_warp_sums(const float (&part)[R], float *redb, int warp, int lane) {
+    constexpr unsigned FULL = 0xffffffffu;
+    const bool up16 = (lane & 16) != 0, up8 = (lane & 8) != 0;
+#pragma unroll
+    for (int c = 0; c < (R + 3) / 4; ++c) {
+        const int n = R - 4 * c < 4 ? R - 4 * c : 4;   // rows of this chunk
+        float b;
+        if (n == 1) {
+            b = part[4 * c];
+            b += __shfl_xor_sync(FULL, b, 16);
+            b += __shfl_xor_sync(FULL, b, 8);
+        } else {
+            // (indices clamped where the chunk has fewer rows: those values are not used)
+            const float v0 = part[4 * c], v1 = part[4 * c + 1 < R ? 4 * c + 1 : 0];
+            const float a0 = (up16 ? v1 : v0) + __shfl_xor_sync(FULL, up16 ? v0 : v1, 16);
+            if (n == 2) {
+                b = a0 + __shfl_xor_sync(FULL, a0, 8);
+            } else {
+                const float v2 = part[4 * c + 2 < R ? 4 * c + 2 : 0], v3 = n == 4 ? part[4 * c + 3 < R ? 4 * c + 3 : 0] : 0.f;
+                const float a1 = (up16 ? v3 : v2) + __shfl_xor_sync(FULL, up16 ? v2 : v3, 16);
+                b = (up8 ? a1 : a0) + __shfl_xor_sync(FULL, up8 ? a0 : a1, 8);
+            }
+        }
+        b += __shfl_xor_sync(FULL, b, 4);
+        b += __shfl_xor_sync(FULL, b, 2);
+        b += __shfl_xor_sync(FULL, b, 1);
+        // n == 1: every class holds row 0; n == 2: classes with bit 4 hold row 1 (both bit-3 classes alike)
+        const int row = n == 1 ? 0 : (n == 2 ? (lane >> 4) & 1 : ((lane >> 3) & 1) * 2 + ((lane >> 4) & 1));
+        if ((lane & 7) == 0) redb[c * 32 + row * 8 + warp] = b;
+    }
+}
+
+// The residual sums of the block's rows from the eight warps' partial sums: lane l reads the entry of row
+// l >> 3 and warp l & 7 of each chunk, three exchange steps add the eight warps, and a shuffle hands every
+// lane the sum of each row (10 instructions per chunk against 2 loads and 7 additions per row).
+template <int R>
+__device__ __forceinline__ void pg_block_sums(const float *redb, int lane, float (&z)[R]) {
+    constexpr unsigned FULL = 0xffffffffu;
+#pragma unroll
+    for (int c = 0; c < (R + 3) / 4; ++c) {
+        float v = redb[c * 32 + lane];
+        v += __shfl_xor_sync(FULL, v, 4);
+        v += __shfl_xor_sync(FULL, v, 2);
+        v += __shfl_xor_sync(FULL, v, 1);
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (4 * c + j < R) z[4 * c + j] = __shfl_sync(FULL, v, j * 8);
+    }
+}
 
 // GENERAL = false is the case of one slot per item without slot coefficient, kept free of the bookkeeping of
 // the general one (measured: 5 % faster on 2048 x 4096 partitions).
 // Per block a thread reads its share of every row from shared memory ONCE, into registers: the same
 // values serve the residuals (pass A) and, once the residuals are known, the gradient update (pass B).
-// Every thread then folds the eight per-warp partial sums of each row itself, so one CTA-wide barrier
-// per block is all the synchronisation there is -- it also tells that everybody has read the buffer, so
-// the copy of block blk + S goes into it at once.  (The first version read X from shared memory in both
-// passes and took three barriers per block: shared-memory wavefronts 48 %, DRAM 48 % of peak.)
+// One CTA-wide barrier per block is all the synchronisation there is -- it also tells that everybody has
+// read the buffer, so the copy of block blk + S goes into it at once.  What a block costs besides its
+// multiply-adds is a chain of dependent instructions that every warp runs once per block, whatever the
+// number of rows (measured: blocks of one row take as long as blocks of three), so that chain is kept
+// short: 32-bit shared-memory addresses, buffer and phase counted up instead of divided out, the warp
+// sums of all rows in one butterfly, the cross-warp sums by shuffles.
+// (The first version read X from shared memory in both passes and took three barriers per block:
+// shared-memory wavefronts 48 %, DRAM 48 % of peak.)
 template <int KPT, bool GENERAL, bool LOGISTIC>
 __global__ void __launch_bounds__(256, 2)
 cr_partial_fused_kernel(const PgArgs a) {
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
     constexpr int RBC = pg_block_rows(KPT);
+    constexpr int REDW = pg_red_words(KPT);
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const long long d = a.d;
+    const int d = (int)a.d;              // d <= 1024 * KPT
     const int RB = a.RB, S = a.stages;   // RB <= RBC
     const size_t stage_elems = (size_t)RB * d;
     float *ring = reinterpret_cast<float *>(smem_raw);
     float *gpart = ring + (size_t)S * stage_elems;          // [d] this CTA's partial gradient
-    float *red = gpart + d;                                 // [2][RBC][8] per-warp partial residuals, double buffered
-    uint64_t *full = reinterpret_cast<uint64_t *>(red + 2 * RBC * 8);
+    float *red = gpart + d;                                 // [2][REDW] per-warp partial residuals, double buffered
+    uint64_t *full = reinterpret_cast<uint64_t *>(red + 2 * REDW);
     volatile int *flags = reinterpret_cast<volatile int *>(full + S);
 
     if (tid == 0) {
@@ -1329,104 +1397,122 @@ cr_partial_fused_kernel(const PgArgs a) {
     const int b0 = min(total_blocks, (int)blockIdx.x * per_cta);
     const int nblocks = min(total_blocks, b0 + per_cta) - b0;
     // Position in the list, kept incrementally (no division and no dependent load per block): slot
-    // within the item, block within the slot, the slot's partition; one copy for the thread that
-    // issues the copies (it runs S blocks ahead), one for the consumers.
+    // within the item, block within the slot, where the block's rows and labels start; one copy for the
+    // thread that issues the copies (it runs S blocks ahead), one for the consumers.
     const int slot0 = b0 / bps;
     int i_slot = slot0, i_bi = b0 - slot0 * bps, c_slot = slot0, c_bi = i_bi;
-    int i_p = 0, c_p = 0;
+    const float *i_src = a.X, *c_y = a.y;
     float c_scale = 1.f;
     if (nblocks > 0) {
-        c_p = __ldg(&a.part[item * spi + slot0]);
-        i_p = c_p;
+        const int p0 = __ldg(&a.part[item * spi + slot0]);
+        i_src = a.X + ((size_t)p0 * a.rows + (size_t)i_bi * RB) * d;
+        c_y = a.y + (size_t)p0 * a.rows + (size_t)c_bi * RB;
         if (GENERAL && a.coeff) c_scale = __ldg(&a.coeff[item * spi + slot0]);
     }
 
     float4 wv[KPT], acc[KPT];
+    uint32_t koff[KPT];   // byte offset of the thread's k-th column group in a row; a group beyond d reads
+                          // the row's first four columns instead (always there: finite numbers, against a
+                          // zero weight, never stored)
 #pragma unroll
     for (int k = 0; k < KPT; ++k) {
-        const long long col = 4ll * tid + 1024ll * k;
+        const int col = 4 * tid + 1024 * k;
         wv[k] = col < d ? __ldg(reinterpret_cast<const float4 *>(a.w + col)) : make_float4(0.f, 0.f, 0.f, 0.f);
+        koff[k] = col < d ? (uint32_t)col * 4u : 0u;
         acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
     }
+    const uint32_t ring_u32 = smem_u32(ring);
+    const uint32_t row_bytes = (uint32_t)d * 4u, stage_bytes = (uint32_t)RB * row_bytes;
 
-    int issued = 0;
-    auto issue = [&](int blk) {  // thread 0 only; blocks are issued in order
+    int issued = 0, i_stage = 0;
+    auto issue = [&]() {  // thread 0 only; blocks are issued in order
         const int nr_i = min(RB, a.rows - i_bi * RB);
-        const uint32_t bytes = (uint32_t)((size_t)nr_i * d * sizeof(float));
-        mbar_expect_tx(&full[blk % S], bytes);
-        bulk_load_1d(ring + (size_t)(blk % S) * stage_elems, a.X + ((size_t)i_p * a.rows + (size_t)i_bi * RB) * d,
-                     bytes, &full[blk % S]);
+        const uint32_t bytes = (uint32_t)nr_i * row_bytes;
+        mbar_expect_tx(&full[i_stage], bytes);
+        bulk_load_1d(ring + (size_t)i_stage * stage_elems, i_src, bytes, &full[i_stage]);
+        i_src += (size_t)nr_i * d;
+        if (++i_stage == S) i_stage = 0;
         ++i_bi;
+        ++issued;
         if (GENERAL && i_bi == bps) {
             i_bi = 0; ++i_slot;
-            if (blk + 1 < nblocks) i_p = __ldg(&a.part[item * spi + i_slot]);
+            if (issued < nblocks) i_src = a.X + (size_t)__ldg(&a.part[item * spi + i_slot]) * a.rows * d;
         }
     };
     if (tid == 0)
-        for (; issued < nblocks && issued < S; ++issued) issue(issued);
+        while (issued < nblocks && issued < S) issue();
 
-    int done = 0;
+    int done = 0, stage = 0;
+    uint32_t phase = 0;
     for (int blk = 0; blk < nblocks; ++blk) {
         const int nr = min(RB, a.rows - c_bi * RB);
         // labels of the block's rows, fetched before the wait so that their latency hides behind it
         float yv[RBC];
 #pragma unroll
-        for (int r = 0; r < RBC; ++r) yv[r] = r < nr ? __ldg(a.y + (size_t)c_p * a.rows + (size_t)c_bi * RB + r) : 0.f;
+        for (int r = 0; r < RBC; ++r) yv[r] = r < nr ? __ldg(c_y + r) : 0.f;
         const float scale = c_scale;
+        c_y += RB;
         ++c_bi;
         if (GENERAL && c_bi == bps) {     // the next block opens the next slot of the item
             c_bi = 0; ++c_slot;
             if (blk + 1 < nblocks) {
-                c_p = __ldg(&a.part[item * spi + c_slot]);
+                c_y = a.y + (size_t)__ldg(&a.part[item * spi + c_slot]) * a.rows;
                 if (a.coeff) c_scale = __ldg(&a.coeff[item * spi + c_slot]);
             }
         }
-        const int ok = mbar_wait(&full[blk % S], (uint32_t)((blk / S) & 1), &flags[1], a.wait_ns) ? 1 : 0;
-        const float *Xb = ring + (size_t)(blk % S) * stage_elems;
+        const int ok = mbar_wait(&full[stage], phase, &flags[1], a.wait_ns) ? 1 : 0;
+        const uint32_t xb = ring_u32 + (uint32_t)stage * stage_bytes;
         // this thread's share of the block, read once; pass A: partial residuals
         float4 xf[RBC][KPT];
         float part[RBC];
+        if (nr == RBC) {
+#pragma unroll
+            for (int r = 0; r < RBC; ++r)
+#pragma unroll
+                for (int k = 0; k < KPT; ++k) xf[r][k] = lds128(xb + (uint32_t)r * row_bytes + koff[k]);
+        } else {   // the last block of a slot: rows the copy did not bring count as zeros
+#pragma unroll
+            for (int r = 0; r < RBC; ++r)
+#pragma unroll
+                for (int k = 0; k < KPT; ++k)
+                    xf[r][k] = r < nr ? lds128(xb + (uint32_t)r * row_bytes + koff[k]) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
 #pragma unroll
         for (int r = 0; r < RBC; ++r) {
-            part[r] = 0.f;
+            // two chains of multiply-adds per row
+            float p0 = xf[r][0].x * wv[0].x, p1 = xf[r][0].y * wv[0].y;
+            p0 = fmaf(xf[r][0].z, wv[0].z, p0); p1 = fmaf(xf[r][0].w, wv[0].w, p1);
 #pragma unroll
-            for (int k = 0; k < KPT; ++k) {
-                const long long col = 4ll * tid + 1024ll * k;
-                xf[r][k] = (r < nr && col < d) ? *reinterpret_cast<const float4 *>(Xb + (size_t)r * d + col)
-                                               : make_float4(0.f, 0.f, 0.f, 0.f);
-                part[r] += xf[r][k].x * wv[k].x + xf[r][k].y * wv[k].y + xf[r][k].z * wv[k].z + xf[r][k].w * wv[k].w;
+            for (int k = 1; k < KPT; ++k) {
+                p0 = fmaf(xf[r][k].x, wv[k].x, p0); p1 = fmaf(xf[r][k].y, wv[k].y, p1);
+                p0 = fmaf(xf[r][k].z, wv[k].z, p0); p1 = fmaf(xf[r][k].w, wv[k].w, p1);
             }
+            part[r] = p0 + p1;
         }
-        float *redb = red + (blk & 1) * (RBC * 8);
-#pragma unroll
-        for (int r = 0; r < RBC; ++r) {
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) part[r] += __shfl_xor_sync(0xffffffffu, part[r], o);
-            if (lane == 0) redb[r * 8 + warp] = part[r];
-        }
+        float *redb = red + (blk & 1) * REDW;
+        pg_warp_sums<RBC>(part, redb, warp, lane);
         // the one barrier of the block: the partial sums are visible, and everybody has read the buffer
         if (!__syncthreads_and(ok)) break;
         if (tid == 0 && issued < nblocks) {
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            issue(issued);
-            ++issued;
+            issue();
         }
         // pass B from the registers: acc += r[row] * X_b[row, cols]
+        float z[RBC];
+        pg_block_sums<RBC>(redb, lane, z);
 #pragma unroll
         for (int r = 0; r < RBC; ++r) {
-            if (r < nr) {
-                const float4 p0 = *reinterpret_cast<const float4 *>(redb + r * 8);
-                const float4 p1 = *reinterpret_cast<const float4 *>(redb + r * 8 + 4);
-                float z = ((p0.x + p0.y) + (p0.z + p0.w)) + ((p1.x + p1.y) + (p1.z + p1.w));
-                if (LOGISTIC) z = 1.f / (1.f + expf(-z));
-                const float rr = GENERAL ? scale * (z - yv[r]) : z - yv[r];
+            float zr = z[r];
+            if (LOGISTIC) zr = 1.f / (1.f + expf(-zr));
+            float rr = GENERAL ? scale * (zr - yv[r]) : zr - yv[r];
+            if (r >= nr) rr = 0.f;
 #pragma unroll
-                for (int k = 0; k < KPT; ++k) {
-                    acc[k].x += rr * xf[r][k].x; acc[k].y += rr * xf[r][k].y;
-                    acc[k].z += rr * xf[r][k].z; acc[k].w += rr * xf[r][k].w;
-                }
+            for (int k = 0; k < KPT; ++k) {
+                acc[k].x = fmaf(rr, xf[r][k].x, acc[k].x); acc[k].y = fmaf(rr, xf[r][k].y, acc[k].y);
+                acc[k].z = fmaf(rr, xf[r][k].z, acc[k].z); acc[k].w = fmaf(rr, xf[r][k].w, acc[k].w);
             }
         }
+        if (++stage == S) { stage = 0; phase ^= 1u; }
         ++done;
     }
     if (done < nblocks) {
@@ -2102,7 +2188,7 @@ cudaError_t launch_partial_gradients_fused(const float *X, const float *y, const
     // few items (coded gradients of a small tree): a cluster of 16 fills more of the GPU
     if (csplit == 8 && items * 8 < 2 * dev.sm_count && item_blocks / 16 >= 4) csplit = 16;
     if (tune.pg_cluster) csplit = tune.pg_cluster;
-    const size_t smem = (size_t)stages * RB * d * 4 + (size_t)d * 4 + (size_t)2 * rbc * 8 * 4 + (size_t)stages * 8 + 16;
+    const size_t smem = (size_t)stages * RB * d * 4 + (size_t)d * 4 + (size_t)2 * pg_red_words(kpt) * 4 + (size_t)stages * 8 + 16;
     if (smem > (size_t)dev.smem_optin) return cudaErrorInvalidConfiguration;
     PgArgs pa;
     pa.X = X; pa.y = y; pa.w = w; pa.part = part; pa.order = slots_per_item == 1 ? order : nullptr; pa.coeff = coeff; pa.G = G; pa.rows = rows;
