@@ -518,7 +518,6 @@ cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchA
     }
     __syncthreads();
 
-    const T *coeff = reinterpret_cast<const T *>(a.coeff);
     const uint32_t stage_bytes = (uint32_t)(stage_elems * sizeof(T));
 
     if (warp < NLW) {
