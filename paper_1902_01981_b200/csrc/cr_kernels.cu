@@ -1329,21 +1329,17 @@ __device__ __forceinline__ void pg_warp_sums(const float (&part)[R], float *redb
     }
 }
 
-// The residual sums of the block's rows from the eight warps' partial sums: lane l reads the entry of row
-// l >> 3 and warp l & 7 of each chunk, three exchange steps add the eight warps, and a shuffle hands every
-// lane the sum of each row (10 instructions per chunk against 2 loads and 7 additions per row).
+// The residual sums of the block's rows from the eight warps' partial sums: every thread reads the eight
+// values of each row (two broadcast loads) and adds them as a tree.  (Letting lane l read one entry and
+// adding across lanes takes a third of the instructions but four dependent shuffles; the block's time
+// is set by the length of this chain, not by the instruction count.)
 template <int R>
 __device__ __forceinline__ void pg_block_sums(const float *redb, int lane, float (&z)[R]) {
-    constexpr unsigned FULL = 0xffffffffu;
 #pragma unroll
-    for (int c = 0; c < (R + 3) / 4; ++c) {
-        float v = redb[c * 32 + lane];
-        v += __shfl_xor_sync(FULL, v, 4);
-        v += __shfl_xor_sync(FULL, v, 2);
-        v += __shfl_xor_sync(FULL, v, 1);
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-            if (4 * c + j < R) z[4 * c + j] = __shfl_sync(FULL, v, j * 8);
+    for (int r = 0; r < R; ++r) {
+        const float4 p0 = *reinterpret_cast<const float4 *>(redb + (r / 4) * 32 + (r % 4) * 8);
+        const float4 p1 = *reinterpret_cast<const float4 *>(redb + (r / 4) * 32 + (r % 4) * 8 + 4);
+        z[r] = ((p0.x + p0.y) + (p0.z + p0.w)) + ((p1.x + p1.y) + (p1.z + p1.w));
     }
 }
 
