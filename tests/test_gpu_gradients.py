@@ -35,6 +35,9 @@ CASES = [dict(n=3, L=2, s=1, P=15, d=512, code="printed_3_1", rows=37),      # o
          dict(n=4, L=2, s=1, P=24, d=1000, code="cyclic", rows=100),          # cluster of CTAs, d not a power of two
          dict(n=4, L=2, s=1, P=48, d=4096, code="cyclic", rows=64),
          dict(n=5, L=1, s=2, P=5, d=8192, code="cyclic", rows=50),            # widest one-pass case
+         dict(n=4, L=2, s=1, P=24, d=2048, code="cyclic", rows=33),           # two column groups per thread, six-row blocks, ragged
+         dict(n=3, L=2, s=1, P=15, d=6000, code="printed_3_1", rows=25),      # six groups, the last one partly beyond d
+         dict(n=4, L=2, s=1, P=24, d=6500, code="cyclic", rows=19),           # seven groups, one-row blocks (a model size of Section V)
          dict(n=3, L=2, s=1, P=15, d=1027, code="printed_3_1", rows=21)]      # two-pass path (d % 4 != 0)
 
 
