@@ -468,8 +468,10 @@ __device__ __forceinline__ void full_box_rows(const T *src, const uint32_t (&cb)
 
 // SHARE: the instance that forms shared messages first; the other one is free of that code and of its
 // registers (a node's children live in registers while its variants are formed).
+// The eight-warp form (four loaders, four replay warps) is held to 128 registers so that two CTAs share an SM
+// when the union is small: a tile of a small tree is a short chain of waits, and two chains overlap.
 template <typename T, int LMAX, int NLW, int NRW, bool SHARE>
-__global__ void __launch_bounds__((NLW + NRW) * 32, 1)
+__global__ void __launch_bounds__((NLW + NRW) * 32, (NLW + NRW) <= 8 ? 2 : 1)
 cr_fused_batch_tma_kernel(const __grid_constant__ CUtensorMap tmap, const BatchArgs a) {
     constexpr int TILE = 128;
     constexpr int NP = LMAX <= 4 ? 4 : 2;  // patterns replayed together by one warp
@@ -1786,9 +1788,10 @@ static cudaError_t run_batch_l(int lmax, const CUtensorMap &map, const BatchArgs
 template <typename T>
 static cudaError_t run_batch_w(int nlw, int nrw, int lmax, const CUtensorMap &map, const BatchArgs &ba, int grid,
                                size_t smem, cudaStream_t stream) {
-    if (ba.n_ops)   // shared messages: eight replay warps always
+    if (ba.n_ops)   // shared messages: eight replay warps, or four in the two-CTAs-per-SM form
         return nlw == 6 ? run_batch_l<T, 6, 8, true>(lmax, map, ba, grid, smem, stream)
-                        : run_batch_l<T, 4, 8, true>(lmax, map, ba, grid, smem, stream);
+                        : (nrw == 4 ? run_batch_l<T, 4, 4, true>(lmax, map, ba, grid, smem, stream)
+                                    : run_batch_l<T, 4, 8, true>(lmax, map, ba, grid, smem, stream));
     if (nlw == 6) return nrw == 4 ? run_batch_l<T, 6, 4, false>(lmax, map, ba, grid, smem, stream)
                                   : run_batch_l<T, 6, 8, false>(lmax, map, ba, grid, smem, stream);
     return nrw == 4 ? run_batch_l<T, 4, 4, false>(lmax, map, ba, grid, smem, stream)
@@ -1864,7 +1867,17 @@ BatchShape batch_shape(const AggArgs &a, const DeviceInfo &dev, const Tuning &tu
         smem += vtab_bytes;
     }
     const long long ntiles = (a.d + tile - 1) / tile;
-    const int grid = (int)std::min<long long>(ntiles, (long long)std::max(1, dev.sm_count));
+    int grid = (int)std::min<long long>(ntiles, (long long)std::max(1, dev.sm_count));
+    // Small unions: with four loaders and four replay warps two CTAs fit an SM (shared memory and registers),
+    // and a CTA's tile -- a handful of boxes, then the replay, each a chain of waits -- overlaps the other's.
+    // Measured, 16 patterns on the (4,2,1) tree at d = 2^20: one CTA of 14 warps per SM 0.138 ms.
+    if (!tune.ncw && !tune.ctas_per_sm && nbuf == 2) {
+        const size_t smem4 = smem - (size_t)(nlw - 4) * stages * (stage_bytes + 8);
+        if (smem4 + 1024 <= (size_t)dev.smem_per_sm / 2 && ntiles >= 4ll * dev.sm_count) {
+            nlw = 4; sh.nrw = 4; smem = smem4;
+            grid = (int)std::min<long long>(ntiles, 2ll * dev.sm_count);
+        }
+    }
     sh.cpn = multi ? 1 : a.m / R;
     sh.n_groups = multi ? a.n_boxes : a.n_union;
     // box counters are 32-bit

@@ -46,6 +46,10 @@ def aggregate(plan, G_dev, masks, d, flags=B.CR_AGG_FUSED, dtype=torch.float32):
     (tree(6, 2, 2, "repetition", 1300), 16, "i32", True),     # 0/1 code: few children consulted, most of the union unused
     (tree(16, 2, 1, "repetition", 520), 9, "f32", False),     # widest parents
     (tree(2, 5, 1, "cyclic", 900), 12, "f32", False),         # L = 5: the eight-layer instance
+    # small unions over many tiles: the form with two CTAs of eight warps per SM
+    (tree(4, 2, 1, "cyclic", 77060), 16, "f32", False),
+    (tree(3, 2, 1, "printed_3_1", 80004), 5, "i32", False),
+    (tree(5, 2, 2, "cyclic", 76804, P=80), 12, "f32", True),
 ])
 def test_shared_messages_match_the_oracle(cfg, batch, dtype, exactly):
     n, L, s, d = cfg["n"], cfg["L"], cfg["s"], cfg["d"]
