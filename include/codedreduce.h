@@ -322,7 +322,9 @@ cr_status_t cr_aggregate_bytes(const cr_plan_t *plan, const uint32_t *masks_host
  * of the shared-memory ring (2..16), ctas_per_sm = persistent CTAs per SM (1..8), rows_per_box = slot
  * rows per TMA box (must divide m, at most 16).  Batch kernel (one CTA per SM): consumer_warps = replay
  * warps (4 or 8), stages = boxes per loader warp, ctas_per_sm = loader warps (4 or 6), rows_per_box as
- * above.  Shapes that do not fit shared memory fall back to smaller ones or to plain loads. */
+ * above.  With both left at 0, a batch whose union is small enough for two CTAs of eight warps (four loaders,
+ * four replay warps) to share an SM runs in that form.  Shapes that do not fit shared memory fall back to
+ * smaller ones or to plain loads. */
 cr_status_t cr_plan_tune(cr_plan_t *plan, int32_t consumer_warps, int32_t stages, int32_t ctas_per_sm,
                          int32_t rows_per_box);
 
