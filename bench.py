@@ -446,6 +446,34 @@ class AggregateSetup:
                 "ctypes_call_that_launches_nothing": float(np.median(trivial)) * 1e-3,
                 "note": "host clock around the call through the Python binding, stream idle, median of %d" % calls}
 
+    def graph_replay_ms(self, flags, reps=100):
+        """Device time of one scheduled call replayed as a CUDA graph (one fixed pattern): the launch-bound
+        end of the table without the host in the loop."""
+        torch, B = self.torch, self.B
+        sched = B.cr_schedule_create(self.plan, self.masks[0], flags)
+        try:
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                B.cr_aggregate_scheduled(self.plan, self.G_slots, sched, self.out, None, torch.cuda.current_stream())
+            for _ in range(3):
+                graph.replay()
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            tt = []
+            for i in range(reps):
+                if self.flush is not None:
+                    self.flush(i)
+                a.record()
+                graph.replay()
+                b.record()
+                torch.cuda.synchronize()
+                tt.append(a.elapsed_time(b))
+            return float(np.median(tt))
+        finally:
+            B.cr_schedule_destroy(sched)
+
     def parity_on_sample(self, cols, flags, patterns=2):
         """The GPU result on the first `cols` columns against the CPU oracle for the last straggler patterns:
         worst relative L2 error (fp32) or exact equality (int32)."""
@@ -655,6 +683,12 @@ def run_ours(args, cfg):
             extras["unfused_per_level"] = {"GB/s": bytes_k / float(p2.mean()) / 1e9, "ms_per_step": float(p2.mean()) * 1e3}
             del wsb
         host_cost = ws0.host_cost_us(B.CR_AGG_FUSED)
+        try:    # short launches: the same call captured once in a CUDA graph and replayed
+            host_cost["graph_replay_ms"] = ws0.graph_replay_ms(B.CR_AGG_FUSED)
+        except Exception as exc:
+            host_cost["graph_replay_ms"] = None
+            host_cost["graph_replay_unavailable"] = repr(exc)[:200]
+            torch.cuda.synchronize()
 
     # ---- end to end through the host-buffer entry point: H2D of the slots and D2H of the result
     # inside the timed region
@@ -839,6 +873,55 @@ def run_linreg(args, cfg):
         e2e_sec = (time.perf_counter() - t0) / e2e_steps
         e2e = {"value": step_bytes / e2e_sec / 1e9, "unit": UNIT, "h2d_bytes_per_step": int(4 * d + masks[0].nbytes),
                "d2h_bytes_per_step": int(4 * d), "steps": e2e_steps, "ms_per_step": e2e_sec * 1e3}
+    # The same step as one CUDA graph (gradients, aggregation with a schedule made beforehand, model update),
+    # replayed: what a launch-bound step costs once the host is out of the loop.  A graph bakes its arguments
+    # in, so every replay runs the straggler pattern of the schedule it was captured with.
+    graph_leg = None
+    if not args.no_extras:
+        try:
+            agg_flags = (B.CR_AGG_FUSED | B.CR_AGG_FROM_CODED) if coded else B.CR_AGG_FUSED
+            sched = B.cr_schedule_create(plan, masks[0], agg_flags)
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                cs = torch.cuda.current_stream()
+                if coded:
+                    B.cr_coded_gradients(plan, loss, X_dev, y_dev, rows, w_dev, E_coded, cs)
+                else:
+                    B.cr_partial_gradients_loss(plan, loss, X_dev, y_dev, rows, w_dev, G_slots, ws, cs)
+                B.cr_aggregate_scheduled(plan, E_coded if coded else G_slots, sched, out, None, cs)
+                w_dev.sub_(out[0], alpha=lr_eff)
+            w_keep = w_dev.clone()
+            reps = max(20, min(args.steps, 200))
+            for _ in range(3):
+                graph.replay()
+            torch.cuda.synchronize()
+            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            if flush is None:
+                g0.record()
+                for _ in range(reps):
+                    graph.replay()
+                g1.record()
+                torch.cuda.synchronize()
+                graph_ms = g0.elapsed_time(g1) / reps
+            else:   # data that fit L2 are flushed before every replay, each timed by itself
+                tt = []
+                for i in range(reps):
+                    flush(i)
+                    g0.record()
+                    graph.replay()
+                    g1.record()
+                    torch.cuda.synchronize()
+                    tt.append(g0.elapsed_time(g1))
+                graph_ms = float(np.mean(tt))
+            w_dev.copy_(w_keep)
+            B.cr_schedule_destroy(sched)
+            graph_leg = {"ms_per_step": graph_ms, "iterations_per_s": 1e3 / graph_ms, "replays": reps,
+                         "note": "one CUDA graph per step (gradient kernels, scheduled aggregation, update), one fixed straggler pattern"}
+        except Exception as exc:   # a capture that the runtime refuses is reported, not fatal
+            graph_leg = {"unavailable": repr(exc)[:200]}
+            torch.cuda.synchronize()
     cpu = None
     if not args.no_cpu_baseline:
         sec, nbytes, sample = oracle_regression_sample(args.workload, cfg, args.cpu_steps, 1, 15.0)
@@ -864,7 +947,7 @@ def run_linreg(args, cfg):
                      "dram_frac": (traffic["bytes"] / float(t_grad.mean()) / 1e9 / peak) if traffic else None,
                      "algorithmic_bytes_per_launch": grad_bytes, "avg_launch_ms": float(t_grad.mean()) * 1e3,
                      "aggregate_ms": float((t_step - t_grad).mean()) * 1e3},
-        "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+        "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks, "graph_replay": graph_leg,
         "normalized_error_rate": float(np.sum((w_final - w_star) ** 2) / np.sum(w_star ** 2)),
     }
     print(json.dumps(line), flush=True)

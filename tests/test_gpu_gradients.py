@@ -128,3 +128,45 @@ def test_logistic_regression_descent_on_paper_shaped_data():
         assert B.cr_plan_device_status(plan) == B.CR_OK
     finally:
         B.cr_plan_destroy(plan)
+
+
+def test_a_step_captured_in_a_cuda_graph_equals_the_direct_step():
+    """Gradients + scheduled aggregation enqueue kernels only (no copy, no wait, no allocation), so a step
+    can be captured in a CUDA graph; its replay must give the bits of the direct calls, and the oracle's
+    gradient within the bar."""
+    cfg = dict(n=4, L=2, s=1, P=24, d=1000, code="cyclic", rows=100)
+    P, d, rows = cfg["P"], cfg["d"], cfg["rows"]
+    plan = make_plan(cfg)
+    try:
+        code, local = check_slot_table(plan, cfg)
+        X, y, w = make_data(B.CR_LOSS_SQUARED, P, rows, d, seed=11)
+        N, m = B.cr_plan_num_nodes(plan), B.cr_plan_load(plan)
+        X_dev, y_dev, w_dev = torch.from_numpy(X).cuda(), torch.from_numpy(y).cuda(), torch.from_numpy(w).cuda()
+        G_slots = torch.zeros((N, m, d), device="cuda")
+        ws = torch.empty(max(16, B.cr_partial_gradients_workspace_bytes(plan, rows)), dtype=torch.uint8, device="cuda")
+        mask = inputs.straggler_masks(cfg["n"], cfg["L"], cfg["s"], 1, seed=5, exactly_s=True)[0]
+        direct = torch.zeros((1, d), device="cuda")
+        B.cr_partial_gradients_loss(plan, B.CR_LOSS_SQUARED, X_dev, y_dev, rows, w_dev, G_slots, ws)
+        B.cr_aggregate(plan, G_slots, mask, direct, B.CR_AGG_FUSED)
+        torch.cuda.synchronize()
+        sched = B.cr_schedule_create(plan, mask, B.CR_AGG_FUSED)
+        out = torch.zeros((1, d), device="cuda")
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            cs = torch.cuda.current_stream()
+            B.cr_partial_gradients_loss(plan, B.CR_LOSS_SQUARED, X_dev, y_dev, rows, w_dev, G_slots, ws, cs)
+            B.cr_aggregate_scheduled(plan, G_slots, sched, out, None, cs)
+        G_slots.zero_()
+        out.zero_()
+        for _ in range(2):
+            graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(out, direct)
+        parts = oracle_parts(B.CR_LOSS_SQUARED, X, y, w)
+        assert rel_l2(out[0].cpu().numpy(), O.execute(code, local, parts, mask)) <= REL_L2_BAR
+        assert B.cr_plan_device_status(plan) == B.CR_OK
+        B.cr_schedule_destroy(sched)
+    finally:
+        B.cr_plan_destroy(plan)
