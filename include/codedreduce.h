@@ -293,6 +293,9 @@ cr_status_t cr_aggregate(cr_plan_t *plan, const void *G_slots, const uint32_t *m
  * validated or expanded, nothing is allocated and nothing is copied.  A schedule belongs to its plan,
  * may be used any number of times, by one stream at a time like the plan itself, and must be destroyed
  * before the plan.  Results are those of cr_aggregate with the same masks and flags, bit for bit.
+ * Since it only enqueues kernels, a cr_aggregate_scheduled call (and a cr_partial_gradients_loss call in
+ * front of it) may be captured in a CUDA graph on a capturing stream and replayed; the graph then holds
+ * the schedule, the buffers and the plan by address, so they must outlive it.
  * cr_schedule_bytes: the algorithmic bytes of one call (as cr_aggregate_bytes). */
 cr_status_t cr_schedule_create(cr_plan_t *plan, const uint32_t *masks_host, int32_t batch, uint32_t flags,
                                cr_schedule_t **out);
